@@ -1,0 +1,146 @@
+/*
+ * civic.h -- C ABI of the CIVIC select + compact + KV-compaction library (CUDA, sm_100a).
+ *
+ * The library implements one hot path of CIVIC's compact inference pathway: deciding which
+ * visual tokens survive, and packing the survivors' rows into contiguous, order-preserving
+ * buffers so that no later stage reads non-contiguous memory.
+ *
+ * Conventions for every call
+ *   - "dev" pointers are CUDA device pointers, "host" pointers ordinary host memory.
+ *   - All buffers are owned by the caller.  Inputs are never written.  Outputs must not
+ *     overlap inputs (checked where both extents are known; overlap -> CIVIC_ERR_INVALID_ARG).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *     enqueued on it and the call returns without synchronising.  The library allocates no
+ *     device memory and keeps no state between calls.
+ *   - Arguments are validated on the host BEFORE anything is launched; on any status other
+ *     than CIVIC_OK nothing was enqueued.  CIVIC_ERR_CUDA wraps a failed launch or attribute
+ *     call (the CUDA error string is available from civic_last_cuda_error()).
+ *   - There are no data-dependent errors: whether the retention floor fits into the budget
+ *     depends on shapes only.  The validity of index arrays passed to the compaction calls
+ *     (in range, one row per output row) is the caller's contract, as they normally come
+ *     straight from civic_select / civic_seq_indices.
+ *   - A token grid is (t, h, w), token index i = (tt*h + hh)*w + ww (row-major), n = t*h*w.
+ */
+#ifndef CIVIC_H_
+#define CIVIC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CIVIC_OK = 0,
+    CIVIC_ERR_INVALID_ARG = 1,     /* null pointer, negative size, inconsistent shapes, overlap   */
+    CIVIC_ERR_K_RANGE = 2,         /* k < 0 or k > n                                              */
+    CIVIC_ERR_FLOOR_EXCEEDS_K = 3, /* sum over regions of min(m, |region|) > k                    */
+    CIVIC_ERR_ALIGNMENT = 4,       /* row size or pointer not a multiple of 4 bytes               */
+    CIVIC_ERR_UNSUPPORTED = 5,     /* segment too large for one thread block's shared memory      */
+    CIVIC_ERR_CUDA = 6             /* a CUDA runtime call failed                                  */
+} civic_status_t;
+
+/* Selection problem of ONE segment (an image or a video); every segment of a call shares it.
+ * The retention floor tiles each temporal slice of the grid into region_h x region_w token
+ * tiles (edge tiles are smaller when h or w is not a multiple) and keeps at least
+ * floor_per_region tokens of every tile (all of a tile that has fewer).  Regions never span t. */
+typedef struct {
+    int32_t t, h, w;            /* token grid, all >= 1                                           */
+    int32_t region_h, region_w; /* tile of the floor in tokens, both >= 1                         */
+    int32_t floor_per_region;   /* m >= 0; 0 = plain top-K                                        */
+    int32_t k;                  /* tokens kept per segment, 0 <= k <= n                           */
+} civic_select_desc_t;
+
+/*
+ * civic_select -- which visual tokens survive.
+ *
+ * Paper: score-rank token dropping (Table 1 caption), selection as a routing overhead
+ * (Eq. 3), kept under the "adaptive spatial retention floor" (Sections 1, 4.5; Table 2
+ * "Min Keep Ratio").  The paper gives no algorithm for the floor; this call implements:
+ *   order    token a beats token b iff score[a] > score[b], or the scores are equal and
+ *            a < b.  Scores are compared in IEEE-754 totalOrder (-0 < +0, NaNs at the ends).
+ *   reserve  in every region its min(m, |region|) best tokens;
+ *   fill     the k - (number reserved) best of the remaining tokens of the segment;
+ *   output   the union as ASCENDING segment-local token indices, exactly k per segment.
+ *
+ * scores    dev  [n_seg, n] fp32, contiguous
+ * desc      host
+ * keep_idx  dev  [n_seg, k] int32, written
+ * One thread block handles one segment with its keys in shared memory:
+ * n <= civic_select_max_tokens() or CIVIC_ERR_UNSUPPORTED.  n_seg == 0 or k == 0 enqueue
+ * nothing and return CIVIC_OK.
+ */
+civic_status_t civic_select(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                            int32_t* keep_idx, void* stream);
+
+/* Largest n = t*h*w that civic_select accepts. */
+int32_t civic_select_max_tokens(void);
+
+/* Number of tokens the floor reserves per segment (shape-only); -1 on invalid arguments. */
+int64_t civic_reserved_count(const civic_select_desc_t* desc);
+
+/*
+ * civic_compact -- pack the surviving tokens' hidden rows and 3-D position ids.
+ *
+ * Paper: Section 3.5 -- the compact visual sequence V_c (Eq. 12) is contiguous, and compact
+ * visual positions are inherited from the dense span (copied, not renumbered).
+ *   hidden_out[s, j, :] = hidden[s, keep_idx[s, j], :]      rows of row_bytes opaque bytes
+ *   pos_out[s, j, :]    = pos_ids[s, keep_idx[s, j], :]     rows of 3 int32
+ *
+ * hidden      dev [n_seg, n, row_bytes] or NULL (then hidden_out must be NULL)
+ * row_bytes   multiple of 4; multiples of 16 with 16-byte aligned buffers take the fast path
+ * pos_ids     dev [n_seg, n, 3] int32 or NULL (then pos_out must be NULL)
+ * keep_idx    dev [n_seg, k] int32, values in [0, n)
+ * Both payloads are moved by ONE launch.
+ */
+civic_status_t civic_compact(const void* hidden, size_t row_bytes, const int32_t* pos_ids,
+                             const int32_t* keep_idx, int32_t n_seg, int32_t n, int32_t k,
+                             void* hidden_out, int32_t* pos_out, void* stream);
+
+/*
+ * civic_seq_indices -- kept rows of the full multimodal sequence.
+ *
+ * Paper: Eq. 13 (the compact prefill replaces the dense visual span by the compact one,
+ * length L + M_p) and Section 3.5 (text positions are preserved).  The visual span of every
+ * sequence is [vis_start, vis_start + n_vis); all positions outside it are text and always
+ * kept.   seq_idx[s, :] = ascending( text positions  U  vis_start + keep_idx[s, :] ).
+ *
+ * keep_idx  dev [n_seq, k] int32 ascending, values in [0, n_vis)
+ * seq_idx   dev [n_seq, seq_len - n_vis + k] int32, written
+ */
+civic_status_t civic_seq_indices(const int32_t* keep_idx, int32_t n_seq, int32_t k, int32_t seq_len,
+                                 int32_t vis_start, int32_t n_vis, int32_t* seq_idx, void* stream);
+
+/*
+ * civic_compact_kv -- pack every layer's prefill K and V rows of the kept positions.
+ *
+ * Paper: the KV-cache storage term of Eq. 2 / Eq. 7 and the cache ratio (L+M_p)/(L+T_p) of
+ * Eq. 14: the compact cache holds exactly the kept rows, contiguously, in source order.
+ *   k_dst[l][s, j, :] = k_src[l][s, seq_idx[s, j], :]   (same for v), l < n_layers
+ *
+ * k_src, v_src  host arrays of n_layers dev pointers, each [n_seq, seq_len, row_bytes]
+ * k_dst, v_dst  host arrays of n_layers dev pointers, each [n_seq, s_out,  row_bytes]
+ * row_bytes     bytes of one token's row (kv_heads * head_dim * element size), multiple of 4
+ * seq_idx       dev [n_seq, s_out] int32, values in [0, seq_len); shared by all layers
+ * The pointer tables are read during the call only (copied into kernel parameters).  All
+ * layers and both of K and V are moved by one launch per 80 layers.
+ */
+civic_status_t civic_compact_kv(const void* const* k_src, const void* const* v_src,
+                                void* const* k_dst, void* const* v_dst, int32_t n_layers,
+                                int32_t n_seq, int32_t seq_len, int32_t s_out, size_t row_bytes,
+                                const int32_t* seq_idx, void* stream);
+
+/* Static, human-readable name of a status. */
+const char* civic_status_string(civic_status_t status);
+
+/* Text of the CUDA error behind the calling thread's last CIVIC_ERR_CUDA ("" if none). */
+const char* civic_last_cuda_error(void);
+
+/* Kernels this library enqueued since it was loaded (all threads). */
+uint64_t civic_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CIVIC_H_ */

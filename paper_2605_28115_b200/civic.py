@@ -1,0 +1,241 @@
+"""Thin ctypes binding of libcivic.so: argument marshalling only.
+
+Every step of the path runs inside the CUDA library; torch is used for device memory and
+streams.  The functions carry the names of the C entry points (include/civic.h).  There is
+no CPU fallback: if the library cannot be loaded, or a tensor is not on a CUDA device,
+the call raises.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcivic.so")
+
+CIVIC_OK = 0
+STATUS_NAMES = ("CIVIC_OK", "CIVIC_ERR_INVALID_ARG", "CIVIC_ERR_K_RANGE", "CIVIC_ERR_FLOOR_EXCEEDS_K",
+                "CIVIC_ERR_ALIGNMENT", "CIVIC_ERR_UNSUPPORTED", "CIVIC_ERR_CUDA")
+
+# every symbol include/civic.h declares
+EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "civic_compact",
+           "civic_seq_indices", "civic_compact_kv", "civic_status_string", "civic_last_cuda_error",
+           "civic_launch_count")
+
+
+class CivicError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name}{(' (' + detail + ')') if detail else ''}")
+        self.status = status
+
+
+class SelectDesc(ctypes.Structure):
+    """civic_select_desc_t"""
+    _fields_ = [("t", ctypes.c_int32), ("h", ctypes.c_int32), ("w", ctypes.c_int32),
+                ("region_h", ctypes.c_int32), ("region_w", ctypes.c_int32),
+                ("floor_per_region", ctypes.c_int32), ("k", ctypes.c_int32)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load libcivic.so (built in-tree by paper_2605_28115_b200.build). Raises if missing."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} not found: build it with `python -m paper_2605_28115_b200.build` "
+                           "(there is no fallback implementation)")
+    lib = ctypes.CDLL(path)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    vpp = ctypes.POINTER(ctypes.c_void_p)
+    lib.civic_select.argtypes = [vp, i32, ctypes.POINTER(SelectDesc), vp, vp]
+    lib.civic_select.restype = ctypes.c_int
+    lib.civic_select_max_tokens.argtypes = []
+    lib.civic_select_max_tokens.restype = i32
+    lib.civic_reserved_count.argtypes = [ctypes.POINTER(SelectDesc)]
+    lib.civic_reserved_count.restype = ctypes.c_int64
+    lib.civic_compact.argtypes = [vp, sz, vp, vp, i32, i32, i32, vp, vp, vp]
+    lib.civic_compact.restype = ctypes.c_int
+    lib.civic_seq_indices.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp]
+    lib.civic_seq_indices.restype = ctypes.c_int
+    lib.civic_compact_kv.argtypes = [vpp, vpp, vpp, vpp, i32, i32, i32, i32, sz, vp, vp]
+    lib.civic_compact_kv.restype = ctypes.c_int
+    lib.civic_status_string.argtypes = [ctypes.c_int]
+    lib.civic_status_string.restype = ctypes.c_char_p
+    lib.civic_last_cuda_error.argtypes = []
+    lib.civic_last_cuda_error.restype = ctypes.c_char_p
+    lib.civic_launch_count.argtypes = []
+    lib.civic_launch_count.restype = ctypes.c_uint64
+    _lib = lib
+    return lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != CIVIC_OK:
+        detail = load().civic_last_cuda_error().decode() if status == 6 else ""
+        raise CivicError(status, where, detail)
+
+
+def _dev_ptr(x: Optional[torch.Tensor], what: str, dtype: Optional[torch.dtype] = None) -> Optional[int]:
+    if x is None:
+        return None
+    if not x.is_cuda:
+        raise ValueError(f"{what} must be a CUDA tensor (no CPU path exists)")
+    if not x.is_contiguous():
+        raise ValueError(f"{what} must be contiguous")
+    if dtype is not None and x.dtype != dtype:
+        raise ValueError(f"{what} must be {dtype}, got {x.dtype}")
+    return x.data_ptr()
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+def launch_count() -> int:
+    return int(load().civic_launch_count())
+
+
+def select_max_tokens() -> int:
+    return int(load().civic_select_max_tokens())
+
+
+def reserved_count(desc: SelectDesc) -> int:
+    return int(load().civic_reserved_count(ctypes.byref(desc)))
+
+
+def civic_select(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optional[torch.Tensor] = None,
+                 stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """scores fp32 [n_seg, n] (CUDA) -> ascending keep indices int32 [n_seg, k]."""
+    if scores.dim() != 2 or scores.shape[1] != desc.t * desc.h * desc.w:
+        raise ValueError("scores must be [n_seg, t*h*w]")
+    n_seg = scores.shape[0]
+    if keep_idx is None:
+        keep_idx = torch.empty((n_seg, max(desc.k, 0)), dtype=torch.int32, device=scores.device)
+    elif tuple(keep_idx.shape) != (n_seg, desc.k):
+        raise ValueError("keep_idx must be [n_seg, k]")
+    args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
+            _dev_ptr(keep_idx, "keep_idx", torch.int32))
+    with torch.cuda.device(scores.device):
+        _check(load().civic_select(*args, _stream_ptr(stream)), "civic_select")
+    return keep_idx
+
+
+def civic_compact(hidden: Optional[torch.Tensor], pos_ids: Optional[torch.Tensor], keep_idx: torch.Tensor,
+                  hidden_out: Optional[torch.Tensor] = None, pos_out: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None):
+    """hidden [n_seg, n, D] (any dtype), pos_ids int32 [n_seg, n, 3] -> ([n_seg, k, D], [n_seg, k, 3])."""
+    n_seg, k = keep_idx.shape
+    n = None
+    row_bytes = 0
+    if hidden is not None:
+        if hidden.dim() != 3 or hidden.shape[0] != n_seg:
+            raise ValueError("hidden must be [n_seg, n, D]")
+        n = hidden.shape[1]
+        row_bytes = hidden.shape[2] * hidden.element_size()
+        if hidden_out is None:
+            hidden_out = torch.empty((n_seg, k, hidden.shape[2]), dtype=hidden.dtype, device=hidden.device)
+        elif tuple(hidden_out.shape) != (n_seg, k, hidden.shape[2]) or hidden_out.dtype != hidden.dtype:
+            raise ValueError("hidden_out must be [n_seg, k, D] of hidden's dtype")
+    if pos_ids is not None:
+        if pos_ids.dim() != 3 or pos_ids.shape[0] != n_seg or pos_ids.shape[2] != 3:
+            raise ValueError("pos_ids must be [n_seg, n, 3]")
+        if n is not None and pos_ids.shape[1] != n:
+            raise ValueError("hidden and pos_ids disagree on n")
+        n = pos_ids.shape[1]
+        if pos_out is None:
+            pos_out = torch.empty((n_seg, k, 3), dtype=torch.int32, device=pos_ids.device)
+        elif tuple(pos_out.shape) != (n_seg, k, 3):
+            raise ValueError("pos_out must be [n_seg, k, 3]")
+    if n is None:
+        raise ValueError("nothing to compact")
+    args = (_dev_ptr(hidden, "hidden"), row_bytes, _dev_ptr(pos_ids, "pos_ids", torch.int32),
+            _dev_ptr(keep_idx, "keep_idx", torch.int32), n_seg, n, k,
+            _dev_ptr(hidden_out, "hidden_out"), _dev_ptr(pos_out, "pos_out", torch.int32))
+    with torch.cuda.device(keep_idx.device):
+        _check(load().civic_compact(*args, _stream_ptr(stream)), "civic_compact")
+    return hidden_out, pos_out
+
+
+def civic_seq_indices(keep_idx: torch.Tensor, seq_len: int, vis_start: int, n_vis: int,
+                      seq_idx: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """keep_idx int32 [n_seq, k] -> kept positions of the full sequence int32 [n_seq, seq_len-n_vis+k]."""
+    n_seq, k = keep_idx.shape
+    s_out = seq_len - n_vis + k
+    if seq_idx is None:
+        seq_idx = torch.empty((n_seq, max(s_out, 0)), dtype=torch.int32, device=keep_idx.device)
+    elif tuple(seq_idx.shape) != (n_seq, s_out):
+        raise ValueError("seq_idx must be [n_seq, seq_len - n_vis + k]")
+    args = (_dev_ptr(keep_idx, "keep_idx", torch.int32), n_seq, k, seq_len, vis_start, n_vis,
+            _dev_ptr(seq_idx, "seq_idx", torch.int32))
+    with torch.cuda.device(keep_idx.device):
+        _check(load().civic_seq_indices(*args, _stream_ptr(stream)), "civic_seq_indices")
+    return seq_idx
+
+
+@dataclasses.dataclass
+class KVTables:
+    """Host pointer tables for civic_compact_kv, built once per set of cache tensors."""
+    k_src: ctypes.Array
+    v_src: ctypes.Array
+    k_dst: ctypes.Array
+    v_dst: ctypes.Array
+    n_layers: int
+    n_seq: int
+    seq_len: int
+    s_out: int
+    row_bytes: int
+    keepalive: tuple
+
+
+def kv_tables(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
+              k_dst: Sequence[torch.Tensor], v_dst: Sequence[torch.Tensor]) -> KVTables:
+    """Marshal per-layer tensors ([n_seq, seq_len, ...] -> [n_seq, s_out, ...]) into pointer tables."""
+    n_layers = len(k_src)
+    if not (len(v_src) == len(k_dst) == len(v_dst) == n_layers):
+        raise ValueError("the four tensor lists must have one entry per layer")
+    if n_layers == 0:
+        raise ValueError("no layers")
+    src_shape, dst_shape = tuple(k_src[0].shape), tuple(k_dst[0].shape)
+    for a in list(k_src) + list(v_src):
+        if tuple(a.shape) != src_shape or a.dtype != k_src[0].dtype:
+            raise ValueError("all source tensors must share shape and dtype")
+    for a in list(k_dst) + list(v_dst):
+        if tuple(a.shape) != dst_shape or a.dtype != k_src[0].dtype:
+            raise ValueError("all destination tensors must share shape and dtype")
+    if len(src_shape) < 3 or src_shape[0] != dst_shape[0] or src_shape[2:] != dst_shape[2:]:
+        raise ValueError("source [n_seq, seq_len, ...] and destination [n_seq, s_out, ...] disagree")
+    row_elems = 1
+    for d in src_shape[2:]:
+        row_elems *= d
+
+    def table(ts, what):
+        return (ctypes.c_void_p * n_layers)(*[_dev_ptr(t, what) for t in ts])
+
+    return KVTables(table(k_src, "k_src"), table(v_src, "v_src"), table(k_dst, "k_dst"),
+                    table(v_dst, "v_dst"), n_layers, src_shape[0], src_shape[1], dst_shape[1],
+                    row_elems * k_src[0].element_size(),
+                    (tuple(k_src), tuple(v_src), tuple(k_dst), tuple(v_dst)))
+
+
+def civic_compact_kv(tables: KVTables, seq_idx: torch.Tensor,
+                     stream: Optional[torch.cuda.Stream] = None) -> None:
+    """k_dst[l][s, j] = k_src[l][s, seq_idx[s, j]] (and V) for every layer, one launch."""
+    if tuple(seq_idx.shape) != (tables.n_seq, tables.s_out):
+        raise ValueError("seq_idx must be [n_seq, s_out]")
+    idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
+    with torch.cuda.device(seq_idx.device):
+        _check(load().civic_compact_kv(tables.k_src, tables.v_src, tables.k_dst, tables.v_dst,
+                                       tables.n_layers, tables.n_seq, tables.seq_len, tables.s_out,
+                                       tables.row_bytes, idx_ptr, _stream_ptr(stream)),
+               "civic_compact_kv")

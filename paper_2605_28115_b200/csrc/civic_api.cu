@@ -1,0 +1,283 @@
+// C ABI of the library: host-side validation and kernel launches.  See include/civic.h
+// for the contract of every entry point.
+#include "../../include/civic.h"
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "gather.cuh"
+#include "select.cuh"
+
+namespace {
+
+constexpr size_t kMaxDynamicSmem = 227 * 1024;
+
+std::atomic<uint64_t> g_launches{0};
+thread_local char g_cuda_error[256] = "";
+
+civic_status_t cuda_fail(cudaError_t e, const char* what)
+{
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    return CIVIC_ERR_CUDA;
+}
+
+#define CIVIC_CUDA_TRY(expr)                                        \
+    do {                                                            \
+        cudaError_t e_ = (expr);                                    \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #expr);         \
+    } while (0)
+
+bool overlaps(const void* a, size_t a_bytes, const void* b, size_t b_bytes)
+{
+    if (!a || !b || a_bytes == 0 || b_bytes == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
+bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+int64_t reserved_count(const civic_select_desc_t& d)
+{
+    if (d.t < 1 || d.h < 1 || d.w < 1 || d.region_h < 1 || d.region_w < 1 || d.floor_per_region < 0)
+        return -1;
+    const int64_t m = d.floor_per_region;
+    const int64_t fh = d.h / d.region_h, eh = d.h % d.region_h;  // full tiles, edge extent
+    const int64_t fw = d.w / d.region_w, ew = d.w % d.region_w;
+    auto take = [m](int64_t size) { return size < m ? size : m; };
+    int64_t per_slice = fh * fw * take((int64_t)d.region_h * d.region_w);
+    if (ew) per_slice += fh * take((int64_t)d.region_h * ew);
+    if (eh) per_slice += fw * take(eh * (int64_t)d.region_w);
+    if (eh && ew) per_slice += take(eh * ew);
+    return per_slice * d.t;
+}
+
+int sm_count()
+{
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int v = cached[dev].load(std::memory_order_relaxed);
+    if (v == 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+            v = 148;
+        cached[dev].store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
+
+// Launch the row gather for up to kMaxGatherTensors tensors sharing one index array.
+civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
+{
+    const long long total_rows = (long long)p.n_tensors * p.n_seq * p.s_out;
+    const bool has_pos = p.pos_src != nullptr;
+    const long long pos_elems = has_pos ? (long long)p.n_seq * p.s_out * 3 : 0;
+    if (total_rows == 0 && pos_elems == 0) return CIVIC_OK;
+
+    const int threads = 256, warps = threads / 32;
+    const int resident = sm_count() * (2048 / threads);
+    long long main_blocks = (total_rows + warps - 1) / warps;
+    if (main_blocks > resident) main_blocks = resident;
+    long long pos_blocks = (pos_elems + threads - 1) / threads;
+    if (pos_blocks > sm_count()) pos_blocks = sm_count();
+    p.main_blocks = (uint32_t)main_blocks;
+    const unsigned grid = (unsigned)(main_blocks + pos_blocks);
+
+    bool vec16 = p.row_bytes % 16 == 0;
+    for (int i = 0; i < p.n_tensors && vec16; ++i)
+        vec16 = aligned(p.src[i], 16) && aligned(p.dst[i], 16);
+    if (vec16)
+        civic::gather_rows_kernel<uint4, 4><<<grid, threads, 0, stream>>>(p);
+    else
+        civic::gather_rows_kernel<uint32_t, 8><<<grid, threads, 0, stream>>>(p);
+    CIVIC_CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* civic_status_string(civic_status_t s)
+{
+    switch (s) {
+        case CIVIC_OK: return "CIVIC_OK";
+        case CIVIC_ERR_INVALID_ARG: return "CIVIC_ERR_INVALID_ARG";
+        case CIVIC_ERR_K_RANGE: return "CIVIC_ERR_K_RANGE";
+        case CIVIC_ERR_FLOOR_EXCEEDS_K: return "CIVIC_ERR_FLOOR_EXCEEDS_K";
+        case CIVIC_ERR_ALIGNMENT: return "CIVIC_ERR_ALIGNMENT";
+        case CIVIC_ERR_UNSUPPORTED: return "CIVIC_ERR_UNSUPPORTED";
+        case CIVIC_ERR_CUDA: return "CIVIC_ERR_CUDA";
+    }
+    return "CIVIC_ERR_UNKNOWN";
+}
+
+const char* civic_last_cuda_error(void) { return g_cuda_error; }
+
+uint64_t civic_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int32_t civic_select_max_tokens(void)
+{
+    // largest n whose keys, reserved bits and histogram fit into one block's shared memory;
+    // the scan also packs two counts of at most n into 16 bits each
+    int32_t words = (int32_t)((kMaxDynamicSmem / sizeof(uint32_t) - (256 + 32 + 4)) / 33);
+    int32_t n = words * 32;
+    return n < 65535 ? n : 65535;
+}
+
+int64_t civic_reserved_count(const civic_select_desc_t* desc)
+{
+    return desc ? reserved_count(*desc) : -1;
+}
+
+civic_status_t civic_select(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                            int32_t* keep_idx, void* stream)
+{
+    if (!desc || n_seg < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n_res = reserved_count(*desc);
+    if (n_res < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)desc->t * desc->h * desc->w;
+    if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (desc->k < 0 || desc->k > n) return CIVIC_ERR_K_RANGE;
+    if (n_res > desc->k) return CIVIC_ERR_FLOOR_EXCEEDS_K;
+    if (n_seg == 0 || desc->k == 0) return CIVIC_OK;
+    if (!scores || !keep_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(scores, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (n > civic_select_max_tokens()) return CIVIC_ERR_UNSUPPORTED;
+    if (overlaps(scores, (size_t)n_seg * n * 4, keep_idx, (size_t)n_seg * desc->k * 4))
+        return CIVIC_ERR_INVALID_ARG;
+
+    civic::SelectParams p;
+    p.scores = scores;
+    p.keep_idx = keep_idx;
+    p.n = (int32_t)n;
+    p.t = desc->t; p.h = desc->h; p.w = desc->w;
+    p.region_h = desc->region_h; p.region_w = desc->region_w;
+    p.m = desc->floor_per_region;
+    p.k = desc->k;
+    p.k_fill = (int32_t)(desc->k - n_res);
+
+    const size_t smem = civic::select_smem_bytes(p.n);
+    if (smem > 48 * 1024)
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int threads = (p.n + 31) / 32 * 32;
+    threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
+    civic::select_kernel<<<(unsigned)n_seg, threads, smem, (cudaStream_t)stream>>>(p);
+    CIVIC_CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+civic_status_t civic_compact(const void* hidden, size_t row_bytes, const int32_t* pos_ids,
+                             const int32_t* keep_idx, int32_t n_seg, int32_t n, int32_t k,
+                             void* hidden_out, int32_t* pos_out, void* stream)
+{
+    if (n_seg < 0 || n < 0 || k < 0) return CIVIC_ERR_INVALID_ARG;
+    if (k > n) return CIVIC_ERR_K_RANGE;
+    if ((hidden == nullptr) != (hidden_out == nullptr)) return CIVIC_ERR_INVALID_ARG;
+    if ((pos_ids == nullptr) != (pos_out == nullptr)) return CIVIC_ERR_INVALID_ARG;
+    if (hidden && (row_bytes == 0 || row_bytes > UINT32_MAX)) return CIVIC_ERR_INVALID_ARG;
+    if (hidden && (row_bytes % 4 || !aligned(hidden, 4) || !aligned(hidden_out, 4)))
+        return CIVIC_ERR_ALIGNMENT;
+    if (!aligned(pos_ids, 4) || !aligned(pos_out, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (n_seg == 0 || k == 0 || (!hidden && !pos_ids)) return CIVIC_OK;
+    if (!keep_idx) return CIVIC_ERR_INVALID_ARG;
+    const size_t in_rows = (size_t)n_seg * n, out_rows = (size_t)n_seg * k;
+    if (overlaps(hidden, in_rows * row_bytes, hidden_out, out_rows * row_bytes) ||
+        overlaps(pos_ids, in_rows * 12, pos_out, out_rows * 12) ||
+        overlaps(keep_idx, out_rows * 4, hidden_out, out_rows * row_bytes) ||
+        overlaps(keep_idx, out_rows * 4, pos_out, out_rows * 12))
+        return CIVIC_ERR_INVALID_ARG;
+
+    civic::GatherParams p;
+    memset(&p, 0, sizeof p);
+    p.n_tensors = hidden ? 1 : 0;
+    p.src[0] = (const char*)hidden;
+    p.dst[0] = (char*)hidden_out;
+    p.idx = keep_idx;
+    p.pos_src = pos_ids;
+    p.pos_dst = pos_out;
+    p.n_seq = n_seg; p.seq_len = n; p.s_out = k;
+    p.row_bytes = hidden ? (uint32_t)row_bytes : 4;
+    return launch_gather(p, (cudaStream_t)stream);
+}
+
+civic_status_t civic_seq_indices(const int32_t* keep_idx, int32_t n_seq, int32_t k, int32_t seq_len,
+                                 int32_t vis_start, int32_t n_vis, int32_t* seq_idx, void* stream)
+{
+    if (n_seq < 0 || k < 0 || seq_len < 0 || vis_start < 0 || n_vis < 0) return CIVIC_ERR_INVALID_ARG;
+    if ((int64_t)vis_start + n_vis > seq_len) return CIVIC_ERR_INVALID_ARG;
+    if (k > n_vis) return CIVIC_ERR_K_RANGE;
+    const int64_t s_out = (int64_t)seq_len - n_vis + k;
+    if (n_seq == 0 || s_out == 0) return CIVIC_OK;
+    if (!seq_idx || (k > 0 && !keep_idx)) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(seq_idx, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (overlaps(keep_idx, (size_t)n_seq * k * 4, seq_idx, (size_t)n_seq * s_out * 4))
+        return CIVIC_ERR_INVALID_ARG;
+    const long long total = (long long)n_seq * s_out;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    if (blocks > 4LL * sm_count()) blocks = 4LL * sm_count();
+    civic::seq_indices_kernel<<<(unsigned)blocks, threads, 0, (cudaStream_t)stream>>>(
+        keep_idx, seq_idx, n_seq, k, vis_start, n_vis, (int)s_out);
+    CIVIC_CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+civic_status_t civic_compact_kv(const void* const* k_src, const void* const* v_src,
+                                void* const* k_dst, void* const* v_dst, int32_t n_layers,
+                                int32_t n_seq, int32_t seq_len, int32_t s_out, size_t row_bytes,
+                                const int32_t* seq_idx, void* stream)
+{
+    if (n_layers < 0 || n_seq < 0 || seq_len < 0 || s_out < 0) return CIVIC_ERR_INVALID_ARG;
+    if (s_out > seq_len) return CIVIC_ERR_K_RANGE;
+    if (row_bytes == 0 || row_bytes > UINT32_MAX) return CIVIC_ERR_INVALID_ARG;
+    if (row_bytes % 4) return CIVIC_ERR_ALIGNMENT;
+    if (n_layers == 0 || n_seq == 0 || s_out == 0) return CIVIC_OK;
+    if (!k_src || !v_src || !k_dst || !v_dst || !seq_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(seq_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    const size_t src_bytes = (size_t)n_seq * seq_len * row_bytes;
+    const size_t dst_bytes = (size_t)n_seq * s_out * row_bytes;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!k_src[l] || !v_src[l] || !k_dst[l] || !v_dst[l]) return CIVIC_ERR_INVALID_ARG;
+        if (!aligned(k_src[l], 4) || !aligned(v_src[l], 4) || !aligned(k_dst[l], 4) ||
+            !aligned(v_dst[l], 4))
+            return CIVIC_ERR_ALIGNMENT;
+    }
+    // no destination may overlap a source, another destination or the index array
+    for (int a = 0; a < 2 * n_layers; ++a) {
+        const void* da = (a & 1) ? v_dst[a >> 1] : k_dst[a >> 1];
+        if (overlaps(da, dst_bytes, seq_idx, (size_t)n_seq * s_out * 4)) return CIVIC_ERR_INVALID_ARG;
+        for (int b = 0; b < 2 * n_layers; ++b) {
+            const void* sb = (b & 1) ? v_src[b >> 1] : k_src[b >> 1];
+            const void* db = (b & 1) ? v_dst[b >> 1] : k_dst[b >> 1];
+            if (overlaps(da, dst_bytes, sb, src_bytes)) return CIVIC_ERR_INVALID_ARG;
+            if (a != b && overlaps(da, dst_bytes, db, dst_bytes)) return CIVIC_ERR_INVALID_ARG;
+        }
+    }
+
+    const int layers_per_launch = civic::kMaxGatherTensors / 2;
+    for (int l0 = 0; l0 < n_layers; l0 += layers_per_launch) {
+        const int nl = n_layers - l0 < layers_per_launch ? n_layers - l0 : layers_per_launch;
+        civic::GatherParams p;
+        memset(&p, 0, sizeof p);
+        for (int l = 0; l < nl; ++l) {
+            p.src[2 * l] = (const char*)k_src[l0 + l];
+            p.dst[2 * l] = (char*)k_dst[l0 + l];
+            p.src[2 * l + 1] = (const char*)v_src[l0 + l];
+            p.dst[2 * l + 1] = (char*)v_dst[l0 + l];
+        }
+        p.n_tensors = 2 * nl;
+        p.idx = seq_idx;
+        p.n_seq = n_seq; p.seq_len = seq_len; p.s_out = s_out;
+        p.row_bytes = (uint32_t)row_bytes;
+        civic_status_t st = launch_gather(p, (cudaStream_t)stream);
+        if (st != CIVIC_OK) return st;
+    }
+    return CIVIC_OK;
+}
+
+}  // extern "C"

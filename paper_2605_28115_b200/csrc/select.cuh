@@ -1,0 +1,201 @@
+// Token selection: top-K by fp32 score under a per-region retention floor.
+// One thread block per segment; the segment's keys live in shared memory.
+//
+// Steps (all integer work on the fp32 bit patterns):
+//   1. key transform   monotone map fp32 -> uint32, so that unsigned key order equals
+//                      IEEE-754 totalOrder on the scores;
+//   2. floor           a token is reserved iff fewer than m tokens of its region beat it
+//                      (higher key, or equal key and lower index);
+//   3. radix select    over the non-reserved tokens, 4 passes of 8 bits from the top:
+//                      the exact key T of the k'-th best and how many tokens with key == T
+//                      are still needed (k' = k - number reserved);
+//   4. mask + scan     keep = reserved | key > T | (key == T and fewer than `need_eq`
+//                      equal-keyed non-reserved tokens precede it); destinations come from
+//                      a ballot/popc scan in index order, so the output is ascending.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace civic {
+
+struct SelectParams {
+    const float* scores;  // [n_seg, n]
+    int32_t* keep_idx;    // [n_seg, k]
+    int32_t n, t, h, w;
+    int32_t region_h, region_w;
+    int32_t m;      // floor per region
+    int32_t k;      // kept per segment
+    int32_t k_fill; // k - reserved count (>= 0), shape-only
+};
+
+__host__ __device__ inline size_t select_smem_bytes(int n)
+{
+    const size_t words = (size_t)(n + 31) / 32;
+    // keys | reserved bit words | 256-bin histogram | per-warp totals (32) | 4 scalars
+    return (words * 32 + words + 256 + 32 + 4) * sizeof(uint32_t);
+}
+
+__device__ __forceinline__ uint32_t score_key(float s)
+{
+    const uint32_t b = __float_as_uint(s);
+    return b ^ ((b & 0x80000000u) ? 0xFFFFFFFFu : 0x80000000u);
+}
+
+__global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
+{
+    extern __shared__ uint32_t smem[];
+    const int n = p.n;
+    const int n_words = (n + 31) >> 5;
+    const int n_pad = n_words << 5;
+    uint32_t* keys = smem;                 // [n_pad]
+    uint32_t* resv = keys + n_pad;         // [n_words] bit i%32 of word i/32
+    uint32_t* hist = resv + n_words;       // [256]
+    uint32_t* warp_tot = hist + 256;       // [32]
+    uint32_t* scal = warp_tot + 32;        // [0] digit, [1] remaining rank
+
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
+    const float* scores = p.scores + (size_t)blockIdx.x * n;
+    int32_t* out = p.keep_idx + (size_t)blockIdx.x * p.k;
+
+    // 1. keys
+    for (int i = tid; i < n_pad; i += nt) keys[i] = i < n ? score_key(scores[i]) : 0u;
+    __syncthreads();
+
+    // 2. floor: rank of every token inside its region, by direct counting
+    if (p.m > 0) {
+        const int hw = p.h * p.w;
+        for (int i = tid; i < n_pad; i += nt) {
+            bool r = false;
+            if (i < n) {
+                const int tt = i / hw, rem = i - tt * hw;
+                const int hh = rem / p.w, ww = rem - hh * p.w;
+                const int h0 = (hh / p.region_h) * p.region_h, w0 = (ww / p.region_w) * p.region_w;
+                const int h1 = min(h0 + p.region_h, p.h), w1 = min(w0 + p.region_w, p.w);
+                const uint32_t mine = keys[i];
+                int better = 0;
+                for (int y = h0; y < h1; ++y) {
+                    const int row = (tt * p.h + y) * p.w;
+                    for (int x = w0; x < w1; ++x) {
+                        const int j = row + x;
+                        const uint32_t other = keys[j];
+                        better += (other > mine) || (other == mine && j < i);
+                    }
+                }
+                r = better < p.m;
+            }
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, r);
+            if (lane == 0) resv[i >> 5] = word;
+        }
+    } else {
+        for (int i = tid; i < n_words; i += nt) resv[i] = 0u;
+    }
+    __syncthreads();
+
+    // 3. radix select of the k_fill-th best non-reserved key
+    uint32_t prefix = 0xFFFFFFFFu, need_eq = 0;
+    if (p.k_fill > 0) {
+        uint32_t mask = 0;
+        uint32_t rank = (uint32_t)p.k_fill;  // 1-based rank among the candidates still matching
+        prefix = 0;
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int b = tid; b < 256; b += nt) hist[b] = 0;
+            __syncthreads();
+            for (int i = tid; i < n_pad; i += nt) {
+                const uint32_t key = keys[i];
+                const bool cand = i < n && !((resv[i >> 5] >> (i & 31)) & 1u) && (key & mask) == prefix;
+                const uint32_t digit = (key >> shift) & 0xFFu;
+                // one shared-memory atomic per distinct digit in the warp
+                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, cand ? digit : (0x100u | lane));
+                if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+            }
+            __syncthreads();
+            if (warp == 0) {
+                // lane l owns bins 255-8l .. 248-8l (descending); find the bin holding `rank`
+                uint32_t c[8], local = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { c[q] = hist[255 - 8 * lane - q]; local += c[q]; }
+                uint32_t incl = local;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= d) incl += v;
+                }
+                const uint32_t excl = incl - local;
+                if (excl < rank && rank <= incl) {
+                    uint32_t above = excl;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (above < rank && rank <= above + c[q]) {
+                            scal[0] = 255 - 8 * lane - q;
+                            scal[1] = rank - above;
+                        }
+                        above += c[q];
+                    }
+                }
+            }
+            __syncthreads();
+            prefix |= scal[0] << shift;
+            mask |= 0xFFu << shift;
+            rank = scal[1];
+        }
+        need_eq = rank;
+    }
+    const uint32_t T = prefix;
+
+    // 4. keep mask and ascending destinations.  Each warp owns a contiguous run of 32-token
+    // words; pass A counts, pass B places.
+    const int words_per_warp = (n_words + n_warps - 1) / n_warps;
+    const int w_begin = min(warp * words_per_warp, n_words);
+    const int w_end = min(w_begin + words_per_warp, n_words);
+    uint32_t sure_cnt = 0, eq_cnt = 0;
+    for (int wd = w_begin; wd < w_end; ++wd) {
+        const int i = (wd << 5) + lane;
+        const uint32_t key = keys[i];
+        const bool r = (resv[wd] >> lane) & 1u;
+        const bool sure = i < n && (r || (p.k_fill > 0 && key > T));
+        const bool eq = i < n && !r && p.k_fill > 0 && key == T;
+        sure_cnt += __popc(__ballot_sync(0xFFFFFFFFu, sure));
+        eq_cnt += __popc(__ballot_sync(0xFFFFFFFFu, eq));
+    }
+    if (lane == 0) warp_tot[warp] = (eq_cnt << 16) | sure_cnt;  // n <= 65535 per field
+    __syncthreads();
+    uint32_t base = (lane < warp) ? warp_tot[lane] : 0u;  // n_warps <= 32
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) base += __shfl_xor_sync(0xFFFFFFFFu, base, d);
+    uint32_t sure_before = base & 0xFFFFu, eq_before = base >> 16;
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int wd = w_begin; wd < w_end; ++wd) {
+        const int i = (wd << 5) + lane;
+        const uint32_t key = keys[i];
+        const bool r = (resv[wd] >> lane) & 1u;
+        const bool sure = i < n && (r || (p.k_fill > 0 && key > T));
+        const bool eq = i < n && !r && p.k_fill > 0 && key == T;
+        const uint32_t sb = __ballot_sync(0xFFFFFFFFu, sure), eb = __ballot_sync(0xFFFFFFFFu, eq);
+        const uint32_t my_eq_before = eq_before + __popc(eb & lt);
+        const uint32_t my_sure_before = sure_before + __popc(sb & lt);
+        if (sure || (eq && my_eq_before < need_eq))
+            out[my_sure_before + min(my_eq_before, need_eq)] = i;
+        sure_before += __popc(sb);
+        eq_before += __popc(eb);
+    }
+}
+
+// seq_idx[s, :] = text positions before the visual span, vis_start + kept visual indices,
+// text positions behind the span.
+__global__ void seq_indices_kernel(const int32_t* __restrict__ keep_idx, int32_t* __restrict__ seq_idx,
+                                   int n_seq, int k, int vis_start, int n_vis, int s_out)
+{
+    const long long total = (long long)n_seq * s_out;
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const int s = (int)(e / s_out), j = (int)(e - (long long)s * s_out);
+        int32_t v;
+        if (j < vis_start) v = j;
+        else if (j < vis_start + k) v = vis_start + keep_idx[(size_t)s * k + (j - vis_start)];
+        else v = j - k + n_vis;
+        seq_idx[e] = v;
+    }
+}
+
+}  // namespace civic

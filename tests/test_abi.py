@@ -1,0 +1,137 @@
+"""The C-ABI library: loads without a GPU, exports what include/civic.h declares, and
+rejects bad arguments on the host before anything is launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2605_28115_b200 import build, civic
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return civic.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "civic.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(civic_[a-z_]+)\s*\(", text)))
+
+
+def test_exports_match_header(lib):
+    names = declared_functions()
+    assert sorted(civic.EXPORTS) == names
+    for name in names:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings(lib):
+    for code, name in enumerate(civic.STATUS_NAMES):
+        assert lib.civic_status_string(code).decode() == name
+    assert lib.civic_status_string(99).decode() == "CIVIC_ERR_UNKNOWN"
+    assert lib.civic_last_cuda_error().decode() == ""
+
+
+def test_max_tokens_covers_workloads(lib):
+    assert lib.civic_select_max_tokens() >= 3136
+    assert lib.civic_select_max_tokens() <= 65535
+
+
+def test_reserved_count_matches_region_enumeration(lib):
+    rng = np.random.default_rng(0)
+    for _ in range(300):
+        t, h, w = (int(rng.integers(1, 5)), int(rng.integers(1, 40)), int(rng.integers(1, 40)))
+        rh, rw, m = int(rng.integers(1, 9)), int(rng.integers(1, 9)), int(rng.integers(0, 20))
+        d = civic.SelectDesc(t, h, w, rh, rw, m, 0)
+        assert civic.reserved_count(d) == oracle.default.reserved_count(t, h, w, rh, rw, m)
+    assert civic.reserved_count(civic.SelectDesc(1, 4, 4, 0, 1, 1, 1)) == -1
+
+
+def _select_status(lib, desc, n_seg=1, scores=0x1000, out=0x2000):
+    return lib.civic_select(scores, n_seg, ctypes.byref(desc), out, None)
+
+
+def test_select_validation_happens_on_host(lib):
+    D = civic.SelectDesc
+    before = lib.civic_launch_count()
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 17)) == 2  # k > n
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, -1)) == 2
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 3)) == 3  # floor needs 4
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 5, 15)) == 3
+    assert _select_status(lib, D(0, 4, 4, 2, 2, 1, 3)) == 1
+    assert _select_status(lib, D(1, 4, 4, 2, 0, 1, 3)) == 1
+    assert _select_status(lib, D(1, 4, 4, 2, 2, -1, 3)) == 1
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 8), n_seg=-1) == 1
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 8), scores=None) == 1
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 8), out=None) == 1
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 8), scores=0x1002) == 4
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 8), scores=0x1000, out=0x1010) == 1  # overlap
+    assert _select_status(lib, D(1, 300, 300, 2, 2, 0, 8)) == 5  # 90000 tokens > one block
+    assert _select_status(lib, D(2, 40000, 40000, 2, 2, 0, 8)) == 5
+    assert lib.civic_select(None, 1, None, None, None) == 1
+    # nothing to do: OK without touching the device
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 0, 0)) == 0
+    assert _select_status(lib, D(1, 4, 4, 2, 2, 1, 8), n_seg=0) == 0
+    assert lib.civic_launch_count() == before
+
+
+def test_compact_validation(lib):
+    f = lib.civic_compact
+    before = lib.civic_launch_count()
+    assert f(0x10000, 64, None, 0x100, 1, 8, 9, 0x20000, None, None) == 2  # k > n
+    assert f(0x10000, 64, None, 0x100, 1, 8, 4, None, None, None) == 1  # hidden without out
+    assert f(None, 64, 0x10000, 0x100, 1, 8, 4, None, None, None) == 1  # pos without out
+    assert f(0x10000, 6, None, 0x100, 1, 8, 4, 0x20000, None, None) == 4  # row not multiple of 4
+    assert f(0x10002, 64, None, 0x100, 1, 8, 4, 0x20000, None, None) == 4
+    assert f(0x10000, 64, None, 0x100, 1, 8, 4, 0x10100, None, None) == 1  # overlap
+    assert f(0x10000, 64, None, None, 1, 8, 4, 0x20000, None, None) == 1  # no indices
+    assert f(0x10000, 64, None, 0x100, -1, 8, 4, 0x20000, None, None) == 1
+    assert f(0x10000, 64, None, 0x100, 0, 8, 4, 0x20000, None, None) == 0
+    assert f(0x10000, 64, None, 0x100, 1, 8, 0, 0x20000, None, None) == 0
+    assert lib.civic_launch_count() == before
+
+
+def test_seq_indices_validation(lib):
+    f = lib.civic_seq_indices
+    assert f(0x100, 1, 5, 20, 3, 12, None, None) == 1
+    assert f(0x100, 1, 13, 20, 3, 12, 0x1000, None) == 2  # k > n_vis
+    assert f(0x100, 1, 5, 20, 10, 12, 0x1000, None) == 1  # span runs past the end
+    assert f(0x100, 1, 5, 20, -1, 12, 0x1000, None) == 1
+    assert f(0x100, 0, 5, 20, 3, 12, 0x1000, None) == 0
+
+
+def test_compact_kv_validation(lib):
+    f = lib.civic_compact_kv
+    P = ctypes.c_void_p * 2
+    ks, vs = P(0x100000, 0x200000), P(0x300000, 0x400000)
+    kd, vd = P(0x500000, 0x600000), P(0x700000, 0x800000)
+    assert f(ks, vs, kd, vd, 2, 2, 16, 17, 64, 0x10, None) == 2  # s_out > seq_len
+    assert f(ks, vs, kd, vd, 2, 2, 16, 8, 0, 0x10, None) == 1
+    assert f(ks, vs, kd, vd, 2, 2, 16, 8, 6, 0x10, None) == 4
+    assert f(ks, vs, kd, vd, 2, 2, 16, 8, 64, None, None) == 1
+    assert f(None, vs, kd, vd, 2, 2, 16, 8, 64, 0x10, None) == 1
+    assert f(ks, vs, ks, vd, 2, 2, 16, 8, 64, 0x10, None) == 1  # destination is a source
+    assert f(ks, vs, kd, kd, 2, 2, 16, 8, 64, 0x10, None) == 1  # two destinations coincide
+    assert f(ks, vs, P(0x500000, None), vd, 2, 2, 16, 8, 64, 0x10, None) == 1
+    assert f(ks, vs, kd, vd, 0, 2, 16, 8, 64, 0x10, None) == 0
+    assert f(ks, vs, kd, vd, -1, 2, 16, 8, 64, 0x10, None) == 1
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+
+    d = civic.SelectDesc(1, 4, 4, 2, 2, 1, 8)
+    with pytest.raises(ValueError, match="CUDA"):
+        civic.civic_select(torch.zeros(1, 16), d, keep_idx=torch.zeros(1, 8, dtype=torch.int32))
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    with pytest.raises(RuntimeError, match="no fallback"):
+        civic.load(str(tmp_path / "libcivic.so"))
