@@ -1,0 +1,452 @@
+#!/usr/bin/env python
+"""Benchmark of the select + compact + KV-compaction path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one pass of the whole path over one batch of synthetic input:
+civic_select -> civic_compact (hidden + position ids) -> civic_seq_indices -> civic_compact_kv
+(all layers, K and V).  The default workload is the Qwen3-VL-8B-shaped K/V compaction
+configuration (16 sequences x 1088 tokens, 36 layers), with the batch's hidden states and
+position ids included so that every step of the path runs.
+
+Prints ONE JSON line (rank 0).  `value` is whole-job compacted GB/s with inputs resident in
+HBM: the bytes the method has to move (every kept row read once and written once, plus
+scores in and indices out) divided by the device time of a step.  With N > 1 every rank
+compacts its own batch (no data-path collective; weak scaling) and the line reports the sum.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compacted_GBps_select_compact_kv"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used when MEASURED_PEAKS.json is absent
+
+# DRAM bytes (read + write) of ONE civic_compact_kv launch, from the ncu capture summarised in
+# profiles/; keyed by workload name.  None = not captured for that workload.
+NCU_DRAM_TRAFFIC_PER_LAUNCH = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="c3_kv_qwen3vl8b")
+    ap.add_argument("--impl", default="civic", choices=["civic", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="shrink the workload to this many K/V layers (profiling a small case); "
+                         "the JSON line then names the reduced workload")
+    return ap.parse_args()
+
+
+def step_bytes(wl):
+    """Algorithmic bytes of one step, by part."""
+    from paper_2605_28115_b200 import workloads as W
+
+    kv = W.kv_algorithmic_bytes(wl)
+    hidden = 2 * wl.n_seg * wl.k * wl.hidden_row_bytes if wl.hidden_dim else 0
+    pos = 2 * wl.n_seg * wl.k * 12
+    select = wl.n_seg * wl.n * 4 + wl.n_seg * wl.k * 4
+    seq = (wl.n_seg * wl.k * 4 + wl.n_seg * wl.s_out * 4) if wl.n_layers else 0
+    return {"kv": kv, "hidden": hidden, "pos": pos, "select": select, "seq_idx": seq,
+            "total": kv + hidden + pos + select + seq}
+
+
+def pick_workload(args):
+    from paper_2605_28115_b200 import workloads as W
+
+    wl = W.BY_NAME[args.workload]
+    if args.layers and wl.n_layers:
+        wl = wl.replace(name=f"{wl.name}_reduced_to_{args.layers}_layers", n_layers=args.layers)
+    return wl
+
+
+def config_of(wl, extra=None):
+    cfg = {"workload": wl.name, "n_seg": wl.n_seg, "grid_thw": [wl.t, wl.h, wl.w],
+           "region_hw": [wl.region_h, wl.region_w], "floor_per_region": wl.floor_m, "k": wl.k,
+           "scores": wl.score_kind, "hidden_dim": wl.hidden_dim, "layers": wl.n_layers,
+           "kv_row_bytes": wl.kv_row_bytes, "seq_len": wl.seq_len, "s_out": wl.s_out,
+           "text_tokens": [wl.text_before, wl.text_after],
+           "l2": "inputs larger than L2: each step streams the whole K/V set through it, no flush"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while the
+    timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+               0x100: "display_clock_setting", 0x10: "sync_boost"}
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.02):
+        self.period = period_s
+        self.samples = []
+        self.reason_bits = 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self.error = None
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # pragma: no cover - depends on the box
+            self.error = repr(e)
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+            except Exception as e:  # pragma: no cover
+                self.error = repr(e)
+                return
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        out = {"sm_mhz": int(statistics.median(self.samples)) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
+               "reasons": sorted(name for bit, name in self.REASONS.items() if self.reason_bits & bit)}
+        if self.error:
+            out["error"] = self.error
+        return out
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+
+class DeviceState:
+    """Inputs and outputs of one rank, resident on its GPU."""
+
+    def __init__(self, wl, dev, rank):
+        import torch
+
+        from paper_2605_28115_b200 import civic
+        from paper_2605_28115_b200 import workloads as W
+
+        self.wl, self.dev = wl, dev
+        wl_r = wl.replace(config_id=wl.config_id + 100 * rank) if rank else wl  # per-rank seeds
+        self.scores_host = W.scores(wl_r)
+        self.pos_host = W.pos_ids(wl)
+        self.scores = torch.from_numpy(self.scores_host).to(dev)
+        self.pos = torch.from_numpy(self.pos_host).to(dev)
+        self.hidden = W.hidden(wl_r, dev) if wl.hidden_dim else None
+        self.desc = civic.SelectDesc(wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+        self.keep = torch.empty((wl.n_seg, wl.k), dtype=torch.int32, device=dev)
+        self.hidden_out = (torch.empty((wl.n_seg, wl.k, wl.hidden_dim), dtype=torch.bfloat16, device=dev)
+                           if wl.hidden_dim else None)
+        self.pos_out = torch.empty((wl.n_seg, wl.k, 3), dtype=torch.int32, device=dev)
+        self.seq_idx = torch.empty((wl.n_seg, wl.s_out), dtype=torch.int32, device=dev)
+        self.k_src = [W.kv_layer(wl_r, l, 0, dev) for l in range(wl.n_layers)]
+        self.v_src = [W.kv_layer(wl_r, l, 1, dev) for l in range(wl.n_layers)]
+        shape = (wl.n_seg, wl.s_out, wl.kv_heads, wl.head_dim)
+        self.k_dst = [torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(wl.n_layers)]
+        self.v_dst = [torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(wl.n_layers)]
+        self.tables = (civic.kv_tables(self.k_src, self.v_src, self.k_dst, self.v_dst)
+                       if wl.n_layers else None)
+
+    def step(self, kv_events=None):
+        """One pass of the whole path on the current stream (asynchronous)."""
+        from paper_2605_28115_b200 import civic
+
+        wl = self.wl
+        civic.civic_select(self.scores, self.desc, keep_idx=self.keep)
+        civic.civic_compact(self.hidden, self.pos, self.keep, hidden_out=self.hidden_out, pos_out=self.pos_out)
+        if self.tables is not None:
+            civic.civic_seq_indices(self.keep, wl.seq_len, wl.text_before, wl.n, seq_idx=self.seq_idx)
+            if kv_events is not None:
+                kv_events[0].record()
+            civic.civic_compact_kv(self.tables, self.seq_idx)
+            if kv_events is not None:
+                kv_events[1].record()
+
+
+class HostState:
+    """Pinned host copies of one rank's inputs and result buffers for the end-to-end number."""
+
+    def __init__(self, st: DeviceState):
+        import torch
+
+        pin = lambda x: torch.empty(x.shape, dtype=x.dtype, device="cpu", pin_memory=True).copy_(x)
+        empty = lambda x: torch.empty(x.shape, dtype=x.dtype, device="cpu", pin_memory=True)
+        self.st = st
+        self.inputs = [(pin(st.scores), st.scores), (pin(st.pos), st.pos)]
+        if st.hidden is not None:
+            self.inputs.append((pin(st.hidden), st.hidden))
+        for x in st.k_src + st.v_src:
+            self.inputs.append((pin(x), x))
+        outs = [st.keep, st.pos_out] + ([st.hidden_out] if st.hidden_out is not None else [])
+        outs += st.k_dst + st.v_dst
+        self.outputs = [(x, empty(x)) for x in outs]
+        self.h2d_bytes = sum(h.numel() * h.element_size() for h, _ in self.inputs)
+        self.d2h_bytes = sum(h.numel() * h.element_size() for _, h in self.outputs)
+
+    def step(self):
+        for h, d in self.inputs:
+            d.copy_(h, non_blocking=True)
+        self.st.step()
+        for d, h in self.outputs:
+            h.copy_(d, non_blocking=True)
+
+
+def cpu_baseline(st: DeviceState, budget_s: float = 20.0):
+    """The oracle as it stands, timed on this machine's host cores on the same inputs (copied
+    from the device): a few whole passes, bounded by `budget_s`."""
+    import numpy as np
+    import torch
+
+    import oracle
+
+    wl = st.wl
+    o = oracle.default
+    threads = o.set_threads(0)
+    bits = lambda x: x.contiguous().view(torch.int16).cpu().numpy()
+    n_layers = wl.n_layers
+    row = wl.kv_heads * wl.head_dim
+    ks = [bits(x).reshape(wl.n_seg, -1, row) for x in st.k_src[:n_layers]]
+    vs = [bits(x).reshape(wl.n_seg, -1, row) for x in st.v_src[:n_layers]]
+    hidden = bits(st.hidden) if st.hidden is not None else None
+    sample = wl.replace(n_layers=n_layers)
+    nbytes = step_bytes(sample)["total"]
+    times = []
+    t_begin = time.perf_counter()
+    while len(times) < 3 or (time.perf_counter() - t_begin < budget_s / 2 and len(times) < 15):
+        t0 = time.perf_counter()
+        keep = o.select(st.scores_host, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+        o.compact(hidden, st.pos_host, keep)
+        if n_layers:
+            idx = o.seq_indices(keep, wl.seq_len, wl.text_before, wl.n)
+            o.compact_kv(ks, vs, idx)
+        times.append(time.perf_counter() - t0)
+    med = statistics.median(times)
+    return {"value": nbytes / med / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"whole path on {wl.n_seg} segments with all {n_layers} K/V layers, "
+                      f"median of {len(times)} runs, {med * 1e3:.1f} ms per run",
+            "ms_per_sample": med * 1e3}
+
+
+def run_civic(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_28115_b200 import build as civic_build
+    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        civic_build.build()
+    if world > 1:
+        dist.barrier()
+    civic.load()
+
+    wl = pick_workload(args)
+    st = DeviceState(wl, dev, rank)
+    nbytes = step_bytes(wl)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        st.step()
+    barrier()
+
+    kv_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range(args.steps)] if wl.n_layers else None
+    sampler = ClockSampler(local_rank)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = civic.launch_count()
+    sampler.start()
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        st.step(kv_ev[i] if kv_ev else None)
+    end.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = civic.launch_count() - launches0
+    ms = start.elapsed_time(end)
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    ms_per_step = ms_max / args.steps
+    value = world * nbytes["total"] / (ms_per_step * 1e-3) / 1e9
+
+    roofline = None
+    if kv_ev:
+        kv_ms = [a.elapsed_time(b) for a, b in kv_ev]
+        kv_avg = sum(kv_ms) / len(kv_ms)
+        peak, which = measured_peak()
+        achieved = nbytes["kv"] / (kv_avg * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "civic_compact_kv", "achieved": achieved, "peak": peak,
+                    "unit": "GB/s", "frac": achieved / peak, "peak_source": which,
+                    "traffic": NCU_DRAM_TRAFFIC_PER_LAUNCH.get(wl.name),
+                    "algorithmic_bytes_per_launch": nbytes["kv"], "us_per_launch": kv_avg * 1e3,
+                    "us_per_launch_min": min(kv_ms) * 1e3, "frac_of_8TBps_nominal": achieved / 8000.0}
+
+    # end to end: pinned host inputs -> device -> path -> pinned host results, every step
+    e2e = None
+    if not args.no_e2e:
+        hs = HostState(st)
+        hs.step()
+        barrier()
+        n_e2e = max(1, args.e2e_steps)
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record()
+        for _ in range(n_e2e):
+            hs.step()
+        e2.record()
+        barrier()
+        t2 = torch.tensor([s2.elapsed_time(e2)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t2.item()) / n_e2e
+        e2e = {"value": world * nbytes["total"] / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
+               "ms_per_step": ms_e2e, "steps": n_e2e,
+               "how": "pinned host buffers, cudaMemcpyAsync of every input and result around the C-ABI calls"}
+        del hs
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(st)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+                "config": config_of(wl, {"parallelism": f"dp{world}" if world > 1 else "single"}),
+                "bytes_per_step": nbytes, "gpu_launches": launches, "clocks": clocks,
+                "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    """The CPU oracle on this machine's host cores, same metric and workload; at most 50 steps."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    from paper_2605_28115_b200 import workloads as W
+
+    wl = pick_workload(args)
+    o = oracle.default
+    threads = o.set_threads(0)
+    n_layers = wl.n_layers
+    sample = wl
+    rng = np.random.default_rng(wl.seed)
+    row = wl.kv_heads * wl.head_dim
+
+    def payload(shape):  # opaque 16-bit patterns; values never influence the path
+        return rng.integers(0, 1 << 16, size=shape, dtype=np.uint16)
+
+    scores = W.scores(wl)
+    pos = W.pos_ids(wl)
+    hidden = payload((wl.n_seg, wl.n, wl.hidden_dim)) if wl.hidden_dim else None
+    ks = [payload((wl.n_seg, wl.seq_len, row)) for _ in range(n_layers)]
+    vs = [payload((wl.n_seg, wl.seq_len, row)) for _ in range(n_layers)]
+    nbytes = step_bytes(sample)["total"]
+
+    def step():
+        keep = o.select(scores, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+        o.compact(hidden, pos, keep)
+        if n_layers:
+            o.compact_kv(ks, vs, o.seq_indices(keep, wl.seq_len, wl.text_before, wl.n))
+
+    steps = min(args.steps, 50)
+    warm = min(max(args.warmup, 3), 5)
+    for _ in range(warm):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    value = nbytes / (ms * 1e-3) / 1e9
+    sample_txt = (f"each step = whole path on {wl.n_seg} segments with all {n_layers} "
+                  f"K/V layers on the host")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": config_of(wl, {"sample": sample_txt}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": sample_txt},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_civic(a)
