@@ -278,7 +278,7 @@ def run_civic(args):
     import torch.distributed as dist
 
     from paper_2605_28115_b200 import build as civic_build
-    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import civic, sharding
     from paper_2605_28115_b200 import workloads as W
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -326,13 +326,8 @@ def run_civic(args):
     barrier()
     clocks = sampler.stop()
     launches = civic.launch_count() - launches0
-    ms = start.elapsed_time(end)
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    ms_per_step = ms_max / args.steps
-    value = world * nbytes["total"] / (ms_per_step * 1e-3) / 1e9
+    ms_per_step = sharding.max_over_ranks(start.elapsed_time(end), dev) / args.steps
+    value = sharding.job_throughput_gbs(nbytes["total"], world, ms_per_step)
 
     roofline = None
     if kv_ev:
@@ -359,11 +354,8 @@ def run_civic(args):
             hs.step()
         e2.record()
         barrier()
-        t2 = torch.tensor([s2.elapsed_time(e2)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t2.item()) / n_e2e
-        e2e = {"value": world * nbytes["total"] / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+        ms_e2e = sharding.max_over_ranks(s2.elapsed_time(e2), dev) / n_e2e
+        e2e = {"value": sharding.job_throughput_gbs(nbytes["total"], world, ms_e2e), "unit": UNIT,
                "h2d_bytes_per_step": hs.h2d_bytes, "d2h_bytes_per_step": hs.d2h_bytes,
                "ms_per_step": ms_e2e, "steps": n_e2e,
                "how": "pinned host buffers, cudaMemcpyAsync of every input and result around the C-ABI calls"}

@@ -74,18 +74,19 @@ civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
     const long long pos_elems = has_pos ? (long long)p.n_seq * p.s_out * 3 : 0;
     if (total_rows == 0 && pos_elems == 0) return CIVIC_OK;
 
-    const int threads = 256, warps = threads / 32;
-    const int resident = sm_count() * (2048 / threads);
-    long long main_blocks = (total_rows + warps - 1) / warps;
-    if (main_blocks > resident) main_blocks = resident;
-    long long pos_blocks = (pos_elems + threads - 1) / threads;
-    if (pos_blocks > sm_count()) pos_blocks = sm_count();
-    p.main_blocks = (uint32_t)main_blocks;
-    const unsigned grid = (unsigned)(main_blocks + pos_blocks);
-
     bool vec16 = p.row_bytes % 16 == 0;
     for (int i = 0; i < p.n_tensors && vec16; ++i)
         vec16 = aligned(p.src[i], 16) && aligned(p.dst[i], 16);
+    // one warp per segment of 32 * UNROLL vectors of a row
+    const int threads = civic::kGatherThreads, warps = threads / 32;
+    const long long seg_bytes = vec16 ? 32 * 4 * 16 : 32 * 8 * 4;
+    const long long segs_per_row = ((long long)p.row_bytes + seg_bytes - 1) / seg_bytes;
+    const long long main_blocks = (total_rows * segs_per_row + warps - 1) / warps;
+    long long pos_blocks = (pos_elems + threads - 1) / threads;
+    if (pos_blocks > sm_count()) pos_blocks = sm_count();
+    if (main_blocks + pos_blocks > 0x7FFFFFFFLL) return CIVIC_ERR_UNSUPPORTED;
+    p.main_blocks = (uint32_t)main_blocks;
+    const unsigned grid = (unsigned)(main_blocks + pos_blocks);
     if (vec16)
         civic::gather_rows_kernel<uint4, 4><<<grid, threads, 0, stream>>>(p);
     else

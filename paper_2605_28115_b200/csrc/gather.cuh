@@ -8,6 +8,7 @@
 namespace civic {
 
 constexpr int kMaxGatherTensors = 160;  // K and V of 80 layers per launch
+constexpr int kGatherThreads = 256;
 
 struct GatherParams {
     const char* src[kMaxGatherTensors];  // each [n_seq, seq_len, row_bytes]
@@ -54,41 +55,44 @@ __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int
     }
 }
 
-// One warp per destination row; lanes stride over the row's vectors, UNROLL loads in
-// flight per lane before the first store.
+// One warp per row segment, no grid-stride loop.  A segment is up to 32 * UNROLL vectors
+// (2 KB for 16-byte vectors) of one destination row; segments are numbered row-major, so
+// the hardware block scheduler sweeps source and destination in address order, which
+// measured faster on B200 than a persistent grid-stride loop.  Every lane has its UNROLL
+// loads in flight before its first store.
 template <typename VecT, int UNROLL>
-__global__ void __launch_bounds__(256) gather_rows_kernel(const __grid_constant__ GatherParams p)
+__global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __grid_constant__ GatherParams p)
 {
     if (blockIdx.x >= p.main_blocks) {
         gather_pos(p, blockIdx.x - p.main_blocks, gridDim.x - p.main_blocks);
         return;
     }
+    constexpr int kSegVecs = 32 * UNROLL;
     const int lane = threadIdx.x & 31;
-    const int warps_per_block = blockDim.x >> 5;
-    const long long n_warps = (long long)p.main_blocks * warps_per_block;
-    const long long rows_per_tensor = (long long)p.n_seq * p.s_out;
-    const long long total_rows = rows_per_tensor * p.n_tensors;
     const int vecs = p.row_bytes / sizeof(VecT);
+    const int segs_per_row = (vecs + kSegVecs - 1) / kSegVecs;
+    const long long rows_per_tensor = (long long)p.n_seq * p.s_out;
+    const long long total_segs = rows_per_tensor * p.n_tensors * segs_per_row;
+    const long long item = (long long)blockIdx.x * (kGatherThreads / 32) + (threadIdx.x >> 5);
+    if (item >= total_segs) return;
 
-    for (long long row = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
-         row < total_rows; row += n_warps) {
-        const int tensor = (int)(row / rows_per_tensor);
-        const long long rem = row - (long long)tensor * rows_per_tensor;  // s * s_out + j
-        const int s = (int)(rem / p.s_out);
-        const int32_t i = __ldg(p.idx + rem);
-        const VecT* src = reinterpret_cast<const VecT*>(
-            p.src[tensor] + ((size_t)s * p.seq_len + i) * p.row_bytes);
-        VecT* dst = reinterpret_cast<VecT*>(p.dst[tensor] + (size_t)rem * p.row_bytes);
-        for (int v0 = lane; v0 < vecs; v0 += 32 * UNROLL) {
-            VecT buf[UNROLL];
+    const long long row = item / segs_per_row;
+    const int seg = (int)(item - row * segs_per_row);
+    const int tensor = (int)(row / rows_per_tensor);
+    const long long rem = row - (long long)tensor * rows_per_tensor;  // s * s_out + j
+    const int s = (int)(rem / p.s_out);
+    const int32_t i = __ldg(p.idx + rem);
+    const VecT* src = reinterpret_cast<const VecT*>(p.src[tensor] + ((size_t)s * p.seq_len + i) * p.row_bytes);
+    VecT* dst = reinterpret_cast<VecT*>(p.dst[tensor] + (size_t)rem * p.row_bytes);
+
+    const int v0 = seg * kSegVecs + lane;
+    VecT buf[UNROLL];
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u)
-                if (v0 + 32 * u < vecs) buf[u] = load_stream(src + v0 + 32 * u);
+    for (int u = 0; u < UNROLL; ++u)
+        if (v0 + 32 * u < vecs) buf[u] = load_stream(src + v0 + 32 * u);
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u)
-                if (v0 + 32 * u < vecs) store_stream(dst + v0 + 32 * u, buf[u]);
-        }
-    }
+    for (int u = 0; u < UNROLL; ++u)
+        if (v0 + 32 * u < vecs) store_stream(dst + v0 + 32 * u, buf[u]);
 }
 
 }  // namespace civic
