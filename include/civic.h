@@ -7,6 +7,9 @@
  *
  * Conventions for every call
  *   - "dev" pointers are CUDA device pointers, "host" pointers ordinary host memory.
+ *     A "dev" pointer may also be pinned, device-mapped host memory (cudaHostAlloc under
+ *     unified addressing): the kernels then read only the rows they keep across PCIe and can
+ *     write results straight to host memory, with no staging copy.
  *   - All buffers are owned by the caller.  Inputs are never written.  Outputs must not
  *     overlap inputs (checked where both extents are known; overlap -> CIVIC_ERR_INVALID_ARG).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is

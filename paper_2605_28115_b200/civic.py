@@ -2,8 +2,8 @@
 
 Every step of the path runs inside the CUDA library; torch is used for device memory and
 streams.  The functions carry the names of the C entry points (include/civic.h).  There is
-no CPU fallback: if the library cannot be loaded, or a tensor is not on a CUDA device,
-the call raises.
+no CPU fallback: if the library cannot be loaded, or a tensor is neither on a CUDA device
+nor in pinned host memory (which the GPU reads and writes directly over PCIe), the call raises.
 """
 
 from __future__ import annotations
@@ -88,13 +88,22 @@ def _check(status: int, where: str) -> None:
 def _dev_ptr(x: Optional[torch.Tensor], what: str, dtype: Optional[torch.dtype] = None) -> Optional[int]:
     if x is None:
         return None
-    if not x.is_cuda:
-        raise ValueError(f"{what} must be a CUDA tensor (no CPU path exists)")
+    if not (x.is_cuda or x.is_pinned()):
+        raise ValueError(f"{what} must be a CUDA tensor or pinned (device-mapped) host memory: "
+                         "the kernels run on the GPU only, there is no CPU path")
     if not x.is_contiguous():
         raise ValueError(f"{what} must be contiguous")
     if dtype is not None and x.dtype != dtype:
         raise ValueError(f"{what} must be {dtype}, got {x.dtype}")
     return x.data_ptr()
+
+
+def _device_of(*tensors) -> torch.device:
+    """The CUDA device to launch on: that of the first CUDA tensor, else the current device."""
+    for t in tensors:
+        if t is not None and t.is_cuda:
+            return t.device
+    return torch.device("cuda", torch.cuda.current_device())
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -120,12 +129,12 @@ def civic_select(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optional[torc
         raise ValueError("scores must be [n_seg, t*h*w]")
     n_seg = scores.shape[0]
     if keep_idx is None:
-        keep_idx = torch.empty((n_seg, max(desc.k, 0)), dtype=torch.int32, device=scores.device)
+        keep_idx = torch.empty((n_seg, max(desc.k, 0)), dtype=torch.int32, device=_device_of(scores))
     elif tuple(keep_idx.shape) != (n_seg, desc.k):
         raise ValueError("keep_idx must be [n_seg, k]")
     args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
             _dev_ptr(keep_idx, "keep_idx", torch.int32))
-    with torch.cuda.device(scores.device):
+    with torch.cuda.device(_device_of(scores, keep_idx)):
         _check(load().civic_select(*args, _stream_ptr(stream)), "civic_select")
     return keep_idx
 
@@ -143,7 +152,7 @@ def civic_compact(hidden: Optional[torch.Tensor], pos_ids: Optional[torch.Tensor
         n = hidden.shape[1]
         row_bytes = hidden.shape[2] * hidden.element_size()
         if hidden_out is None:
-            hidden_out = torch.empty((n_seg, k, hidden.shape[2]), dtype=hidden.dtype, device=hidden.device)
+            hidden_out = torch.empty((n_seg, k, hidden.shape[2]), dtype=hidden.dtype, device=_device_of(keep_idx, hidden))
         elif tuple(hidden_out.shape) != (n_seg, k, hidden.shape[2]) or hidden_out.dtype != hidden.dtype:
             raise ValueError("hidden_out must be [n_seg, k, D] of hidden's dtype")
     if pos_ids is not None:
@@ -153,7 +162,7 @@ def civic_compact(hidden: Optional[torch.Tensor], pos_ids: Optional[torch.Tensor
             raise ValueError("hidden and pos_ids disagree on n")
         n = pos_ids.shape[1]
         if pos_out is None:
-            pos_out = torch.empty((n_seg, k, 3), dtype=torch.int32, device=pos_ids.device)
+            pos_out = torch.empty((n_seg, k, 3), dtype=torch.int32, device=_device_of(keep_idx, pos_ids))
         elif tuple(pos_out.shape) != (n_seg, k, 3):
             raise ValueError("pos_out must be [n_seg, k, 3]")
     if n is None:
@@ -161,7 +170,7 @@ def civic_compact(hidden: Optional[torch.Tensor], pos_ids: Optional[torch.Tensor
     args = (_dev_ptr(hidden, "hidden"), row_bytes, _dev_ptr(pos_ids, "pos_ids", torch.int32),
             _dev_ptr(keep_idx, "keep_idx", torch.int32), n_seg, n, k,
             _dev_ptr(hidden_out, "hidden_out"), _dev_ptr(pos_out, "pos_out", torch.int32))
-    with torch.cuda.device(keep_idx.device):
+    with torch.cuda.device(_device_of(keep_idx, hidden, pos_ids)):
         _check(load().civic_compact(*args, _stream_ptr(stream)), "civic_compact")
     return hidden_out, pos_out
 
@@ -173,12 +182,12 @@ def civic_seq_indices(keep_idx: torch.Tensor, seq_len: int, vis_start: int, n_vi
     n_seq, k = keep_idx.shape
     s_out = seq_len - n_vis + k
     if seq_idx is None:
-        seq_idx = torch.empty((n_seq, max(s_out, 0)), dtype=torch.int32, device=keep_idx.device)
+        seq_idx = torch.empty((n_seq, max(s_out, 0)), dtype=torch.int32, device=_device_of(keep_idx))
     elif tuple(seq_idx.shape) != (n_seq, s_out):
         raise ValueError("seq_idx must be [n_seq, seq_len - n_vis + k]")
     args = (_dev_ptr(keep_idx, "keep_idx", torch.int32), n_seq, k, seq_len, vis_start, n_vis,
             _dev_ptr(seq_idx, "seq_idx", torch.int32))
-    with torch.cuda.device(keep_idx.device):
+    with torch.cuda.device(_device_of(keep_idx, seq_idx)):
         _check(load().civic_seq_indices(*args, _stream_ptr(stream)), "civic_seq_indices")
     return seq_idx
 
@@ -234,7 +243,7 @@ def civic_compact_kv(tables: KVTables, seq_idx: torch.Tensor,
     if tuple(seq_idx.shape) != (tables.n_seq, tables.s_out):
         raise ValueError("seq_idx must be [n_seq, s_out]")
     idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
-    with torch.cuda.device(seq_idx.device):
+    with torch.cuda.device(_device_of(seq_idx, *tables.keepalive[0], *tables.keepalive[2])):
         _check(load().civic_compact_kv(tables.k_src, tables.v_src, tables.k_dst, tables.v_dst,
                                        tables.n_layers, tables.n_seq, tables.seq_len, tables.s_out,
                                        tables.row_bytes, idx_ptr, _stream_ptr(stream)),

@@ -122,7 +122,7 @@ int32_t civic_select_max_tokens(void)
 {
     // largest n whose keys, reserved bits and histogram fit into one block's shared memory;
     // the scan also packs two counts of at most n into 16 bits each
-    int32_t words = (int32_t)((kMaxDynamicSmem / sizeof(uint32_t) - (256 + 32 + 4)) / 33);
+    int32_t words = (int32_t)((kMaxDynamicSmem / sizeof(uint32_t) - (4 * 256 + 32 + 4)) / 33);
     int32_t n = words * 32;
     return n < 65535 ? n : 65535;
 }

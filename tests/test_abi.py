@@ -128,7 +128,7 @@ def test_binding_refuses_cpu_tensors():
     import torch
 
     d = civic.SelectDesc(1, 4, 4, 2, 2, 1, 8)
-    with pytest.raises(ValueError, match="CUDA"):
+    with pytest.raises(ValueError, match="CUDA tensor or pinned"):
         civic.civic_select(torch.zeros(1, 16), d, keep_idx=torch.zeros(1, 8, dtype=torch.int32))
 
 

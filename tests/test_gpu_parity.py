@@ -280,3 +280,36 @@ def test_compact_kv_full_size(wl):
     L = wl.text_before + wl.text_after
     assert compact_bytes * (L + wl.n) == dense_bytes * (L + wl.k)
     assert 2 * compact_bytes == W.kv_algorithmic_bytes(wl)
+
+
+def test_pinned_host_buffers_zero_copy():
+    """Payload sources and results in pinned host memory: the kernels read and write them
+    directly; results must still equal the oracle's."""
+    wl = W.C3.replace(n_seg=3, n_layers=2)
+    s = W.scores(wl)
+    keep_o = O.select(s, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+    idx_o = O.seq_indices(keep_o, wl.seq_len, wl.text_before, wl.n)
+    pin = lambda x: torch.empty(x.shape, dtype=x.dtype, pin_memory=True).copy_(x)
+    keep = torch.from_numpy(keep_o).to(DEV)
+    idx = torch.from_numpy(idx_o).to(DEV)
+    hidden = pin(W.hidden(wl, "cpu"))
+    pos = W.pos_ids(wl)
+    h_out = torch.zeros((wl.n_seg, wl.k, wl.hidden_dim), dtype=torch.bfloat16).pin_memory()
+    p_out = torch.zeros((wl.n_seg, wl.k, 3), dtype=torch.int32).pin_memory()
+    civic.civic_compact(hidden, pin(torch.from_numpy(pos)), keep, hidden_out=h_out, pos_out=p_out)
+    ks = [pin(W.kv_layer(wl, l, 0, "cpu")) for l in range(wl.n_layers)]
+    vs = [pin(W.kv_layer(wl, l, 1, "cpu")) for l in range(wl.n_layers)]
+    shape = (wl.n_seg, wl.s_out, wl.kv_heads, wl.head_dim)
+    kd = [torch.zeros(shape, dtype=torch.bfloat16).pin_memory() for _ in ks]
+    vd = [torch.zeros(shape, dtype=torch.bfloat16).pin_memory() for _ in vs]
+    civic.civic_compact_kv(civic.kv_tables(ks, vs, kd, vd), idx)
+    torch.cuda.synchronize()
+    want_h, want_p = O.compact(bits16(hidden), pos, keep_o)
+    assert np.array_equal(bits16(h_out), want_h) and np.array_equal(p_out.numpy(), want_p)
+    row = wl.kv_heads * wl.head_dim
+    flat = lambda x: bits16(x).reshape(wl.n_seg, -1, row)
+    want_k, want_v = O.compact_kv([flat(x) for x in ks], [flat(x) for x in vs], idx_o)
+    for l in range(wl.n_layers):
+        assert np.array_equal(flat(kd[l]), want_k[l]) and np.array_equal(flat(vd[l]), want_v[l])
+    with pytest.raises(ValueError, match="pinned"):
+        civic.civic_compact(W.hidden(wl, "cpu"), None, keep)
