@@ -35,7 +35,11 @@ FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used when MEASURE
 
 # DRAM bytes (read + write) of ONE civic_compact_kv launch, from the ncu capture summarised in
 # profiles/; keyed by workload name.  None = not captured for that workload.
-NCU_DRAM_TRAFFIC_PER_LAUNCH = {}
+NCU_DRAM_TRAFFIC_PER_LAUNCH = {
+    # profiles/gather_rows_kernel_c3_kv.md: 8-layer capture, reads x4.5, writes = algorithmic minus
+    # the 51.8 MB that were still dirty in L2 when the kernel ended
+    "c3_kv_qwen3vl8b": 1_859_400_000,
+}
 
 
 def parse_args():
