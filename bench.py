@@ -4,10 +4,10 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
 One "step" is one pass of the whole path over one batch of synthetic input:
-civic_select -> civic_compact (hidden + position ids) -> civic_seq_indices -> civic_compact_kv
-(all layers, K and V).  The default workload is the Qwen3-VL-8B-shaped K/V compaction
-configuration (16 sequences x 1088 tokens, 36 layers), with the batch's hidden states and
-position ids included so that every step of the path runs.
+civic_select_seq (selection and sequence-level indices, one launch) -> civic_compact (hidden +
+position ids) -> civic_compact_kv (all layers, K and V).  The default workload is the
+Qwen3-VL-8B-shaped K/V compaction configuration (16 sequences x 1088 tokens, 36 layers), with
+the batch's hidden states and position ids included so that every step of the path runs.
 
 Prints ONE JSON line (rank 0).  `value` is whole-job compacted GB/s with inputs resident in
 HBM: the bytes the method has to move (every kept row read once and written once, plus
@@ -31,14 +31,15 @@ if ROOT not in sys.path:
 
 METRIC = "compacted_GBps_select_compact_kv"
 UNIT = "GB/s"
+KV_EVENT_STRIDE = 10
 FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used when MEASURED_PEAKS.json is absent
 
 # DRAM bytes (read + write) of ONE civic_compact_kv launch, from the ncu capture summarised in
 # profiles/; keyed by workload name.  None = not captured for that workload.
 NCU_DRAM_TRAFFIC_PER_LAUNCH = {
     # profiles/gather_rows_kernel_c3_kv.md: 8-layer capture, reads x4.5, writes = algorithmic minus
-    # the 51.8 MB that were still dirty in L2 when the kernel ended
-    "c3_kv_qwen3vl8b": 1_859_400_000,
+    # the 50.6 MB that were still dirty in L2 when the kernel ended
+    "c3_kv_qwen3vl8b": 1_860_600_000,
 }
 
 
@@ -202,10 +203,13 @@ class DeviceState:
         from paper_2605_28115_b200 import civic
 
         wl = self.wl
-        civic.civic_select(self.scores, self.desc, keep_idx=self.keep)
+        if self.tables is not None:
+            civic.civic_select_seq(self.scores, self.desc, wl.seq_len, wl.text_before,
+                                   keep_idx=self.keep, seq_idx=self.seq_idx)
+        else:
+            civic.civic_select(self.scores, self.desc, keep_idx=self.keep)
         civic.civic_compact(self.hidden, self.pos, self.keep, hidden_out=self.hidden_out, pos_out=self.pos_out)
         if self.tables is not None:
-            civic.civic_seq_indices(self.keep, wl.seq_len, wl.text_before, wl.n, seq_idx=self.seq_idx)
             if kv_events is not None:
                 kv_events[0].record()
             civic.civic_compact_kv(self.tables, self.seq_idx)
@@ -263,11 +267,14 @@ class HostState:
         for h, d in self.small_in:
             d.copy_(h, non_blocking=True)
         if self.mode == "zero_copy":
-            civic.civic_select(st.scores, st.desc, keep_idx=st.keep)
+            if self.tables is not None:
+                civic.civic_select_seq(st.scores, st.desc, wl.seq_len, wl.text_before,
+                                       keep_idx=st.keep, seq_idx=st.seq_idx)
+            else:
+                civic.civic_select(st.scores, st.desc, keep_idx=st.keep)
             civic.civic_compact(self.hidden_h, st.pos, st.keep, hidden_out=self.hidden_out_h,
                                 pos_out=st.pos_out)
             if self.tables is not None:
-                civic.civic_seq_indices(st.keep, wl.seq_len, wl.text_before, wl.n, seq_idx=st.seq_idx)
                 civic.civic_compact_kv(self.tables, st.seq_idx)
         else:
             if self.hidden_h is not None:
@@ -369,8 +376,12 @@ def run_civic(args):
         st.step()
     barrier()
 
-    kv_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-             for _ in range(args.steps)] if wl.n_layers else None
+    # The K/V kernel is bracketed by events on every KV_EVENT_STRIDE-th timed step only: an event
+    # record between two kernels takes away their programmatic launch overlap, so bracketing
+    # every step would slow the very steps being timed.
+    stride = max(1, min(KV_EVENT_STRIDE, args.steps // 20))
+    kv_ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for i in range(0, args.steps, stride)} if wl.n_layers else None
     sampler = ClockSampler(local_rank)
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = civic.launch_count()
@@ -378,7 +389,7 @@ def run_civic(args):
     barrier()
     start.record()
     for i in range(args.steps):
-        st.step(kv_ev[i] if kv_ev else None)
+        st.step(kv_ev.get(i) if kv_ev else None)
     end.record()
     barrier()
     clocks = sampler.stop()
@@ -388,7 +399,7 @@ def run_civic(args):
 
     roofline = None
     if kv_ev:
-        kv_ms = [a.elapsed_time(b) for a, b in kv_ev]
+        kv_ms = [a.elapsed_time(b) for a, b in kv_ev.values()]
         kv_avg = sum(kv_ms) / len(kv_ms)
         peak, which = measured_peak()
         achieved = nbytes["kv"] / (kv_avg * 1e-3) / 1e9
@@ -396,7 +407,7 @@ def run_civic(args):
                     "unit": "GB/s", "frac": achieved / peak, "peak_source": which,
                     "traffic": NCU_DRAM_TRAFFIC_PER_LAUNCH.get(wl.name),
                     "algorithmic_bytes_per_launch": nbytes["kv"], "us_per_launch": kv_avg * 1e3,
-                    "us_per_launch_min": min(kv_ms) * 1e3, "frac_of_8TBps_nominal": achieved / 8000.0}
+                    "us_per_launch_min": min(kv_ms) * 1e3, "launches_timed": len(kv_ms), "frac_of_8TBps_nominal": achieved / 8000.0}
 
     # end to end: pinned host inputs -> path -> pinned host results, every step
     e2e = None

@@ -77,6 +77,22 @@ typedef struct {
 civic_status_t civic_select(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
                             int32_t* keep_idx, void* stream);
 
+/*
+ * civic_select_seq -- civic_select and civic_seq_indices in ONE launch.
+ *
+ * Paper: as civic_select, followed by the index form of Eq. 13 / Section 3.5 (see
+ * civic_seq_indices).  Every sequence is `vis_start` text tokens, the n = t*h*w visual tokens of
+ * one segment, then seq_len - vis_start - n text tokens; segment s belongs to sequence s.
+ *
+ * keep_idx  dev [n_seq, k] int32, written (as by civic_select)
+ * seq_idx   dev [n_seq, seq_len - n + k] int32, written (as by civic_seq_indices with n_vis = n)
+ * Same limits and errors as the two separate calls; vis_start + n > seq_len is
+ * CIVIC_ERR_INVALID_ARG.
+ */
+civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_select_desc_t* desc,
+                                int32_t seq_len, int32_t vis_start, int32_t* keep_idx,
+                                int32_t* seq_idx, void* stream);
+
 /* Largest n = t*h*w that civic_select accepts. */
 int32_t civic_select_max_tokens(void);
 
@@ -142,6 +158,15 @@ const char* civic_last_cuda_error(void);
 
 /* Kernels this library enqueued since it was loaded (all threads). */
 uint64_t civic_launch_count(void);
+
+/*
+ * Kernels are enqueued with CUDA's programmatic-dependent-launch attribute: a kernel may become
+ * resident while the previous kernel of the stream drains, and waits for that kernel's
+ * completion before its first memory access, so stream-order semantics are unchanged while the
+ * gap between the library's own consecutive kernels shrinks.  enable = 0 switches to plain
+ * launches (process-wide); returns the previous setting.  Default: enabled.
+ */
+int32_t civic_set_programmatic_launch(int32_t enable);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,7 @@ STATUS_NAMES = ("CIVIC_OK", "CIVIC_ERR_INVALID_ARG", "CIVIC_ERR_K_RANGE", "CIVIC
 # every symbol include/civic.h declares
 EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "civic_compact",
            "civic_seq_indices", "civic_compact_kv", "civic_status_string", "civic_last_cuda_error",
-           "civic_launch_count")
+           "civic_launch_count", "civic_select_seq", "civic_set_programmatic_launch")
 
 
 class CivicError(RuntimeError):
@@ -75,6 +75,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_last_cuda_error.restype = ctypes.c_char_p
     lib.civic_launch_count.argtypes = []
     lib.civic_launch_count.restype = ctypes.c_uint64
+    lib.civic_select_seq.argtypes = [vp, i32, ctypes.POINTER(SelectDesc), i32, i32, vp, vp, vp]
+    lib.civic_select_seq.restype = ctypes.c_int
+    lib.civic_set_programmatic_launch.argtypes = [i32]
+    lib.civic_set_programmatic_launch.restype = i32
     _lib = lib
     return lib
 
@@ -137,6 +141,36 @@ def civic_select(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optional[torc
     with torch.cuda.device(_device_of(scores, keep_idx)):
         _check(load().civic_select(*args, _stream_ptr(stream)), "civic_select")
     return keep_idx
+
+
+def civic_select_seq(scores: torch.Tensor, desc: SelectDesc, seq_len: int, vis_start: int,
+                     keep_idx: Optional[torch.Tensor] = None, seq_idx: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None):
+    """civic_select and civic_seq_indices in one launch: -> (keep_idx [n_seq, k], seq_idx [n_seq, seq_len-n+k])."""
+    n = desc.t * desc.h * desc.w
+    if scores.dim() != 2 or scores.shape[1] != n:
+        raise ValueError("scores must be [n_seq, t*h*w]")
+    n_seq = scores.shape[0]
+    s_out = seq_len - n + desc.k
+    dev = _device_of(scores)
+    if keep_idx is None:
+        keep_idx = torch.empty((n_seq, max(desc.k, 0)), dtype=torch.int32, device=dev)
+    elif tuple(keep_idx.shape) != (n_seq, desc.k):
+        raise ValueError("keep_idx must be [n_seq, k]")
+    if seq_idx is None:
+        seq_idx = torch.empty((n_seq, max(s_out, 0)), dtype=torch.int32, device=dev)
+    elif tuple(seq_idx.shape) != (n_seq, s_out):
+        raise ValueError("seq_idx must be [n_seq, seq_len - n + k]")
+    args = (_dev_ptr(scores, "scores", torch.float32), n_seq, ctypes.byref(desc), seq_len, vis_start,
+            _dev_ptr(keep_idx, "keep_idx", torch.int32), _dev_ptr(seq_idx, "seq_idx", torch.int32))
+    with torch.cuda.device(_device_of(scores, keep_idx)):
+        _check(load().civic_select_seq(*args, _stream_ptr(stream)), "civic_select_seq")
+    return keep_idx, seq_idx
+
+
+def set_programmatic_launch(enable: bool) -> bool:
+    """Switch programmatic dependent launch on or off (process-wide); returns the old setting."""
+    return bool(load().civic_set_programmatic_launch(1 if enable else 0))
 
 
 def civic_compact(hidden: Optional[torch.Tensor], pos_ids: Optional[torch.Tensor], keep_idx: torch.Tensor,

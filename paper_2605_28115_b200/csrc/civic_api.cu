@@ -14,6 +14,9 @@ namespace {
 constexpr size_t kMaxDynamicSmem = 227 * 1024;
 
 std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_programmatic{1};
+
+bool programmatic() { return g_programmatic.load(std::memory_order_relaxed) != 0; }
 thread_local char g_cuda_error[256] = "";
 
 civic_status_t cuda_fail(cudaError_t e, const char* what)
@@ -88,10 +91,54 @@ civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
     p.main_blocks = (uint32_t)main_blocks;
     const unsigned grid = (unsigned)(main_blocks + pos_blocks);
     if (vec16)
-        civic::gather_rows_kernel<uint4, 4><<<grid, threads, 0, stream>>>(p);
+        CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::gather_rows_kernel<uint4, 4>, grid, threads, 0,
+                                     stream, p));
     else
-        civic::gather_rows_kernel<uint32_t, 8><<<grid, threads, 0, stream>>>(p);
-    CIVIC_CUDA_TRY(cudaGetLastError());
+        CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::gather_rows_kernel<uint32_t, 8>, grid, threads,
+                                     0, stream, p));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                           int32_t* keep_idx, int32_t* seq_idx, int32_t seq_len, int32_t vis_start,
+                           void* stream)
+{
+    if (!desc || n_seg < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n_res = reserved_count(*desc);
+    if (n_res < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)desc->t * desc->h * desc->w;
+    if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (desc->k < 0 || desc->k > n) return CIVIC_ERR_K_RANGE;
+    if (n_res > desc->k) return CIVIC_ERR_FLOOR_EXCEEDS_K;
+    if (n_seg == 0 || desc->k == 0) return CIVIC_OK;
+    if (!scores || !keep_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(scores, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (n > civic_select_max_tokens()) return CIVIC_ERR_UNSUPPORTED;
+    if (overlaps(scores, (size_t)n_seg * n * 4, keep_idx, (size_t)n_seg * desc->k * 4))
+        return CIVIC_ERR_INVALID_ARG;
+
+    civic::SelectParams p;
+    p.scores = scores;
+    p.keep_idx = keep_idx;
+    p.n = (int32_t)n;
+    p.t = desc->t; p.h = desc->h; p.w = desc->w;
+    p.region_h = desc->region_h; p.region_w = desc->region_w;
+    p.m = desc->floor_per_region;
+    p.k = desc->k;
+    p.k_fill = (int32_t)(desc->k - n_res);
+    p.seq_idx = seq_idx;
+    p.seq_len = seq_len;
+    p.vis_start = vis_start;
+
+    const size_t smem = civic::select_smem_bytes(p.n);
+    if (smem > 48 * 1024)
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int threads = (p.n + 31) / 32 * 32;
+    threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
+    CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::select_kernel, (unsigned)n_seg, (unsigned)threads,
+                                 smem, (cudaStream_t)stream, p));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CIVIC_OK;
 }
@@ -118,6 +165,11 @@ const char* civic_last_cuda_error(void) { return g_cuda_error; }
 
 uint64_t civic_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+int32_t civic_set_programmatic_launch(int32_t enable)
+{
+    return g_programmatic.exchange(enable ? 1 : 0, std::memory_order_relaxed);
+}
+
 int32_t civic_select_max_tokens(void)
 {
     // largest n whose keys, reserved bits and histogram fit into one block's shared memory;
@@ -135,40 +187,33 @@ int64_t civic_reserved_count(const civic_select_desc_t* desc)
 civic_status_t civic_select(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
                             int32_t* keep_idx, void* stream)
 {
-    if (!desc || n_seg < 0) return CIVIC_ERR_INVALID_ARG;
-    const int64_t n_res = reserved_count(*desc);
-    if (n_res < 0) return CIVIC_ERR_INVALID_ARG;
+    return select_impl(scores, n_seg, desc, keep_idx, nullptr, 0, 0, stream);
+}
+
+civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_select_desc_t* desc,
+                                int32_t seq_len, int32_t vis_start, int32_t* keep_idx,
+                                int32_t* seq_idx, void* stream)
+{
+    if (!desc || seq_len < 0 || vis_start < 0) return CIVIC_ERR_INVALID_ARG;
     const int64_t n = (int64_t)desc->t * desc->h * desc->w;
-    if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (desc->t < 1 || desc->h < 1 || desc->w < 1 || n > INT32_MAX) return CIVIC_ERR_INVALID_ARG;
+    if ((int64_t)vis_start + n > seq_len) return CIVIC_ERR_INVALID_ARG;
     if (desc->k < 0 || desc->k > n) return CIVIC_ERR_K_RANGE;
-    if (n_res > desc->k) return CIVIC_ERR_FLOOR_EXCEEDS_K;
-    if (n_seg == 0 || desc->k == 0) return CIVIC_OK;
-    if (!scores || !keep_idx) return CIVIC_ERR_INVALID_ARG;
-    if (!aligned(scores, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
-    if (n > civic_select_max_tokens()) return CIVIC_ERR_UNSUPPORTED;
-    if (overlaps(scores, (size_t)n_seg * n * 4, keep_idx, (size_t)n_seg * desc->k * 4))
-        return CIVIC_ERR_INVALID_ARG;
-
-    civic::SelectParams p;
-    p.scores = scores;
-    p.keep_idx = keep_idx;
-    p.n = (int32_t)n;
-    p.t = desc->t; p.h = desc->h; p.w = desc->w;
-    p.region_h = desc->region_h; p.region_w = desc->region_w;
-    p.m = desc->floor_per_region;
-    p.k = desc->k;
-    p.k_fill = (int32_t)(desc->k - n_res);
-
-    const size_t smem = civic::select_smem_bytes(p.n);
-    if (smem > 48 * 1024)
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int threads = (p.n + 31) / 32 * 32;
-    threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
-    civic::select_kernel<<<(unsigned)n_seg, threads, smem, (cudaStream_t)stream>>>(p);
-    CIVIC_CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return CIVIC_OK;
+    const int64_t s_out = (int64_t)seq_len - n + desc->k;
+    if (n_seq > 0 && s_out > 0) {
+        if (!seq_idx) return CIVIC_ERR_INVALID_ARG;
+        if (!aligned(seq_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+        if (overlaps(seq_idx, (size_t)n_seq * s_out * 4, keep_idx, (size_t)n_seq * desc->k * 4) ||
+            overlaps(seq_idx, (size_t)n_seq * s_out * 4, scores, (size_t)n_seq * n * 4))
+            return CIVIC_ERR_INVALID_ARG;
+    }
+    if (desc->k == 0) {
+        // nothing to select: the sequence indices are the text positions alone
+        const civic_status_t st = select_impl(scores, n_seq, desc, keep_idx, nullptr, 0, 0, stream);
+        if (st != CIVIC_OK) return st;
+        return civic_seq_indices(keep_idx, n_seq, 0, seq_len, vis_start, (int32_t)n, seq_idx, stream);
+    }
+    return select_impl(scores, n_seq, desc, keep_idx, seq_idx, seq_len, vis_start, stream);
 }
 
 civic_status_t civic_compact(const void* hidden, size_t row_bytes, const int32_t* pos_ids,
@@ -221,9 +266,9 @@ civic_status_t civic_seq_indices(const int32_t* keep_idx, int32_t n_seq, int32_t
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
     if (blocks > 4LL * sm_count()) blocks = 4LL * sm_count();
-    civic::seq_indices_kernel<<<(unsigned)blocks, threads, 0, (cudaStream_t)stream>>>(
-        keep_idx, seq_idx, n_seq, k, vis_start, n_vis, (int)s_out);
-    CIVIC_CUDA_TRY(cudaGetLastError());
+    CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::seq_indices_kernel, (unsigned)blocks, threads, 0,
+                                 (cudaStream_t)stream, keep_idx, seq_idx, n_seq, k, vis_start, n_vis,
+                                 (int)s_out));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CIVIC_OK;
 }

@@ -5,6 +5,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "pdl.cuh"
+
 namespace civic {
 
 constexpr int kMaxGatherTensors = 160;  // K and V of 80 layers per launch
@@ -63,6 +65,7 @@ __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int
 template <typename VecT, int UNROLL>
 __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __grid_constant__ GatherParams p)
 {
+    wait_for_prior_kernels();
     if (blockIdx.x >= p.main_blocks) {
         gather_pos(p, blockIdx.x - p.main_blocks, gridDim.x - p.main_blocks);
         return;

@@ -16,6 +16,8 @@
 #include <cstdint>
 #include <cuda_runtime.h>
 
+#include "pdl.cuh"
+
 namespace civic {
 
 struct SelectParams {
@@ -26,6 +28,9 @@ struct SelectParams {
     int32_t m;      // floor per region
     int32_t k;      // kept per segment
     int32_t k_fill; // k - reserved count (>= 0), shape-only
+    // optional fused epilogue: kept positions of the full sequence, see seq_indices_kernel
+    int32_t* seq_idx;   // [n_seg, seq_len - n + k] or NULL
+    int32_t seq_len, vis_start;
 };
 
 __host__ __device__ inline size_t select_smem_bytes(int n)
@@ -62,6 +67,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
     const int lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
     const float* scores = p.scores + (size_t)blockIdx.x * n;
     int32_t* out = p.keep_idx + (size_t)blockIdx.x * p.k;
+    release_next_kernel();
+    wait_for_prior_kernels();
 
     // 1. keys; clear the histograms and the reserved bits
     for (int i = tid; i < n_pad; i += nt) keys[i] = i < n ? score_key(__ldg(scores + i)) : 0u;
@@ -192,6 +199,7 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) base += __shfl_xor_sync(0xFFFFFFFFu, base, d);
     uint32_t sure_before = base & 0xFFFFu, eq_before = base >> 16;
+    int32_t* seq = p.seq_idx ? p.seq_idx + (size_t)blockIdx.x * (p.seq_len - n + p.k) : nullptr;
     const uint32_t lt = (1u << lane) - 1u;
     for (int wd = w_begin; wd < w_end; ++wd) {
         const int i = (wd << 5) + lane;
@@ -202,10 +210,20 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
         const uint32_t sb = __ballot_sync(0xFFFFFFFFu, sure), eb = __ballot_sync(0xFFFFFFFFu, eq);
         const uint32_t my_eq_before = eq_before + __popc(eb & lt);
         const uint32_t my_sure_before = sure_before + __popc(sb & lt);
-        if (sure || (eq && my_eq_before < need_eq))
-            out[my_sure_before + min(my_eq_before, need_eq)] = i;
+        if (sure || (eq && my_eq_before < need_eq)) {
+            const uint32_t j = my_sure_before + min(my_eq_before, need_eq);
+            out[j] = i;
+            if (seq) seq[p.vis_start + j] = p.vis_start + i;
+        }
         sure_before += __popc(sb);
         eq_before += __popc(eb);
+    }
+    // fused sequence indices: text in front of the visual span keeps its positions, text
+    // behind it moves up by the n - k dropped visual tokens
+    if (seq) {
+        for (int j = tid; j < p.vis_start; j += nt) seq[j] = j;
+        const int s_out = p.seq_len - n + p.k;
+        for (int j = p.vis_start + p.k + tid; j < s_out; j += nt) seq[j] = j - p.k + n;
     }
 }
 
@@ -214,6 +232,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
 __global__ void seq_indices_kernel(const int32_t* __restrict__ keep_idx, int32_t* __restrict__ seq_idx,
                                    int n_seq, int k, int vis_start, int n_vis, int s_out)
 {
+    release_next_kernel();
+    wait_for_prior_kernels();
     const long long total = (long long)n_seq * s_out;
     for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
          e += (long long)gridDim.x * blockDim.x) {

@@ -107,6 +107,24 @@ def test_seq_indices_validation(lib):
     assert f(0x100, 0, 5, 20, 3, 12, 0x1000, None) == 0
 
 
+def test_select_seq_validation(lib):
+    D = civic.SelectDesc
+    f = lambda d, seq_len, vis_start, n_seq=1, scores=0x1000, keep=0x2000, seq=0x3000: \
+        lib.civic_select_seq(scores, n_seq, ctypes.byref(d), seq_len, vis_start, keep, seq, None)
+    before = lib.civic_launch_count()
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 15, 0) == 1  # visual span longer than the sequence
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 20, 5) == 1  # span runs past the end
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 20, -1) == 1
+    assert f(D(1, 4, 4, 2, 2, 1, 17), 20, 2) == 2
+    assert f(D(1, 4, 4, 2, 2, 1, 3), 20, 2) == 3
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 20, 2, seq=None) == 1
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 20, 2, seq=0x3002) == 4
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 20, 2, seq=0x2010) == 1  # seq_idx overlaps keep_idx
+    assert f(D(1, 4, 4, 2, 2, 1, 8), 20, 2, n_seq=0) == 0
+    assert lib.civic_launch_count() == before
+    assert lib.civic_set_programmatic_launch(1) == 1  # on by default, setter returns the old value
+
+
 def test_compact_kv_validation(lib):
     f = lib.civic_compact_kv
     P = ctypes.c_void_p * 2

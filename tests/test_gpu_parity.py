@@ -229,6 +229,44 @@ def test_seq_indices():
         chk()
 
 
+def test_select_seq_fused_matches_the_two_calls():
+    """One launch writes keep_idx and seq_idx; both equal the oracle's select and sequence indices."""
+    rng = np.random.default_rng(808)
+    cases = [(W.C3, 16, 48), (W.C3.replace(n_seg=3), 0, 0), (W.C5_THIRD, 5, 0), (W.C4, 0, 7),
+             (W.C1, 3, 2)]
+    for wl, before, after in cases:
+        s = W.scores(wl)
+        seq_len = before + wl.n + after
+        for k in (wl.k, O.reserved_count(wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m), wl.n):
+            want_keep = O.select(s, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, k)
+            want_seq = O.seq_indices(want_keep, seq_len, before, wl.n)
+            keep, chk_k = padded((wl.n_seg, k), torch.int32, CANARY)
+            seq, chk_s = padded((wl.n_seg, seq_len - wl.n + k), torch.int32, CANARY)
+            desc = civic.SelectDesc(wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, k)
+            civic.civic_select_seq(torch.from_numpy(s).to(DEV), desc, seq_len, before, keep_idx=keep, seq_idx=seq)
+            assert np.array_equal(keep.cpu().numpy(), want_keep)
+            assert np.array_equal(seq.cpu().numpy(), want_seq)
+            chk_k()
+            chk_s()
+    # k = 0: only text survives
+    s = rng.random((2, 6 * 6)).astype(np.float32)
+    keep, seq = civic.civic_select_seq(torch.from_numpy(s).to(DEV), civic.SelectDesc(1, 6, 6, 2, 2, 0, 0), 41, 2)
+    assert keep.shape == (2, 0)
+    assert np.array_equal(seq.cpu().numpy(), O.seq_indices(np.zeros((2, 0), np.int32), 41, 2, 36))
+
+
+def test_plain_launches_give_the_same_results():
+    """Programmatic dependent launch switched off: same bytes."""
+    wl = W.C3.replace(n_seg=3, n_layers=2)
+    old = civic.set_programmatic_launch(False)
+    try:
+        assert old is True
+        run_kv(wl)
+    finally:
+        civic.set_programmatic_launch(True)
+    run_kv(wl)
+
+
 def run_kv(wl, layers_on_host=True):
     """select -> seq_indices -> compact_kv on the GPU; oracle on the host copy of the same inputs."""
     s = W.scores(wl)
