@@ -59,6 +59,19 @@ def _bind(path: str) -> ctypes.CDLL:
     lib.oracle_seq_indices.restype = i32
     lib.oracle_compact_kv.argtypes = [vpp, vpp, vpp, vpp, i32, i32, i32, i32, sz, i32p]
     lib.oracle_compact_kv.restype = i32
+    lib.oracle_merge_embeddings.argtypes = [vp, vp, sz, i32p, i32, i32, i32, i32, i32, vp]
+    lib.oracle_merge_embeddings.restype = i32
+    lib.oracle_compact_pos_planes.argtypes = [i32p, i32, i32, i32, i32p, i32, i32p]
+    lib.oracle_compact_pos_planes.restype = i32
+    lib.oracle_compact_kv_heads.argtypes = [vpp, vpp, vpp, vpp, i32, i32, i32, i32, i32, sz, i32p]
+    lib.oracle_compact_kv_heads.restype = i32
+    lib.oracle_compact_kv_paged.argtypes = [vpp, vpp, vpp, vpp, i32, i32, i32, i32, sz, i32p, i32p,
+                                            i32, i32, i32]
+    lib.oracle_compact_kv_paged.restype = i32
+    lib.oracle_floor_from_ratio.argtypes = [i32] * 4
+    lib.oracle_floor_from_ratio.restype = ctypes.c_int64
+    lib.oracle_select_ragged.argtypes = [f32p, i32, i32p, i32p, i32p]
+    lib.oracle_select_ragged.restype = i32
     lib.oracle_set_threads.argtypes = [i32]
     lib.oracle_set_threads.restype = i32
     return lib
@@ -188,6 +201,88 @@ class Oracle:
                                         row * np.dtype(dt).itemsize, _i32p(seq_idx)),
                "oracle_compact_kv")
         return k_dst, v_dst
+
+    def merge_embeddings(self, text: np.ndarray, visual: np.ndarray, keep_idx: np.ndarray,
+                         vis_start: int) -> np.ndarray:
+        """text [n_seq, seq_len, row], visual [n_seq, n_vis, row] -> [n_seq, seq_len - n_vis + k, row]."""
+        text, visual = np.ascontiguousarray(text), np.ascontiguousarray(visual)
+        keep_idx = np.ascontiguousarray(keep_idx, dtype=np.int32)
+        n_seq, seq_len, row = text.shape
+        n_vis, k = visual.shape[1], keep_idx.shape[1]
+        assert visual.shape == (n_seq, n_vis, row) and visual.dtype == text.dtype
+        out = np.zeros((n_seq, seq_len - n_vis + k, row), dtype=text.dtype)
+        _check(self.h.oracle_merge_embeddings(text.ctypes.data, visual.ctypes.data, row * text.itemsize,
+                                              _i32p(keep_idx), n_seq, seq_len, vis_start, n_vis, k,
+                                              out.ctypes.data), "oracle_merge_embeddings")
+        return out
+
+    def compact_pos_planes(self, pos: np.ndarray, seq_idx: np.ndarray) -> np.ndarray:
+        """pos int32 [n_planes, n_seq, seq_len], seq_idx [n_seq, s_out] -> [n_planes, n_seq, s_out]."""
+        pos = np.ascontiguousarray(pos, dtype=np.int32)
+        seq_idx = np.ascontiguousarray(seq_idx, dtype=np.int32)
+        n_planes, n_seq, seq_len = pos.shape
+        s_out = seq_idx.shape[1]
+        out = np.full((n_planes, n_seq, s_out), -1, dtype=np.int32)
+        _check(self.h.oracle_compact_pos_planes(_i32p(pos), n_planes, n_seq, seq_len, _i32p(seq_idx),
+                                                s_out, _i32p(out)), "oracle_compact_pos_planes")
+        return out
+
+    def compact_kv_heads(self, k_src: Sequence[np.ndarray], v_src: Sequence[np.ndarray],
+                         seq_idx: np.ndarray):
+        """Per layer K and V as [n_seq, n_heads, seq_len, d] -> lists of [n_seq, n_heads, s_out, d]."""
+        seq_idx = np.ascontiguousarray(seq_idx, dtype=np.int32)
+        n_seq, s_out = seq_idx.shape
+        n_layers = len(k_src)
+        k_src = [np.ascontiguousarray(a) for a in k_src]
+        v_src = [np.ascontiguousarray(a) for a in v_src]
+        a0 = k_src[0]
+        _, n_heads, seq_len, d = a0.shape
+        assert all(a.shape == a0.shape and a.dtype == a0.dtype for a in k_src + v_src)
+        k_dst = [np.zeros((n_seq, n_heads, s_out, d), dtype=a0.dtype) for _ in range(n_layers)]
+        v_dst = [np.zeros((n_seq, n_heads, s_out, d), dtype=a0.dtype) for _ in range(n_layers)]
+        table = lambda arrs: (ctypes.c_void_p * n_layers)(*[a.ctypes.data for a in arrs])
+        _check(self.h.oracle_compact_kv_heads(table(k_src), table(v_src), table(k_dst), table(v_dst),
+                                              n_layers, n_seq, n_heads, seq_len, s_out,
+                                              d * a0.itemsize, _i32p(seq_idx)), "oracle_compact_kv_heads")
+        return k_dst, v_dst
+
+    def compact_kv_paged(self, k_src: Sequence[np.ndarray], v_src: Sequence[np.ndarray],
+                         seq_idx: np.ndarray, block_table: np.ndarray, page_size: int,
+                         k_cache: Sequence[np.ndarray], v_cache: Sequence[np.ndarray]) -> None:
+        """Writes the kept rows of src [n_seq, seq_len, row] into caches [n_pages, page_size, row]
+        (modified in place) through block_table int32 [n_seq, max_pages_per_seq]."""
+        seq_idx = np.ascontiguousarray(seq_idx, dtype=np.int32)
+        block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+        n_seq, s_out = seq_idx.shape
+        n_layers = len(k_src)
+        k_src = [np.ascontiguousarray(a) for a in k_src]
+        v_src = [np.ascontiguousarray(a) for a in v_src]
+        a0, c0 = k_src[0], k_cache[0]
+        seq_len, row = a0.shape[1], a0.shape[2]
+        assert all(c.flags.c_contiguous and c.shape == c0.shape and c.dtype == a0.dtype
+                   for c in list(k_cache) + list(v_cache))
+        assert c0.shape[1] == page_size and c0.shape[2] == row and block_table.shape[0] == n_seq
+        table = lambda arrs: (ctypes.c_void_p * n_layers)(*[a.ctypes.data for a in arrs])
+        _check(self.h.oracle_compact_kv_paged(table(k_src), table(v_src), table(k_cache), table(v_cache),
+                                              n_layers, n_seq, seq_len, s_out, row * a0.itemsize,
+                                              _i32p(seq_idx), _i32p(block_table), block_table.shape[1],
+                                              page_size, c0.shape[0]), "oracle_compact_kv_paged")
+
+    def floor_from_ratio(self, region_h: int, region_w: int, num: int, den: int) -> int:
+        return int(self.h.oracle_floor_from_ratio(region_h, region_w, num, den))
+
+    def select_ragged(self, scores: np.ndarray, descs: Sequence[Sequence[int]]):
+        """scores fp32 [sum n] concatenated, descs [(t, h, w, region_h, region_w, m, k)] ->
+        (segment-local keep indices [sum k], the same tokens numbered over the concatenation)."""
+        scores = np.ascontiguousarray(scores, dtype=np.float32).reshape(-1)
+        d = np.ascontiguousarray(np.asarray(descs, dtype=np.int32).reshape(-1, 7))
+        assert scores.size == int(sum(int(r[0]) * int(r[1]) * int(r[2]) for r in d))
+        total_k = int(d[:, 6].sum()) if len(d) else 0
+        keep = np.full(total_k, -1, dtype=np.int32)
+        flat = np.full(total_k, -1, dtype=np.int32)
+        _check(self.h.oracle_select_ragged(_f32p(scores), len(d), _i32p(d), _i32p(keep), _i32p(flat)),
+               "oracle_select_ragged")
+        return keep, flat
 
     def set_threads(self, n: int) -> int:
         return int(self.h.oracle_set_threads(n))

@@ -27,6 +27,10 @@
  *   compaction       out[j] = in[index[j]] row by row (bytes, never interpreted)
  *   sequence index   text positions (always kept) and vis_start + kept visual
  *                    indices, ascending
+ *   merge            Eq. 13: text rows with the visual span replaced by the kept visual rows
+ *   other layouts    plane-major position ids, head-major K/V, paged K/V destinations:
+ *                    the same row moves with other address arithmetic
+ *   ragged batch     one selection per segment, each with its own grid, floor and budget
  *
  * Everything is done by sorting with the comparator above and by memcpy: no bit
  * tricks, no histograms, no scans.
@@ -279,6 +283,161 @@ int oracle_compact_kv(const void* const* k_src, const void* const* v_src, void* 
         for (int j = 0; j < s_out; ++j)
             memcpy(dst + (size_t)j * row_bytes,
                    src + (size_t)seq_idx[(size_t)s * s_out + j] * row_bytes, row_bytes);
+    }
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------
+ * Steps adjacent to the core path (same semantics, other layouts)
+ * ------------------------------------------------------------------------------------ */
+
+/* Eq. 13: the compact prefill sequence is Merge(E_x, V_c) -- the text embeddings with the
+ * dense visual placeholder span [vis_start, vis_start + n_vis) replaced by the compact visual
+ * rows V_c, where V_c are the kept rows of the dense visual sequence in source order (Eq. 12,
+ * Section 3.5).  text [n_seq, seq_len, row_bytes] (rows inside the span are placeholders and
+ * are never read), visual [n_seq, n_vis, row_bytes], keep_idx [n_seq, k] ->
+ * merged [n_seq, seq_len - n_vis + k, row_bytes]. */
+int oracle_merge_embeddings(const void* text, const void* visual, size_t row_bytes,
+                            const int32_t* keep_idx, int n_seq, int seq_len, int vis_start,
+                            int n_vis, int k, void* merged)
+{
+    if (!text || !visual || !merged || n_seq < 0 || seq_len < 0 || vis_start < 0 || n_vis < 0 ||
+        k < 0 || k > n_vis || vis_start + n_vis > seq_len || (k > 0 && !keep_idx))
+        return ORACLE_ERR_ARG;
+    int s_out = seq_len - n_vis + k;
+    char* v_c = (char*)malloc((size_t)(k > 0 ? k : 1) * row_bytes);
+    if (!v_c) return ORACLE_ERR_NOMEM;
+    for (int s = 0; s < n_seq; ++s) {
+        const char* e_x = (const char*)text + (size_t)s * seq_len * row_bytes;
+        const char* v = (const char*)visual + (size_t)s * n_vis * row_bytes;
+        char* out = (char*)merged + (size_t)s * s_out * row_bytes;
+        /* V_c: the kept visual rows, in order */
+        for (int j = 0; j < k; ++j) {
+            int32_t i = keep_idx[(size_t)s * k + j];
+            if (i < 0 || i >= n_vis) { free(v_c); return ORACLE_ERR_INDEX; }
+            memcpy(v_c + (size_t)j * row_bytes, v + (size_t)i * row_bytes, row_bytes);
+        }
+        /* text before the span | V_c | text behind the span */
+        memcpy(out, e_x, (size_t)vis_start * row_bytes);
+        memcpy(out + (size_t)vis_start * row_bytes, v_c, (size_t)k * row_bytes);
+        memcpy(out + (size_t)(vis_start + k) * row_bytes,
+               e_x + (size_t)(vis_start + n_vis) * row_bytes,
+               (size_t)(seq_len - vis_start - n_vis) * row_bytes);
+    }
+    free(v_c);
+    return ORACLE_OK;
+}
+
+/* Section 3.5 for position ids stored plane-major, pos [n_planes, n_seq, seq_len] (the three
+ * planes are t, h, w): text positions are preserved and compact visual positions inherited, so
+ * out[c, s, j] = pos[c, s, seq_idx[s, j]].  out [n_planes, n_seq, s_out]. */
+int oracle_compact_pos_planes(const int32_t* pos, int n_planes, int n_seq, int seq_len,
+                              const int32_t* seq_idx, int s_out, int32_t* out)
+{
+    if (!pos || !seq_idx || !out || n_planes < 0 || n_seq < 0 || seq_len < 0 || s_out < 0)
+        return ORACLE_ERR_ARG;
+    for (int c = 0; c < n_planes; ++c)
+        for (int s = 0; s < n_seq; ++s)
+            for (int j = 0; j < s_out; ++j) {
+                int32_t i = seq_idx[(size_t)s * s_out + j];
+                if (i < 0 || i >= seq_len) return ORACLE_ERR_INDEX;
+                out[((size_t)c * n_seq + s) * s_out + j] = pos[((size_t)c * n_seq + s) * seq_len + i];
+            }
+    return ORACLE_OK;
+}
+
+/* The prefill cache of Eq. 14 with head-major tensors: src[l] is [n_seq, n_heads, seq_len,
+ * head_bytes], dst[l] is [n_seq, n_heads, s_out, head_bytes];
+ * dst[l][s, h, j, :] = src[l][s, h, seq_idx[s, j], :] for K and for V. */
+int oracle_compact_kv_heads(const void* const* k_src, const void* const* v_src, void* const* k_dst,
+                            void* const* v_dst, int n_layers, int n_seq, int n_heads, int seq_len,
+                            int s_out, size_t head_bytes, const int32_t* seq_idx)
+{
+    if (!k_src || !v_src || !k_dst || !v_dst || !seq_idx || n_layers < 0 || n_seq < 0 ||
+        n_heads < 0 || seq_len < 0 || s_out < 0)
+        return ORACLE_ERR_ARG;
+    for (int s = 0; s < n_seq; ++s)
+        for (int j = 0; j < s_out; ++j) {
+            int32_t i = seq_idx[(size_t)s * s_out + j];
+            if (i < 0 || i >= seq_len) return ORACLE_ERR_INDEX;
+        }
+    for (int l = 0; l < n_layers; ++l)
+        for (int which = 0; which < 2; ++which)
+            for (int s = 0; s < n_seq; ++s)
+                for (int h = 0; h < n_heads; ++h) {
+                    const char* src = (const char*)(which ? v_src[l] : k_src[l]) +
+                                      ((size_t)s * n_heads + h) * seq_len * head_bytes;
+                    char* dst = (char*)(which ? v_dst[l] : k_dst[l]) +
+                                ((size_t)s * n_heads + h) * s_out * head_bytes;
+                    for (int j = 0; j < s_out; ++j)
+                        memcpy(dst + (size_t)j * head_bytes,
+                               src + (size_t)seq_idx[(size_t)s * s_out + j] * head_bytes, head_bytes);
+                }
+    return ORACLE_OK;
+}
+
+/* The prefill cache of Eq. 14 written into a paged cache.  Every layer's K and V cache is
+ * [n_pages, page_size, row_bytes]; sequence s owns the pages block_table[s, 0 .. ], and its
+ * compact position j lives in page block_table[s, j / page_size] at slot j % page_size:
+ * cache[l][page, slot, :] = src[l][s, seq_idx[s, j], :].  src [n_seq, seq_len, row_bytes].
+ * Nothing else in the cache is written. */
+int oracle_compact_kv_paged(const void* const* k_src, const void* const* v_src,
+                            void* const* k_cache, void* const* v_cache, int n_layers, int n_seq,
+                            int seq_len, int s_out, size_t row_bytes, const int32_t* seq_idx,
+                            const int32_t* block_table, int max_pages_per_seq, int page_size,
+                            int n_pages)
+{
+    if (!k_src || !v_src || !k_cache || !v_cache || !seq_idx || !block_table || n_layers < 0 ||
+        n_seq < 0 || seq_len < 0 || s_out < 0 || page_size <= 0 || max_pages_per_seq < 0 ||
+        n_pages < 0)
+        return ORACLE_ERR_ARG;
+    if ((int64_t)max_pages_per_seq * page_size < s_out) return ORACLE_ERR_ARG;
+    for (int l = 0; l < n_layers; ++l)
+        for (int which = 0; which < 2; ++which)
+            for (int s = 0; s < n_seq; ++s) {
+                const char* src = (const char*)(which ? v_src[l] : k_src[l]) +
+                                  (size_t)s * seq_len * row_bytes;
+                char* cache = (char*)(which ? v_cache[l] : k_cache[l]);
+                for (int j = 0; j < s_out; ++j) {
+                    int32_t i = seq_idx[(size_t)s * s_out + j];
+                    int32_t page = block_table[(size_t)s * max_pages_per_seq + j / page_size];
+                    int slot = j % page_size;
+                    if (i < 0 || i >= seq_len || page < 0 || page >= n_pages) return ORACLE_ERR_INDEX;
+                    memcpy(cache + ((size_t)page * page_size + slot) * row_bytes,
+                           src + (size_t)i * row_bytes, row_bytes);
+                }
+            }
+    return ORACLE_OK;
+}
+
+/* Table 2's "Min Keep Ratio" as a per-region token count: the smallest m with
+ * m >= ratio * region_h * region_w for ratio = num / den (0.0 -> 0, plain top-K). */
+int64_t oracle_floor_from_ratio(int region_h, int region_w, int num, int den)
+{
+    if (region_h <= 0 || region_w <= 0 || num < 0 || den <= 0 || num > den) return -1;
+    int64_t size = (int64_t)region_h * region_w, m = 0;
+    while (m * den < size * num) ++m;
+    return m;
+}
+
+/* Ragged batch: segment s has its own grid, floor and budget, desc[s] = {t, h, w, region_h,
+ * region_w, m, k}.  Scores are concatenated (segment s starts at the sum of the earlier
+ * segments' n), keep_idx likewise (sum of the earlier k); indices are segment-local.  flat_idx
+ * (optional) holds the same tokens numbered over the concatenated scores. */
+int oracle_select_ragged(const float* scores, int n_seg, const int32_t* desc, int32_t* keep_idx,
+                         int32_t* flat_idx)
+{
+    if (!desc || n_seg < 0) return ORACLE_ERR_ARG;
+    int64_t tok0 = 0, out0 = 0;
+    for (int s = 0; s < n_seg; ++s) {
+        const int32_t* d = desc + (size_t)s * 7;
+        int rc = oracle_select(scores + tok0, 1, d[0], d[1], d[2], d[3], d[4], d[5], d[6],
+                               keep_idx + out0);
+        if (rc != ORACLE_OK) return rc;
+        if (flat_idx)
+            for (int j = 0; j < d[6]; ++j) flat_idx[out0 + j] = (int32_t)(tok0 + keep_idx[out0 + j]);
+        tok0 += (int64_t)d[0] * d[1] * d[2];
+        out0 += d[6];
     }
     return ORACLE_OK;
 }

@@ -397,8 +397,156 @@ def pin_cache_ratio(o, golden_path):
     assert (L + M_p, L + T_p) == (405, 1088)
 
 
+# ---------------------------------------------------------------- adjacent steps
+
+def _sorted_choice(rng, n, k, rows):
+    return np.stack([np.sort(rng.choice(n, k, replace=False)) for _ in range(rows)]).astype(np.int32) \
+        if k else np.zeros((rows, 0), np.int32)
+
+
+def pin_merge_embeddings(o):
+    """Eq. 13: text rows with the visual span replaced by the kept visual rows -- numpy's own
+    concatenate; the length is L + M_p; keeping everything is the dense merge (Eq. 1); and the
+    compact merge is the dense merge with the dropped rows taken out (sequence indices)."""
+    rng = np.random.default_rng(37)
+    for n_seq, seq_len, vis_start, n_vis, k, row in [(2, 20, 3, 12, 5, 8), (3, 12, 0, 12, 4, 6),
+                                                     (1, 15, 5, 10, 10, 4), (2, 9, 9, 0, 0, 2),
+                                                     (2, 30, 23, 7, 0, 10), (2, 40, 4, 30, 11, 34)]:
+        text = rng.integers(0, 2 ** 16, (n_seq, seq_len, row), dtype=np.uint16)
+        visual = rng.integers(0, 2 ** 16, (n_seq, n_vis, row), dtype=np.uint16)
+        keep = _sorted_choice(rng, n_vis, k, n_seq)
+        got = o.merge_embeddings(text, visual, keep, vis_start)
+        assert got.shape == (n_seq, seq_len - n_vis + k, row)
+        dense = text.copy()
+        dense[:, vis_start:vis_start + n_vis] = visual
+        idx = o.seq_indices(keep, seq_len, vis_start, n_vis)
+        for b in range(n_seq):
+            want = np.concatenate([text[b, :vis_start], visual[b][keep[b]], text[b, vis_start + n_vis:]])
+            assert got[b].tobytes() == want.tobytes()
+            assert got[b].tobytes() == dense[b][idx[b]].tobytes()
+        everything = np.tile(np.arange(n_vis, dtype=np.int32), (n_seq, 1))
+        assert o.merge_embeddings(text, visual, everything, vis_start).tobytes() == dense.tobytes()
+
+
+def pin_pos_planes(o):
+    """Plane-major position ids: numpy's take_along_axis; agrees with the row layout [.., 3]."""
+    rng = np.random.default_rng(41)
+    for n_planes, n_seq, seq_len, s_out in [(3, 2, 17, 6), (3, 4, 40, 40), (1, 1, 5, 1), (4, 2, 9, 0)]:
+        pos = rng.integers(-3, 5000, (n_planes, n_seq, seq_len)).astype(np.int32)
+        idx = _sorted_choice(rng, seq_len, s_out, n_seq)
+        got = o.compact_pos_planes(pos, idx)
+        want = np.take_along_axis(pos, np.broadcast_to(idx[None], (n_planes, n_seq, s_out)), axis=2)
+        assert np.array_equal(got, want)
+        if n_planes == 3 and s_out:
+            _, rows = o.compact(None, np.ascontiguousarray(pos.transpose(1, 2, 0)), idx)
+            assert np.array_equal(got, rows.transpose(2, 0, 1))
+
+
+def pin_kv_heads(o):
+    """Head-major K/V: numpy indexing on the token axis, and the transposed token-major result."""
+    rng = np.random.default_rng(43)
+    n_layers, n_seq, n_heads, seq_len, s_out, d = 2, 3, 4, 23, 9, 6
+    ks = [rng.integers(0, 2 ** 16, (n_seq, n_heads, seq_len, d), dtype=np.uint16) for _ in range(n_layers)]
+    vs = [rng.integers(0, 2 ** 16, (n_seq, n_heads, seq_len, d), dtype=np.uint16) for _ in range(n_layers)]
+    idx = _sorted_choice(rng, seq_len, s_out, n_seq)
+    kd, vd = o.compact_kv_heads(ks, vs, idx)
+    tok = lambda a: np.ascontiguousarray(a.transpose(0, 2, 1, 3)).reshape(n_seq, a.shape[2], n_heads * d)
+    kt, vt = o.compact_kv([tok(a) for a in ks], [tok(a) for a in vs], idx)
+    for l in range(n_layers):
+        for b in range(n_seq):
+            assert kd[l][b].tobytes() == ks[l][b][:, idx[b]].tobytes()
+            assert vd[l][b].tobytes() == vs[l][b][:, idx[b]].tobytes()
+        assert np.array_equal(tok(kd[l]), kt[l]) and np.array_equal(tok(vd[l]), vt[l])
+
+
+def pin_kv_paged(o):
+    """Paged destination: reading the cache back through the block table gives the kept rows;
+    every other slot keeps its old contents; page size 1 with an identity table is the
+    contiguous compaction."""
+    rng = np.random.default_rng(47)
+    for n_seq, seq_len, s_out, row, page in [(3, 29, 13, 8, 4), (2, 16, 16, 4, 16), (2, 21, 7, 6, 1),
+                                            (1, 10, 10, 2, 3)]:
+        n_layers = 2
+        per_seq = -(-s_out // page) + 1  # one spare table entry per sequence, never used
+        n_pages = n_seq * per_seq + 3
+        table = rng.permutation(n_pages)[: n_seq * per_seq].reshape(n_seq, per_seq).astype(np.int32)
+        ks = [rng.integers(0, 2 ** 15, (n_seq, seq_len, row), dtype=np.uint16) for _ in range(n_layers)]
+        vs = [rng.integers(0, 2 ** 15, (n_seq, seq_len, row), dtype=np.uint16) for _ in range(n_layers)]
+        idx = _sorted_choice(rng, seq_len, s_out, n_seq)
+        kc = [np.full((n_pages, page, row), 0xFFFF, dtype=np.uint16) for _ in range(n_layers)]
+        vc = [np.full((n_pages, page, row), 0xFFFE, dtype=np.uint16) for _ in range(n_layers)]
+        o.compact_kv_paged(ks, vs, idx, table, page, kc, vc)
+        for l in range(n_layers):
+            written = np.zeros((n_pages, page), dtype=bool)
+            for b in range(n_seq):
+                for j in range(s_out):
+                    pg, slot = table[b, j // page], j % page
+                    assert np.array_equal(kc[l][pg, slot], ks[l][b, idx[b, j]])
+                    assert np.array_equal(vc[l][pg, slot], vs[l][b, idx[b, j]])
+                    written[pg, slot] = True
+            assert np.all(kc[l][~written] == 0xFFFF) and np.all(vc[l][~written] == 0xFFFE)
+    # page size 1, identity table: the contiguous compaction
+    n_seq, seq_len, s_out, row = 2, 19, 8, 4
+    ks = [rng.integers(0, 2 ** 15, (n_seq, seq_len, row), dtype=np.uint16)]
+    idx = _sorted_choice(rng, seq_len, s_out, n_seq)
+    table = np.arange(n_seq * s_out, dtype=np.int32).reshape(n_seq, s_out)
+    kc = [np.zeros((n_seq * s_out, 1, row), dtype=np.uint16)]
+    vc = [np.zeros((n_seq * s_out, 1, row), dtype=np.uint16)]
+    o.compact_kv_paged(ks, ks, idx, table, 1, kc, vc)
+    kd, _ = o.compact_kv(ks, ks, idx)
+    assert kc[0].tobytes() == kd[0].tobytes() and vc[0].tobytes() == kd[0].tobytes()
+
+
+def pin_floor_from_ratio(o):
+    """Table 2's Min Keep Ratio values on the benchmark's tiles: exact rational ceiling."""
+    from fractions import Fraction
+
+    assert [o.floor_from_ratio(4, 4, n, d) for n, d in [(0, 1), (1, 5), (1, 2)]] == [0, 4, 8]
+    assert [o.floor_from_ratio(2, 2, n, d) for n, d in [(0, 1), (1, 5), (1, 2)]] == [0, 1, 2]
+    for rh in range(1, 7):
+        for rw in range(1, 7):
+            for den in range(1, 9):
+                for num in range(0, den + 1):
+                    assert o.floor_from_ratio(rh, rw, num, den) == math.ceil(Fraction(num, den) * rh * rw)
+    assert o.floor_from_ratio(4, 4, 1, 1) == 16
+    assert o.floor_from_ratio(4, 4, 3, 2) == -1 and o.floor_from_ratio(0, 4, 1, 2) == -1
+
+
+def pin_select_ragged(o):
+    """A ragged batch is the per-segment selection laid end to end: invariants hold segment by
+    segment, offsets follow numpy's cumulative sums, and tiny segments match the brute force."""
+    rng = np.random.default_rng(53)
+    for trial in range(12):
+        descs, parts = [], []
+        for _ in range(int(rng.integers(1, 6))):
+            t, h, w = int(rng.integers(1, 3)), int(rng.integers(1, 7)), int(rng.integers(1, 7))
+            rh, rw = int(rng.integers(1, h + 1)), int(rng.integers(1, w + 1))
+            m = int(rng.integers(0, 3))
+            n = t * h * w
+            n_res = int(floor_need(region_ids(t, h, w, rh, rw), m).sum())
+            k = int(rng.integers(n_res, n + 1))
+            descs.append((t, h, w, rh, rw, m, k))
+            parts.append((rng.integers(0, 4, n) if trial % 2 else rng.random(n)).astype(np.float32))
+        scores = np.concatenate(parts)
+        keep, flat = o.select_ragged(scores, descs)
+        tok0 = np.concatenate([[0], np.cumsum([d[0] * d[1] * d[2] for d in descs])])
+        out0 = np.concatenate([[0], np.cumsum([d[6] for d in descs])])
+        assert len(keep) == out0[-1] and len(flat) == out0[-1]
+        for s, (d, part) in enumerate(zip(descs, parts)):
+            mine = keep[out0[s]:out0[s + 1]]
+            check_invariants(part, *d, mine)
+            assert np.array_equal(flat[out0[s]:out0[s + 1]], mine + tok0[s])
+            if len(part) <= 10:
+                want = best_feasible_subset(part, region_ids(*d[:5]), d[5], d[6])
+                assert list(mine) == list(want)
+        if len(flat):
+            assert np.all(np.diff(flat) > 0), "tokens of the concatenation stay in source order"
+
+
 ALL_SELECT_PINS = [pin_total_order, pin_special_values_in_select, pin_plain_topk_is_stable_argsort,
                    pin_bruteforce_tiny, pin_full_sort_tiny, pin_invariants_on_workloads,
                    pin_invariants_random, pin_floor_inactive, pin_repair_formulation,
                    pin_hand_worked_example, pin_error_codes]
 ALL_COMPACT_PINS = [pin_compact_is_take, pin_seq_indices, pin_compact_kv_is_take]
+ALL_ADJACENT_PINS = [pin_merge_embeddings, pin_pos_planes, pin_kv_heads, pin_kv_paged, pin_floor_from_ratio,
+                     pin_select_ragged]

@@ -54,11 +54,38 @@ MUTANTS = {
         "if (keep_idx[(size_t)s * k + j] == p - vis_start) kept = 1;",
         "if (keep_idx[(size_t)s * k + j] == p) kept = 1;"),
     "kv_v_reads_k": (
-        "const char* src = (const char*)(which ? v_src[l] : k_src[l])",
-        "const char* src = (const char*)(which ? k_src[l] : k_src[l])"),
+        "const char* src = (const char*)(which ? v_src[l] : k_src[l]) + (size_t)s * seq_len * row_bytes;",
+        "const char* src = (const char*)(which ? k_src[l] : k_src[l]) + (size_t)s * seq_len * row_bytes;"),
     "kv_wrong_sequence_index_row": (
         "src + (size_t)seq_idx[(size_t)s * s_out + j] * row_bytes, row_bytes);",
         "src + (size_t)seq_idx[j] * row_bytes, row_bytes);"),
+    "merge_tail_text_from_wrong_offset": (
+        "e_x + (size_t)(vis_start + n_vis) * row_bytes,",
+        "e_x + (size_t)(vis_start + k) * row_bytes,"),
+    "merge_visual_rows_not_gathered": (
+        "memcpy(v_c + (size_t)j * row_bytes, v + (size_t)i * row_bytes, row_bytes);",
+        "memcpy(v_c + (size_t)j * row_bytes, v + (size_t)j * row_bytes, row_bytes);"),
+    "pos_planes_wrong_plane_stride": (
+        "out[((size_t)c * n_seq + s) * s_out + j] = pos[((size_t)c * n_seq + s) * seq_len + i];",
+        "out[((size_t)c * n_seq + s) * s_out + j] = pos[((size_t)s * n_seq + c) * seq_len + i];"),
+    "kv_heads_source_uses_compact_stride": (
+        "((size_t)s * n_heads + h) * seq_len * head_bytes;",
+        "((size_t)s * n_heads + h) * s_out * head_bytes;"),
+    "paged_slot_and_page_swapped": (
+        "int slot = j % page_size;",
+        "int slot = (j / page_size) % page_size;"),
+    "paged_table_row_stride": (
+        "block_table[(size_t)s * max_pages_per_seq + j / page_size];",
+        "block_table[(size_t)s * (max_pages_per_seq - 1) + j / page_size];"),
+    "ratio_floor_rounds_down": (
+        "while (m * den < size * num) ++m;",
+        "while ((m + 1) * den <= size * num) ++m;"),
+    "ragged_flat_index_forgets_offset": (
+        "flat_idx[out0 + j] = (int32_t)(tok0 + keep_idx[out0 + j]);",
+        "flat_idx[out0 + j] = (int32_t)(keep_idx[out0 + j]);"),
+    "ragged_scores_not_advanced": (
+        "tok0 += (int64_t)d[0] * d[1] * d[2];",
+        "tok0 += (int64_t)d[1] * d[2];"),
 }
 
 
@@ -78,7 +105,7 @@ def _build_mutant(tmp_path, name):
 def test_mutant_is_caught(tmp_path, name):
     mutant = _build_mutant(tmp_path, name)
     caught = []
-    for pin in pins.ALL_SELECT_PINS + pins.ALL_COMPACT_PINS:
+    for pin in pins.ALL_SELECT_PINS + pins.ALL_COMPACT_PINS + pins.ALL_ADJACENT_PINS:
         try:
             pin(mutant)
         except (AssertionError, oracle.OracleError):
