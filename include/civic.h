@@ -150,6 +150,84 @@ civic_status_t civic_compact_kv(const void* const* k_src, const void* const* v_s
                                 int32_t n_seq, int32_t seq_len, int32_t s_out, size_t row_bytes,
                                 const int32_t* seq_idx, void* stream);
 
+/*
+ * civic_compact_kv_heads -- civic_compact_kv for head-major cache tensors.
+ *
+ * Paper: as civic_compact_kv (Eq. 2 / Eq. 7 storage term, Eq. 14 cache ratio); only the memory
+ * layout differs: every tensor is [n_seq, n_heads, seq_len, head_bytes], so a token's row is
+ * n_heads separate pieces of head_bytes (head_dim * element size, e.g. 256).
+ *   k_dst[l][s, h, j, :] = k_src[l][s, h, seq_idx[s, j], :]   (same for v)
+ *
+ * k_src, v_src  host arrays of n_layers dev pointers, each [n_seq, n_heads, seq_len, head_bytes]
+ * k_dst, v_dst  host arrays of n_layers dev pointers, each [n_seq, n_heads, s_out,  head_bytes]
+ * head_bytes    multiple of 4; short pieces are packed several to a warp so that the moves stay
+ *               16-byte vectorised
+ * seq_idx       dev [n_seq, s_out] int32, values in [0, seq_len), shared by heads and layers
+ */
+civic_status_t civic_compact_kv_heads(const void* const* k_src, const void* const* v_src,
+                                      void* const* k_dst, void* const* v_dst, int32_t n_layers,
+                                      int32_t n_seq, int32_t n_heads, int32_t seq_len, int32_t s_out,
+                                      size_t head_bytes, const int32_t* seq_idx, void* stream);
+
+/*
+ * civic_compact_kv_paged -- civic_compact_kv writing straight into a paged cache.
+ *
+ * Paper: as civic_compact_kv; the destination is the serving engine's block-structured cache
+ * instead of a dense tensor, so the compact prefill cache never exists in a second copy.
+ * Compact position j of sequence s goes to page block_table[s, j / page_size], slot
+ * j % page_size:   k_cache[l][page, slot, :] = k_src[l][s, seq_idx[s, j], :]   (same for v)
+ *
+ * k_src, v_src      host arrays of n_layers dev pointers, each [n_seq, seq_len, row_bytes]
+ * k_cache, v_cache  host arrays of n_layers dev pointers, each [n_pages, page_size, row_bytes];
+ *                   only the addressed slots are written
+ * block_table       dev [n_seq, max_pages_per_seq] int32, page numbers in [0, n_pages); the
+ *                   first ceil(s_out / page_size) entries of every row are used.  Distinct
+ *                   sequences must own distinct pages (the caller's contract, like index validity)
+ * max_pages_per_seq * page_size < s_out is CIVIC_ERR_INVALID_ARG.
+ */
+civic_status_t civic_compact_kv_paged(const void* const* k_src, const void* const* v_src,
+                                      void* const* k_cache, void* const* v_cache, int32_t n_layers,
+                                      int32_t n_seq, int32_t seq_len, int32_t s_out, size_t row_bytes,
+                                      const int32_t* seq_idx, const int32_t* block_table,
+                                      int32_t max_pages_per_seq, int32_t page_size, int32_t n_pages,
+                                      void* stream);
+
+/*
+ * civic_merge_embeddings -- the compact prefill sequence as data.
+ *
+ * Paper: Eq. 13, x_c = Merge(E_x, V_c): the text embeddings with the dense visual placeholder
+ * span replaced by the compact visual rows (Eq. 12), length L + M_p.  Built in one pass from the
+ * DENSE visual rows and the keep indices, without materialising V_c:
+ *   merged[s, j, :] = text[s, j, :]                                  j <  vis_start
+ *                   = visual[s, keep_idx[s, j - vis_start], :]       vis_start <= j < vis_start + k
+ *                   = text[s, j - k + n_vis, :]                      otherwise
+ *
+ * text      dev [n_seq, seq_len, row_bytes]; rows inside [vis_start, vis_start + n_vis) are
+ *           placeholders and are never read
+ * visual    dev [n_seq, n_vis, row_bytes]
+ * keep_idx  dev [n_seq, k] int32 ascending, values in [0, n_vis)
+ * merged    dev [n_seq, seq_len - n_vis + k, row_bytes], written
+ */
+civic_status_t civic_merge_embeddings(const void* text, const void* visual, size_t row_bytes,
+                                      const int32_t* keep_idx, int32_t n_seq, int32_t seq_len,
+                                      int32_t vis_start, int32_t n_vis, int32_t k, void* merged,
+                                      void* stream);
+
+/*
+ * civic_compact_pos_planes -- position ids of the compact sequence, plane-major layout.
+ *
+ * Paper: Section 3.5 (text positions preserved, compact visual positions inherited), for ids
+ * stored as [n_planes, n_seq, seq_len] (planes t, h, w) over the FULL multimodal sequence:
+ *   pos_out[c, s, j] = pos[c, s, seq_idx[s, j]]
+ *
+ * pos      dev [n_planes, n_seq, seq_len] int32
+ * seq_idx  dev [n_seq, s_out] int32, values in [0, seq_len)
+ * pos_out  dev [n_planes, n_seq, s_out] int32, written
+ */
+civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, int32_t n_seq,
+                                        int32_t seq_len, const int32_t* seq_idx, int32_t s_out,
+                                        int32_t* pos_out, void* stream);
+
 /* Static, human-readable name of a status. */
 const char* civic_status_string(civic_status_t status);
 

@@ -25,7 +25,9 @@ STATUS_NAMES = ("CIVIC_OK", "CIVIC_ERR_INVALID_ARG", "CIVIC_ERR_K_RANGE", "CIVIC
 # every symbol include/civic.h declares
 EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "civic_compact",
            "civic_seq_indices", "civic_compact_kv", "civic_status_string", "civic_last_cuda_error",
-           "civic_launch_count", "civic_select_seq", "civic_set_programmatic_launch")
+           "civic_launch_count", "civic_select_seq", "civic_set_programmatic_launch",
+           "civic_compact_kv_heads", "civic_compact_kv_paged", "civic_merge_embeddings",
+           "civic_compact_pos_planes")
 
 
 class CivicError(RuntimeError):
@@ -79,6 +81,15 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_select_seq.restype = ctypes.c_int
     lib.civic_set_programmatic_launch.argtypes = [i32]
     lib.civic_set_programmatic_launch.restype = i32
+    lib.civic_compact_kv_heads.argtypes = [vpp, vpp, vpp, vpp, i32, i32, i32, i32, i32, sz, vp, vp]
+    lib.civic_compact_kv_heads.restype = ctypes.c_int
+    lib.civic_compact_kv_paged.argtypes = [vpp, vpp, vpp, vpp, i32, i32, i32, i32, sz, vp, vp, i32, i32,
+                                           i32, vp]
+    lib.civic_compact_kv_paged.restype = ctypes.c_int
+    lib.civic_merge_embeddings.argtypes = [vp, vp, sz, vp, i32, i32, i32, i32, i32, vp, vp]
+    lib.civic_merge_embeddings.restype = ctypes.c_int
+    lib.civic_compact_pos_planes.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp]
+    lib.civic_compact_pos_planes.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -282,3 +293,118 @@ def civic_compact_kv(tables: KVTables, seq_idx: torch.Tensor,
                                        tables.n_layers, tables.n_seq, tables.seq_len, tables.s_out,
                                        tables.row_bytes, idx_ptr, _stream_ptr(stream)),
                "civic_compact_kv")
+
+
+def _table(ts: Sequence[torch.Tensor], what: str) -> ctypes.Array:
+    return (ctypes.c_void_p * len(ts))(*[_dev_ptr(t, what) for t in ts])
+
+
+def _same(ts: Sequence[torch.Tensor], what: str):
+    shape, dtype = tuple(ts[0].shape), ts[0].dtype
+    for t in ts:
+        if tuple(t.shape) != shape or t.dtype != dtype:
+            raise ValueError(f"all {what} tensors must share shape and dtype")
+    return shape, dtype
+
+
+def civic_compact_kv_heads(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
+                           k_dst: Sequence[torch.Tensor], v_dst: Sequence[torch.Tensor],
+                           seq_idx: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Head-major caches: [n_seq, n_heads, seq_len, d] -> [n_seq, n_heads, s_out, d] per layer."""
+    n_layers = len(k_src)
+    if n_layers == 0 or not (len(v_src) == len(k_dst) == len(v_dst) == n_layers):
+        raise ValueError("the four tensor lists must have one entry per layer")
+    src_shape, dtype = _same(list(k_src) + list(v_src), "source")
+    dst_shape, dst_dtype = _same(list(k_dst) + list(v_dst), "destination")
+    if len(src_shape) != 4 or len(dst_shape) != 4 or dst_dtype != dtype or \
+            src_shape[:2] != dst_shape[:2] or src_shape[3] != dst_shape[3]:
+        raise ValueError("source [n_seq, n_heads, seq_len, d] and destination [n_seq, n_heads, s_out, d] disagree")
+    n_seq, n_heads, seq_len, d = src_shape
+    s_out = dst_shape[2]
+    if tuple(seq_idx.shape) != (n_seq, s_out):
+        raise ValueError("seq_idx must be [n_seq, s_out]")
+    idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
+    with torch.cuda.device(_device_of(seq_idx, k_src[0], k_dst[0])):
+        _check(load().civic_compact_kv_heads(_table(k_src, "k_src"), _table(v_src, "v_src"),
+                                             _table(k_dst, "k_dst"), _table(v_dst, "v_dst"), n_layers,
+                                             n_seq, n_heads, seq_len, s_out, d * k_src[0].element_size(),
+                                             idx_ptr, _stream_ptr(stream)), "civic_compact_kv_heads")
+
+
+def civic_compact_kv_paged(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
+                           k_cache: Sequence[torch.Tensor], v_cache: Sequence[torch.Tensor],
+                           seq_idx: torch.Tensor, block_table: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Token-major sources [n_seq, seq_len, ...] into paged caches [n_pages, page_size, ...]
+    through block_table int32 [n_seq, max_pages_per_seq]."""
+    n_layers = len(k_src)
+    if n_layers == 0 or not (len(v_src) == len(k_cache) == len(v_cache) == n_layers):
+        raise ValueError("the four tensor lists must have one entry per layer")
+    src_shape, dtype = _same(list(k_src) + list(v_src), "source")
+    cache_shape, cache_dtype = _same(list(k_cache) + list(v_cache), "cache")
+    if len(src_shape) < 3 or len(cache_shape) != len(src_shape) or cache_dtype != dtype or \
+            src_shape[2:] != cache_shape[2:]:
+        raise ValueError("source [n_seq, seq_len, ...] and cache [n_pages, page_size, ...] disagree")
+    n_seq, seq_len = src_shape[:2]
+    n_pages, page_size = cache_shape[:2]
+    row_elems = 1
+    for d in src_shape[2:]:
+        row_elems *= d
+    if seq_idx.dim() != 2 or seq_idx.shape[0] != n_seq:
+        raise ValueError("seq_idx must be [n_seq, s_out]")
+    if block_table.dim() != 2 or block_table.shape[0] != n_seq:
+        raise ValueError("block_table must be [n_seq, max_pages_per_seq]")
+    idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
+    tab_ptr = _dev_ptr(block_table, "block_table", torch.int32)
+    with torch.cuda.device(_device_of(seq_idx, k_src[0], k_cache[0])):
+        _check(load().civic_compact_kv_paged(_table(k_src, "k_src"), _table(v_src, "v_src"),
+                                             _table(k_cache, "k_cache"), _table(v_cache, "v_cache"),
+                                             n_layers, n_seq, seq_len, seq_idx.shape[1],
+                                             row_elems * k_src[0].element_size(), idx_ptr, tab_ptr,
+                                             block_table.shape[1], page_size, n_pages,
+                                             _stream_ptr(stream)), "civic_compact_kv_paged")
+
+
+def civic_merge_embeddings(text: torch.Tensor, visual: torch.Tensor, keep_idx: torch.Tensor,
+                           vis_start: int, merged: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """text [n_seq, seq_len, D], dense visual [n_seq, n_vis, D], keep_idx [n_seq, k] ->
+    merged [n_seq, seq_len - n_vis + k, D] (Eq. 13)."""
+    if text.dim() != 3 or visual.dim() != 3 or text.shape[0] != visual.shape[0] or \
+            text.shape[2] != visual.shape[2] or text.dtype != visual.dtype:
+        raise ValueError("text [n_seq, seq_len, D] and visual [n_seq, n_vis, D] disagree")
+    n_seq, seq_len, dim = text.shape
+    n_vis = visual.shape[1]
+    if keep_idx.dim() != 2 or keep_idx.shape[0] != n_seq:
+        raise ValueError("keep_idx must be [n_seq, k]")
+    k = keep_idx.shape[1]
+    s_out = seq_len - n_vis + k
+    if merged is None:
+        merged = torch.empty((n_seq, max(s_out, 0), dim), dtype=text.dtype, device=_device_of(keep_idx, text))
+    elif tuple(merged.shape) != (n_seq, s_out, dim) or merged.dtype != text.dtype:
+        raise ValueError("merged must be [n_seq, seq_len - n_vis + k, D] of text's dtype")
+    args = (_dev_ptr(text, "text"), _dev_ptr(visual, "visual"), dim * text.element_size(),
+            _dev_ptr(keep_idx, "keep_idx", torch.int32), n_seq, seq_len, vis_start, n_vis, k,
+            _dev_ptr(merged, "merged"))
+    with torch.cuda.device(_device_of(keep_idx, text, visual)):
+        _check(load().civic_merge_embeddings(*args, _stream_ptr(stream)), "civic_merge_embeddings")
+    return merged
+
+
+def civic_compact_pos_planes(pos: torch.Tensor, seq_idx: torch.Tensor,
+                             pos_out: Optional[torch.Tensor] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """pos int32 [n_planes, n_seq, seq_len], seq_idx [n_seq, s_out] -> [n_planes, n_seq, s_out]."""
+    if pos.dim() != 3 or seq_idx.dim() != 2 or pos.shape[1] != seq_idx.shape[0]:
+        raise ValueError("pos must be [n_planes, n_seq, seq_len] and seq_idx [n_seq, s_out]")
+    n_planes, n_seq, seq_len = pos.shape
+    s_out = seq_idx.shape[1]
+    if pos_out is None:
+        pos_out = torch.empty((n_planes, n_seq, s_out), dtype=torch.int32, device=_device_of(seq_idx, pos))
+    elif tuple(pos_out.shape) != (n_planes, n_seq, s_out):
+        raise ValueError("pos_out must be [n_planes, n_seq, s_out]")
+    args = (_dev_ptr(pos, "pos", torch.int32), n_planes, n_seq, seq_len,
+            _dev_ptr(seq_idx, "seq_idx", torch.int32), s_out, _dev_ptr(pos_out, "pos_out", torch.int32))
+    with torch.cuda.device(_device_of(seq_idx, pos)):
+        _check(load().civic_compact_pos_planes(*args, _stream_ptr(stream)), "civic_compact_pos_planes")
+    return pos_out

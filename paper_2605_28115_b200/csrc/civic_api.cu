@@ -70,33 +70,88 @@ int sm_count()
 }
 
 // Launch the row gather for up to kMaxGatherTensors tensors sharing one index array.
+template <int MODE>
 civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
 {
-    const long long total_rows = (long long)p.n_tensors * p.n_seq * p.s_out;
+    const long long total_rows = (long long)p.n_tensors * p.n_planes * p.s_out;
     const bool has_pos = p.pos_src != nullptr;
-    const long long pos_elems = has_pos ? (long long)p.n_seq * p.s_out * 3 : 0;
+    const long long pos_elems = has_pos ? (long long)p.n_planes * p.s_out * 3 : 0;
     if (total_rows == 0 && pos_elems == 0) return CIVIC_OK;
 
-    bool vec16 = p.row_bytes % 16 == 0;
+    bool vec16 = p.row_bytes % 16 == 0 && aligned(p.visual, 16);
     for (int i = 0; i < p.n_tensors && vec16; ++i)
         vec16 = aligned(p.src[i], 16) && aligned(p.dst[i], 16);
-    // one warp per segment of 32 * UNROLL vectors of a row
+    // one warp per tile of 32 * UNROLL vectors: a slice of a long row, or several short rows
     const int threads = civic::kGatherThreads, warps = threads / 32;
-    const long long seg_bytes = vec16 ? 32 * 4 * 16 : 32 * 8 * 4;
-    const long long segs_per_row = ((long long)p.row_bytes + seg_bytes - 1) / seg_bytes;
-    const long long main_blocks = (total_rows * segs_per_row + warps - 1) / warps;
+    const long long tile_vecs = vec16 ? 32 * 4 : 32 * 8;
+    const long long vecs = p.row_bytes / (vec16 ? 16 : 4);
+    const bool small = 2 * vecs <= tile_vecs;
+    const long long items = small ? (total_rows + tile_vecs / vecs - 1) / (tile_vecs / vecs)
+                                  : total_rows * ((vecs + tile_vecs - 1) / tile_vecs);
+    const long long main_blocks = (items + warps - 1) / warps;
     long long pos_blocks = (pos_elems + threads - 1) / threads;
     if (pos_blocks > sm_count()) pos_blocks = sm_count();
     if (main_blocks + pos_blocks > 0x7FFFFFFFLL) return CIVIC_ERR_UNSUPPORTED;
     p.main_blocks = (uint32_t)main_blocks;
     const unsigned grid = (unsigned)(main_blocks + pos_blocks);
+    const bool pdl = programmatic();
+    cudaError_t e;
     if (vec16)
-        CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::gather_rows_kernel<uint4, 4>, grid, threads, 0,
-                                     stream, p));
+        e = small ? civic::launch(pdl, civic::gather_rows_kernel<uint4, 4, MODE, true>, grid, threads, 0, stream, p)
+                  : civic::launch(pdl, civic::gather_rows_kernel<uint4, 4, MODE, false>, grid, threads, 0, stream, p);
     else
-        CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::gather_rows_kernel<uint32_t, 8>, grid, threads,
-                                     0, stream, p));
+        e = small ? civic::launch(pdl, civic::gather_rows_kernel<uint32_t, 8, MODE, true>, grid, threads, 0, stream, p)
+                  : civic::launch(pdl, civic::gather_rows_kernel<uint32_t, 8, MODE, false>, grid, threads, 0, stream, p);
+    CIVIC_CUDA_TRY(e);
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+// Validation shared by the three K/V calls: pointer tables, alignment, no destination
+// overlapping a source, another destination or the index array.
+civic_status_t check_kv_tables(const void* const* k_src, const void* const* v_src, void* const* k_dst,
+                               void* const* v_dst, int32_t n_layers, size_t src_bytes, size_t dst_bytes,
+                               const void* idx, size_t idx_bytes)
+{
+    if (!k_src || !v_src || !k_dst || !v_dst) return CIVIC_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!k_src[l] || !v_src[l] || !k_dst[l] || !v_dst[l]) return CIVIC_ERR_INVALID_ARG;
+        if (!aligned(k_src[l], 4) || !aligned(v_src[l], 4) || !aligned(k_dst[l], 4) ||
+            !aligned(v_dst[l], 4))
+            return CIVIC_ERR_ALIGNMENT;
+    }
+    for (int a = 0; a < 2 * n_layers; ++a) {
+        const void* da = (a & 1) ? v_dst[a >> 1] : k_dst[a >> 1];
+        if (overlaps(da, dst_bytes, idx, idx_bytes)) return CIVIC_ERR_INVALID_ARG;
+        for (int b = 0; b < 2 * n_layers; ++b) {
+            const void* sb = (b & 1) ? v_src[b >> 1] : k_src[b >> 1];
+            const void* db = (b & 1) ? v_dst[b >> 1] : k_dst[b >> 1];
+            if (overlaps(da, dst_bytes, sb, src_bytes)) return CIVIC_ERR_INVALID_ARG;
+            if (a != b && overlaps(da, dst_bytes, db, dst_bytes)) return CIVIC_ERR_INVALID_ARG;
+        }
+    }
+    return CIVIC_OK;
+}
+
+// Fills the pointer tables of `p` chunk by chunk and launches MODE once per chunk of layers.
+template <int MODE>
+civic_status_t launch_kv(civic::GatherParams base, const void* const* k_src, const void* const* v_src,
+                         void* const* k_dst, void* const* v_dst, int32_t n_layers, cudaStream_t stream)
+{
+    const int layers_per_launch = civic::kMaxGatherTensors / 2;
+    for (int l0 = 0; l0 < n_layers; l0 += layers_per_launch) {
+        const int nl = n_layers - l0 < layers_per_launch ? n_layers - l0 : layers_per_launch;
+        civic::GatherParams p = base;
+        for (int l = 0; l < nl; ++l) {
+            p.src[2 * l] = (const char*)k_src[l0 + l];
+            p.dst[2 * l] = (char*)k_dst[l0 + l];
+            p.src[2 * l + 1] = (const char*)v_src[l0 + l];
+            p.dst[2 * l + 1] = (char*)v_dst[l0 + l];
+        }
+        p.n_tensors = 2 * nl;
+        const civic_status_t st = launch_gather<MODE>(p, stream);
+        if (st != CIVIC_OK) return st;
+    }
     return CIVIC_OK;
 }
 
@@ -245,9 +300,10 @@ civic_status_t civic_compact(const void* hidden, size_t row_bytes, const int32_t
     p.idx = keep_idx;
     p.pos_src = pos_ids;
     p.pos_dst = pos_out;
-    p.n_seq = n_seg; p.seq_len = n; p.s_out = k;
+    p.n_planes = n_seg; p.seq_len = n; p.s_out = k;
+    p.idx_div = 1;
     p.row_bytes = hidden ? (uint32_t)row_bytes : 4;
-    return launch_gather(p, (cudaStream_t)stream);
+    return launch_gather<civic::kPlain>(p, (cudaStream_t)stream);
 }
 
 civic_status_t civic_seq_indices(const int32_t* keep_idx, int32_t n_seq, int32_t k, int32_t seq_len,
@@ -283,46 +339,140 @@ civic_status_t civic_compact_kv(const void* const* k_src, const void* const* v_s
     if (row_bytes == 0 || row_bytes > UINT32_MAX) return CIVIC_ERR_INVALID_ARG;
     if (row_bytes % 4) return CIVIC_ERR_ALIGNMENT;
     if (n_layers == 0 || n_seq == 0 || s_out == 0) return CIVIC_OK;
-    if (!k_src || !v_src || !k_dst || !v_dst || !seq_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!seq_idx) return CIVIC_ERR_INVALID_ARG;
     if (!aligned(seq_idx, 4)) return CIVIC_ERR_ALIGNMENT;
-    const size_t src_bytes = (size_t)n_seq * seq_len * row_bytes;
-    const size_t dst_bytes = (size_t)n_seq * s_out * row_bytes;
-    for (int l = 0; l < n_layers; ++l) {
-        if (!k_src[l] || !v_src[l] || !k_dst[l] || !v_dst[l]) return CIVIC_ERR_INVALID_ARG;
-        if (!aligned(k_src[l], 4) || !aligned(v_src[l], 4) || !aligned(k_dst[l], 4) ||
-            !aligned(v_dst[l], 4))
-            return CIVIC_ERR_ALIGNMENT;
-    }
-    // no destination may overlap a source, another destination or the index array
-    for (int a = 0; a < 2 * n_layers; ++a) {
-        const void* da = (a & 1) ? v_dst[a >> 1] : k_dst[a >> 1];
-        if (overlaps(da, dst_bytes, seq_idx, (size_t)n_seq * s_out * 4)) return CIVIC_ERR_INVALID_ARG;
-        for (int b = 0; b < 2 * n_layers; ++b) {
-            const void* sb = (b & 1) ? v_src[b >> 1] : k_src[b >> 1];
-            const void* db = (b & 1) ? v_dst[b >> 1] : k_dst[b >> 1];
-            if (overlaps(da, dst_bytes, sb, src_bytes)) return CIVIC_ERR_INVALID_ARG;
-            if (a != b && overlaps(da, dst_bytes, db, dst_bytes)) return CIVIC_ERR_INVALID_ARG;
-        }
-    }
+    const civic_status_t st =
+        check_kv_tables(k_src, v_src, k_dst, v_dst, n_layers, (size_t)n_seq * seq_len * row_bytes,
+                        (size_t)n_seq * s_out * row_bytes, seq_idx, (size_t)n_seq * s_out * 4);
+    if (st != CIVIC_OK) return st;
+    civic::GatherParams p;
+    memset(&p, 0, sizeof p);
+    p.idx = seq_idx;
+    p.n_planes = n_seq; p.seq_len = seq_len; p.s_out = s_out;
+    p.idx_div = 1;
+    p.row_bytes = (uint32_t)row_bytes;
+    return launch_kv<civic::kPlain>(p, k_src, v_src, k_dst, v_dst, n_layers, (cudaStream_t)stream);
+}
 
-    const int layers_per_launch = civic::kMaxGatherTensors / 2;
-    for (int l0 = 0; l0 < n_layers; l0 += layers_per_launch) {
-        const int nl = n_layers - l0 < layers_per_launch ? n_layers - l0 : layers_per_launch;
-        civic::GatherParams p;
-        memset(&p, 0, sizeof p);
-        for (int l = 0; l < nl; ++l) {
-            p.src[2 * l] = (const char*)k_src[l0 + l];
-            p.dst[2 * l] = (char*)k_dst[l0 + l];
-            p.src[2 * l + 1] = (const char*)v_src[l0 + l];
-            p.dst[2 * l + 1] = (char*)v_dst[l0 + l];
-        }
-        p.n_tensors = 2 * nl;
-        p.idx = seq_idx;
-        p.n_seq = n_seq; p.seq_len = seq_len; p.s_out = s_out;
-        p.row_bytes = (uint32_t)row_bytes;
-        civic_status_t st = launch_gather(p, (cudaStream_t)stream);
-        if (st != CIVIC_OK) return st;
-    }
+civic_status_t civic_compact_kv_heads(const void* const* k_src, const void* const* v_src,
+                                      void* const* k_dst, void* const* v_dst, int32_t n_layers,
+                                      int32_t n_seq, int32_t n_heads, int32_t seq_len, int32_t s_out,
+                                      size_t head_bytes, const int32_t* seq_idx, void* stream)
+{
+    if (n_layers < 0 || n_seq < 0 || n_heads < 0 || seq_len < 0 || s_out < 0) return CIVIC_ERR_INVALID_ARG;
+    if (s_out > seq_len) return CIVIC_ERR_K_RANGE;
+    if (head_bytes == 0 || head_bytes > UINT32_MAX) return CIVIC_ERR_INVALID_ARG;
+    if (head_bytes % 4) return CIVIC_ERR_ALIGNMENT;
+    if ((int64_t)n_seq * n_heads > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (n_layers == 0 || n_seq == 0 || n_heads == 0 || s_out == 0) return CIVIC_OK;
+    if (!seq_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(seq_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    const size_t planes = (size_t)n_seq * n_heads;
+    const civic_status_t st =
+        check_kv_tables(k_src, v_src, k_dst, v_dst, n_layers, planes * seq_len * head_bytes,
+                        planes * s_out * head_bytes, seq_idx, (size_t)n_seq * s_out * 4);
+    if (st != CIVIC_OK) return st;
+    civic::GatherParams p;
+    memset(&p, 0, sizeof p);
+    p.idx = seq_idx;
+    p.n_planes = (int32_t)planes; p.seq_len = seq_len; p.s_out = s_out;
+    p.idx_div = n_heads;
+    p.row_bytes = (uint32_t)head_bytes;
+    return launch_kv<civic::kHeads>(p, k_src, v_src, k_dst, v_dst, n_layers, (cudaStream_t)stream);
+}
+
+civic_status_t civic_compact_kv_paged(const void* const* k_src, const void* const* v_src,
+                                      void* const* k_cache, void* const* v_cache, int32_t n_layers,
+                                      int32_t n_seq, int32_t seq_len, int32_t s_out, size_t row_bytes,
+                                      const int32_t* seq_idx, const int32_t* block_table,
+                                      int32_t max_pages_per_seq, int32_t page_size, int32_t n_pages,
+                                      void* stream)
+{
+    if (n_layers < 0 || n_seq < 0 || seq_len < 0 || s_out < 0 || max_pages_per_seq < 0 ||
+        page_size < 1 || n_pages < 0)
+        return CIVIC_ERR_INVALID_ARG;
+    if (s_out > seq_len) return CIVIC_ERR_K_RANGE;
+    if ((int64_t)max_pages_per_seq * page_size < s_out) return CIVIC_ERR_INVALID_ARG;
+    if (row_bytes == 0 || row_bytes > UINT32_MAX) return CIVIC_ERR_INVALID_ARG;
+    if (row_bytes % 4) return CIVIC_ERR_ALIGNMENT;
+    if (n_layers == 0 || n_seq == 0 || s_out == 0) return CIVIC_OK;
+    if (!seq_idx || !block_table) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(seq_idx, 4) || !aligned(block_table, 4)) return CIVIC_ERR_ALIGNMENT;
+    const size_t cache_bytes = (size_t)n_pages * page_size * row_bytes;
+    civic_status_t st =
+        check_kv_tables(k_src, v_src, k_cache, v_cache, n_layers, (size_t)n_seq * seq_len * row_bytes,
+                        cache_bytes, seq_idx, (size_t)n_seq * s_out * 4);
+    if (st != CIVIC_OK) return st;
+    for (int l = 0; l < n_layers; ++l)
+        if (overlaps(k_cache[l], cache_bytes, block_table, (size_t)n_seq * max_pages_per_seq * 4) ||
+            overlaps(v_cache[l], cache_bytes, block_table, (size_t)n_seq * max_pages_per_seq * 4))
+            return CIVIC_ERR_INVALID_ARG;
+    civic::GatherParams p;
+    memset(&p, 0, sizeof p);
+    p.idx = seq_idx;
+    p.n_planes = n_seq; p.seq_len = seq_len; p.s_out = s_out;
+    p.idx_div = 1;
+    p.row_bytes = (uint32_t)row_bytes;
+    p.block_table = block_table;
+    p.max_pages = max_pages_per_seq;
+    p.page_size = page_size;
+    return launch_kv<civic::kPaged>(p, k_src, v_src, k_cache, v_cache, n_layers, (cudaStream_t)stream);
+}
+
+civic_status_t civic_merge_embeddings(const void* text, const void* visual, size_t row_bytes,
+                                      const int32_t* keep_idx, int32_t n_seq, int32_t seq_len,
+                                      int32_t vis_start, int32_t n_vis, int32_t k, void* merged,
+                                      void* stream)
+{
+    if (n_seq < 0 || seq_len < 0 || vis_start < 0 || n_vis < 0 || k < 0) return CIVIC_ERR_INVALID_ARG;
+    if ((int64_t)vis_start + n_vis > seq_len) return CIVIC_ERR_INVALID_ARG;
+    if (k > n_vis) return CIVIC_ERR_K_RANGE;
+    if (row_bytes == 0 || row_bytes > UINT32_MAX) return CIVIC_ERR_INVALID_ARG;
+    const int64_t s_out = (int64_t)seq_len - n_vis + k;
+    if (n_seq == 0 || s_out == 0) return CIVIC_OK;
+    if (!text || !merged || (k > 0 && (!visual || !keep_idx))) return CIVIC_ERR_INVALID_ARG;
+    if (row_bytes % 4 || !aligned(text, 4) || !aligned(visual, 4) || !aligned(merged, 4) ||
+        !aligned(keep_idx, 4))
+        return CIVIC_ERR_ALIGNMENT;
+    const size_t out_bytes = (size_t)n_seq * s_out * row_bytes;
+    if (overlaps(merged, out_bytes, text, (size_t)n_seq * seq_len * row_bytes) ||
+        overlaps(merged, out_bytes, visual, (size_t)n_seq * n_vis * row_bytes) ||
+        overlaps(merged, out_bytes, keep_idx, (size_t)n_seq * k * 4))
+        return CIVIC_ERR_INVALID_ARG;
+    civic::GatherParams p;
+    memset(&p, 0, sizeof p);
+    p.n_tensors = 1;
+    p.src[0] = (const char*)text;
+    p.dst[0] = (char*)merged;
+    p.idx = keep_idx;
+    p.n_planes = n_seq; p.seq_len = seq_len; p.s_out = (int32_t)s_out;
+    p.idx_div = 1;
+    p.row_bytes = (uint32_t)row_bytes;
+    p.visual = (const char*)visual;
+    p.vis_start = vis_start; p.n_vis = n_vis; p.k_vis = k;
+    return launch_gather<civic::kMerge>(p, (cudaStream_t)stream);
+}
+
+civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, int32_t n_seq,
+                                        int32_t seq_len, const int32_t* seq_idx, int32_t s_out,
+                                        int32_t* pos_out, void* stream)
+{
+    if (n_planes < 0 || n_seq < 0 || seq_len < 0 || s_out < 0) return CIVIC_ERR_INVALID_ARG;
+    if (s_out > seq_len) return CIVIC_ERR_K_RANGE;
+    const long long total = (long long)n_planes * n_seq * s_out;
+    if (total == 0) return CIVIC_OK;
+    if (!pos || !seq_idx || !pos_out) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(pos, 4) || !aligned(seq_idx, 4) || !aligned(pos_out, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (overlaps(pos_out, (size_t)total * 4, pos, (size_t)n_planes * n_seq * seq_len * 4) ||
+        overlaps(pos_out, (size_t)total * 4, seq_idx, (size_t)n_seq * s_out * 4))
+        return CIVIC_ERR_INVALID_ARG;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    if (blocks > 8LL * sm_count()) blocks = 8LL * sm_count();
+    CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::gather_pos_planes_kernel, (unsigned)blocks, threads, 0,
+                                 (cudaStream_t)stream, pos, seq_idx, pos_out, n_planes, n_seq, seq_len,
+                                 s_out));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     return CIVIC_OK;
 }
 

@@ -1,6 +1,17 @@
-// Order-preserving row gather: dst[t][s, j, :] = src[t][s, idx[s, j], :] for a table of
+// Order-preserving row gather: dst[t][q, j, :] = src[t][q, idx[q, j], :] for a table of
 // tensors that share one index array (all layers' K and V, or the hidden states).
 // Pure data movement, HBM-bound: rows are opaque bytes.
+//
+// One kernel template covers the layouts of the library:
+//   kPlain  token-major rows, contiguous destination                (civic_compact, civic_compact_kv)
+//   kHeads  head-major tensors [n_seq, n_heads, seq_len, head_bytes]: a "plane" q is one
+//           (sequence, head) pair and uses index row q / idx_div    (civic_compact_kv_heads)
+//   kPaged  token-major source, destination rows placed through a block table
+//                                                                   (civic_compact_kv_paged)
+//   kMerge  two sources: text rows outside the visual span, kept visual rows inside it
+//                                                                   (civic_merge_embeddings)
+// and two work decompositions: rows of at least one warp tile are cut into tiles (LARGE), shorter
+// rows are packed several to a tile (SMALL) so that every lane still moves full 16-byte vectors.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -12,16 +23,25 @@ namespace civic {
 constexpr int kMaxGatherTensors = 160;  // K and V of 80 layers per launch
 constexpr int kGatherThreads = 256;
 
+enum GatherMode { kPlain = 0, kHeads = 1, kPaged = 2, kMerge = 3 };
+
 struct GatherParams {
-    const char* src[kMaxGatherTensors];  // each [n_seq, seq_len, row_bytes]
-    char* dst[kMaxGatherTensors];        // each [n_seq, s_out, row_bytes]
-    const int32_t* idx;                  // [n_seq, s_out]
+    const char* src[kMaxGatherTensors];  // each [n_planes, seq_len, row_bytes]
+    char* dst[kMaxGatherTensors];        // each [n_planes, s_out, row_bytes] (kPaged: the cache)
+    const int32_t* idx;                  // [n_planes / idx_div, s_out]; kMerge: keep_idx [n_planes, k_vis]
     // optional 3 x int32 rows gathered by the same index (position ids); NULL = none
-    const int32_t* pos_src;              // [n_seq, seq_len, 3]
-    int32_t* pos_dst;                    // [n_seq, s_out, 3]
-    int32_t n_tensors, n_seq, seq_len, s_out;
+    const int32_t* pos_src;              // [n_planes, seq_len, 3]
+    int32_t* pos_dst;                    // [n_planes, s_out, 3]
+    int32_t n_tensors, n_planes, seq_len, s_out;
     uint32_t row_bytes;
     uint32_t main_blocks;  // blocks [0, main_blocks) move rows, the rest move pos ids
+    int32_t idx_div;       // kHeads: planes (heads) per index row
+    // kPaged: row j of plane q lives in page block_table[q, j / page_size], slot j % page_size
+    const int32_t* block_table;  // [n_planes, max_pages]
+    int32_t max_pages, page_size;
+    // kMerge: src[0] is the text [n_planes, seq_len, row], visual the dense visual rows
+    const char* visual;  // [n_planes, n_vis, row]
+    int32_t vis_start, n_vis, k_vis;
 };
 
 template <typename VecT>
@@ -46,7 +66,7 @@ __device__ __forceinline__ void store_stream(uint32_t* p, uint32_t v) { __stcs(p
 
 __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int n_blocks)
 {
-    const long long total = (long long)p.n_seq * p.s_out * 3;
+    const long long total = (long long)p.n_planes * p.s_out * 3;
     for (long long e = (long long)block * blockDim.x + threadIdx.x; e < total;
          e += (long long)n_blocks * blockDim.x) {
         const long long row = e / 3;
@@ -57,12 +77,41 @@ __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int
     }
 }
 
-// One warp per row segment, no grid-stride loop.  A segment is up to 32 * UNROLL vectors
-// (2 KB for 16-byte vectors) of one destination row; segments are numbered row-major, so
-// the hardware block scheduler sweeps source and destination in address order, which
-// measured faster on B200 than a persistent grid-stride loop.  Every lane has its UNROLL
-// loads in flight before its first store.
-template <typename VecT, int UNROLL>
+// Source row of output row j of plane q.
+template <int MODE>
+__device__ __forceinline__ const char* source_row(const GatherParams& p, int tensor, int q, int j)
+{
+    if constexpr (MODE == kMerge) {
+        if (j < p.vis_start) return p.src[0] + ((size_t)q * p.seq_len + j) * p.row_bytes;
+        if (j < p.vis_start + p.k_vis) {
+            const int32_t i = __ldg(p.idx + (size_t)q * p.k_vis + (j - p.vis_start));
+            return p.visual + ((size_t)q * p.n_vis + i) * p.row_bytes;
+        }
+        return p.src[0] + ((size_t)q * p.seq_len + (j - p.k_vis + p.n_vis)) * p.row_bytes;
+    } else {
+        const int idx_row = MODE == kHeads ? q / p.idx_div : q;
+        const int32_t i = __ldg(p.idx + (size_t)idx_row * p.s_out + j);
+        return p.src[tensor] + ((size_t)q * p.seq_len + i) * p.row_bytes;
+    }
+}
+
+template <int MODE>
+__device__ __forceinline__ char* destination_row(const GatherParams& p, int tensor, int q, int j)
+{
+    if constexpr (MODE == kPaged) {
+        const int32_t page = __ldg(p.block_table + (size_t)q * p.max_pages + j / p.page_size);
+        return p.dst[tensor] + ((size_t)page * p.page_size + j % p.page_size) * p.row_bytes;
+    } else {
+        return p.dst[tensor] + ((size_t)q * p.s_out + j) * p.row_bytes;
+    }
+}
+
+// One warp per tile of 32 * UNROLL vectors (2 KB for 16-byte vectors), no grid-stride loop.
+// Tiles are numbered row-major over [tensor][plane][row], so the hardware block scheduler sweeps
+// source and destination in address order, which measured faster on B200 than a persistent
+// grid-stride loop.  Every lane has its UNROLL loads in flight before its first store.
+// LARGE: a row is ceil(vecs / tile) tiles.  SMALL: a tile is floor(tile / vecs) whole rows.
+template <typename VecT, int UNROLL, int MODE, bool SMALL>
 __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __grid_constant__ GatherParams p)
 {
     wait_for_prior_kernels();
@@ -70,32 +119,74 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __gri
         gather_pos(p, blockIdx.x - p.main_blocks, gridDim.x - p.main_blocks);
         return;
     }
-    constexpr int kSegVecs = 32 * UNROLL;
+    constexpr int kTileVecs = 32 * UNROLL;
     const int lane = threadIdx.x & 31;
     const int vecs = p.row_bytes / sizeof(VecT);
-    const int segs_per_row = (vecs + kSegVecs - 1) / kSegVecs;
-    const long long rows_per_tensor = (long long)p.n_seq * p.s_out;
-    const long long total_segs = rows_per_tensor * p.n_tensors * segs_per_row;
+    const long long rows_per_tensor = (long long)p.n_planes * p.s_out;
+    const long long total_rows = rows_per_tensor * p.n_tensors;
     const long long item = (long long)blockIdx.x * (kGatherThreads / 32) + (threadIdx.x >> 5);
-    if (item >= total_segs) return;
 
-    const long long row = item / segs_per_row;
-    const int seg = (int)(item - row * segs_per_row);
-    const int tensor = (int)(row / rows_per_tensor);
-    const long long rem = row - (long long)tensor * rows_per_tensor;  // s * s_out + j
-    const int s = (int)(rem / p.s_out);
-    const int32_t i = __ldg(p.idx + rem);
-    const VecT* src = reinterpret_cast<const VecT*>(p.src[tensor] + ((size_t)s * p.seq_len + i) * p.row_bytes);
-    VecT* dst = reinterpret_cast<VecT*>(p.dst[tensor] + (size_t)rem * p.row_bytes);
+    if constexpr (!SMALL) {
+        const int tiles_per_row = (vecs + kTileVecs - 1) / kTileVecs;
+        if (item >= total_rows * tiles_per_row) return;
+        const long long row = item / tiles_per_row;
+        const int tile = (int)(item - row * tiles_per_row);
+        const int tensor = (int)(row / rows_per_tensor);
+        const long long rem = row - (long long)tensor * rows_per_tensor;  // q * s_out + j
+        const int q = (int)(rem / p.s_out);
+        const int j = (int)(rem - (long long)q * p.s_out);
+        const VecT* src = reinterpret_cast<const VecT*>(source_row<MODE>(p, tensor, q, j));
+        VecT* dst = reinterpret_cast<VecT*>(destination_row<MODE>(p, tensor, q, j));
+        const int v0 = tile * kTileVecs + lane;
+        VecT buf[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (v0 + 32 * u < vecs) buf[u] = load_stream(src + v0 + 32 * u);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (v0 + 32 * u < vecs) store_stream(dst + v0 + 32 * u, buf[u]);
+    } else {
+        const int rows_per_tile = kTileVecs / vecs;  // >= 2 by the host's choice
+        const long long row0 = item * rows_per_tile;
+        if (row0 >= total_rows) return;
+        VecT buf[UNROLL];
+        VecT* dst[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int v = lane + 32 * u;
+            const int r = v / vecs, c = v - r * vecs;
+            const long long row = row0 + r;
+            dst[u] = nullptr;
+            if (r < rows_per_tile && row < total_rows) {
+                const int tensor = (int)(row / rows_per_tensor);
+                const long long rem = row - (long long)tensor * rows_per_tensor;
+                const int q = (int)(rem / p.s_out);
+                const int j = (int)(rem - (long long)q * p.s_out);
+                buf[u] = load_stream(reinterpret_cast<const VecT*>(source_row<MODE>(p, tensor, q, j)) + c);
+                dst[u] = reinterpret_cast<VecT*>(destination_row<MODE>(p, tensor, q, j)) + c;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (dst[u]) store_stream(dst[u], buf[u]);
+    }
+}
 
-    const int v0 = seg * kSegVecs + lane;
-    VecT buf[UNROLL];
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u)
-        if (v0 + 32 * u < vecs) buf[u] = load_stream(src + v0 + 32 * u);
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u)
-        if (v0 + 32 * u < vecs) store_stream(dst + v0 + 32 * u, buf[u]);
+// out[c, s, j] = pos[c, s, idx[s, j]] for plane-major position ids.
+__global__ void gather_pos_planes_kernel(const int32_t* __restrict__ pos, const int32_t* __restrict__ idx,
+                                         int32_t* __restrict__ out, int n_planes, int n_seq, int seq_len,
+                                         int s_out)
+{
+    release_next_kernel();
+    wait_for_prior_kernels();
+    const long long per_plane = (long long)n_seq * s_out, total = per_plane * n_planes;
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(e / per_plane);
+        const long long rem = e - (long long)c * per_plane;  // s * s_out + j
+        const int s = (int)(rem / s_out);
+        out[e] = pos[((size_t)c * n_seq + s) * seq_len + idx[rem]];
+    }
 }
 
 }  // namespace civic

@@ -142,6 +142,40 @@ def test_compact_kv_validation(lib):
     assert f(ks, vs, kd, vd, -1, 2, 16, 8, 64, 0x10, None) == 1
 
 
+def test_adjacent_calls_validation(lib):
+    P = ctypes.c_void_p * 2
+    ks, vs = P(0x100000, 0x200000), P(0x300000, 0x400000)
+    kd, vd = P(0x500000, 0x600000), P(0x700000, 0x800000)
+    before = lib.civic_launch_count()
+    h = lib.civic_compact_kv_heads
+    assert h(ks, vs, kd, vd, 2, 2, 4, 16, 17, 64, 0x10, None) == 2  # s_out > seq_len
+    assert h(ks, vs, kd, vd, 2, 2, 4, 16, 8, 6, 0x10, None) == 4
+    assert h(ks, vs, kd, vd, 2, 2, -1, 16, 8, 64, 0x10, None) == 1
+    assert h(ks, vs, ks, vd, 2, 2, 4, 16, 8, 64, 0x10, None) == 1  # destination is a source
+    assert h(ks, vs, kd, vd, 2, 2, 4, 16, 8, 64, None, None) == 1
+    assert h(ks, vs, kd, vd, 2, 2, 0, 16, 8, 64, 0x10, None) == 0
+    g = lib.civic_compact_kv_paged
+    assert g(ks, vs, kd, vd, 2, 2, 16, 8, 64, 0x10, 0x40, 1, 4, 100, None) == 1  # 1 page of 4 < 8 rows
+    assert g(ks, vs, kd, vd, 2, 2, 16, 8, 64, 0x10, 0x40, 2, 0, 100, None) == 1  # page size 0
+    assert g(ks, vs, kd, vd, 2, 2, 16, 8, 64, 0x10, None, 2, 4, 100, None) == 1  # no block table
+    assert g(ks, vs, kd, vd, 2, 2, 16, 17, 64, 0x10, 0x40, 8, 4, 100, None) == 2
+    assert g(ks, vs, kd, vd, 2, 2, 16, 8, 64, 0x10, 0x42, 2, 4, 100, None) == 4
+    assert g(ks, vs, kd, vd, 2, 0, 16, 8, 64, 0x10, 0x40, 2, 4, 100, None) == 0
+    m = lib.civic_merge_embeddings
+    assert m(0x10000, 0x20000, 64, 0x100, 1, 20, 3, 12, 13, 0x30000, None) == 2  # k > n_vis
+    assert m(0x10000, 0x20000, 64, 0x100, 1, 20, 10, 12, 5, 0x30000, None) == 1  # span past the end
+    assert m(0x10000, 0x20000, 6, 0x100, 1, 20, 3, 12, 5, 0x30000, None) == 4
+    assert m(0x10000, 0x20000, 64, 0x100, 1, 20, 3, 12, 5, 0x10100, None) == 1  # output overlaps text
+    assert m(0x10000, None, 64, 0x100, 1, 20, 3, 12, 5, 0x30000, None) == 1
+    assert m(0x10000, 0x20000, 64, 0x100, 0, 20, 3, 12, 5, 0x30000, None) == 0
+    q = lib.civic_compact_pos_planes
+    assert q(0x10000, 3, 2, 20, 0x100, 21, 0x30000, None) == 2
+    assert q(0x10000, 3, 2, 20, 0x100, 5, None, None) == 1
+    assert q(0x10000, 3, 2, 20, 0x100, 5, 0x10010, None) == 1  # overlap
+    assert q(0x10000, 0, 2, 20, 0x100, 5, 0x30000, None) == 0
+    assert lib.civic_launch_count() == before
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
 
