@@ -85,7 +85,7 @@ civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
     const int threads = civic::kGatherThreads, warps = threads / 32;
     const long long tile_vecs = vec16 ? 32 * 4 : 32 * 8;
     const long long vecs = p.row_bytes / (vec16 ? 16 : 4);
-    const bool small = 2 * vecs <= tile_vecs;
+    const bool small = 2 * vecs <= tile_vecs && total_rows < 0x7FFFFFFFLL;
     const long long items = small ? (total_rows + tile_vecs / vecs - 1) / (tile_vecs / vecs)
                                   : total_rows * ((vecs + tile_vecs - 1) / tile_vecs);
     const long long main_blocks = (items + warps - 1) / warps;

@@ -77,9 +77,9 @@ __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int
     }
 }
 
-// Source row of output row j of plane q.
+// Source row of output row j of plane q; idx_row is the plane's row of the index array.
 template <int MODE>
-__device__ __forceinline__ const char* source_row(const GatherParams& p, int tensor, int q, int j)
+__device__ __forceinline__ const char* source_row(const GatherParams& p, int tensor, int q, int idx_row, int j)
 {
     if constexpr (MODE == kMerge) {
         if (j < p.vis_start) return p.src[0] + ((size_t)q * p.seq_len + j) * p.row_bytes;
@@ -89,7 +89,6 @@ __device__ __forceinline__ const char* source_row(const GatherParams& p, int ten
         }
         return p.src[0] + ((size_t)q * p.seq_len + (j - p.k_vis + p.n_vis)) * p.row_bytes;
     } else {
-        const int idx_row = MODE == kHeads ? q / p.idx_div : q;
         const int32_t i = __ldg(p.idx + (size_t)idx_row * p.s_out + j);
         return p.src[tensor] + ((size_t)q * p.seq_len + i) * p.row_bytes;
     }
@@ -135,7 +134,8 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __gri
         const long long rem = row - (long long)tensor * rows_per_tensor;  // q * s_out + j
         const int q = (int)(rem / p.s_out);
         const int j = (int)(rem - (long long)q * p.s_out);
-        const VecT* src = reinterpret_cast<const VecT*>(source_row<MODE>(p, tensor, q, j));
+        const int idx_row = MODE == kHeads ? q / p.idx_div : q;
+        const VecT* src = reinterpret_cast<const VecT*>(source_row<MODE>(p, tensor, q, idx_row, j));
         VecT* dst = reinterpret_cast<VecT*>(destination_row<MODE>(p, tensor, q, j));
         const int v0 = tile * kTileVecs + lane;
         VecT buf[UNROLL];
@@ -146,25 +146,41 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __gri
         for (int u = 0; u < UNROLL; ++u)
             if (v0 + 32 * u < vecs) store_stream(dst + v0 + 32 * u, buf[u]);
     } else {
-        const int rows_per_tile = kTileVecs / vecs;  // >= 2 by the host's choice
-        const long long row0 = item * rows_per_tile;
-        if (row0 >= total_rows) return;
+        // The host takes this path only when all rows of the launch number below 2^31, so the
+        // tile's first row is decomposed with 32-bit divisions, once; the lanes then step from
+        // it by additions (a tile rarely crosses a plane, almost never a tensor).
+        const uint32_t uvecs = (uint32_t)vecs;
+        const uint32_t rows_per_tile = kTileVecs / uvecs;  // >= 2 by the host's choice
+        const uint32_t row0 = (uint32_t)item * rows_per_tile;
+        if (row0 >= (uint32_t)total_rows) return;
+        const uint32_t s_out = (uint32_t)p.s_out, n_planes = (uint32_t)p.n_planes;
+        const uint32_t tensor0 = row0 / (uint32_t)rows_per_tensor;
+        const uint32_t rem0 = row0 - tensor0 * (uint32_t)rows_per_tensor;
+        const uint32_t q0 = rem0 / s_out, j0 = rem0 - q0 * s_out;
+        const uint32_t heads = MODE == kHeads ? (uint32_t)p.idx_div : 1u;
+        const uint32_t s0 = q0 / heads, h0 = q0 - s0 * heads;
+        const uint32_t step_r = 32u / uvecs, step_c = 32u - step_r * uvecs;
+        uint32_t r = (uint32_t)lane / uvecs, c = (uint32_t)lane - r * uvecs;
         VecT buf[UNROLL];
         VecT* dst[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const int v = lane + 32 * u;
-            const int r = v / vecs, c = v - r * vecs;
-            const long long row = row0 + r;
             dst[u] = nullptr;
-            if (r < rows_per_tile && row < total_rows) {
-                const int tensor = (int)(row / rows_per_tensor);
-                const long long rem = row - (long long)tensor * rows_per_tensor;
-                const int q = (int)(rem / p.s_out);
-                const int j = (int)(rem - (long long)q * p.s_out);
-                buf[u] = load_stream(reinterpret_cast<const VecT*>(source_row<MODE>(p, tensor, q, j)) + c);
-                dst[u] = reinterpret_cast<VecT*>(destination_row<MODE>(p, tensor, q, j)) + c;
+            uint32_t tensor = tensor0, q = q0, idx_row = s0, h = h0, j = j0 + r;
+            while (j >= s_out) {  // next plane; next index row after the last head; next tensor
+                j -= s_out;
+                ++q;
+                if (++h == heads) { h = 0; ++idx_row; }
+                if (q == n_planes) { q = 0; idx_row = 0; ++tensor; }
             }
+            if (r < rows_per_tile && tensor < (uint32_t)p.n_tensors) {
+                buf[u] = load_stream(reinterpret_cast<const VecT*>(
+                                         source_row<MODE>(p, (int)tensor, (int)q, (int)idx_row, (int)j)) + c);
+                dst[u] = reinterpret_cast<VecT*>(destination_row<MODE>(p, (int)tensor, (int)q, (int)j)) + c;
+            }
+            r += step_r;
+            c += step_c;
+            if (c >= uvecs) { c -= uvecs; ++r; }
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u)
