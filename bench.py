@@ -53,13 +53,19 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv-layout", default="token_major", choices=["token_major", "head_major", "paged"],
+                    help="K/V cache layout: [seq, token, heads*dim] rows (default), [seq, head, token, dim] "
+                         "pieces, or token-major sources into a paged cache of 16-token pages")
+    ap.add_argument("--merge", action="store_true",
+                    help="also build the compact prefill sequence (Eq. 13 merge of text and kept visual "
+                         "rows) and its plane-major position ids in every step")
     ap.add_argument("--layers", type=int, default=0,
                     help="shrink the workload to this many K/V layers (profiling a small case); "
                          "the JSON line then names the reduced workload")
     return ap.parse_args()
 
 
-def step_bytes(wl):
+def step_bytes(wl, merge=False):
     """Algorithmic bytes of one step, by part."""
     from paper_2605_28115_b200 import workloads as W
 
@@ -68,8 +74,12 @@ def step_bytes(wl):
     pos = 2 * wl.n_seg * wl.k * 12
     select = wl.n_seg * wl.n * 4 + wl.n_seg * wl.k * 4
     seq = (wl.n_seg * wl.k * 4 + wl.n_seg * wl.s_out * 4) if wl.n_layers else 0
-    return {"kv": kv, "hidden": hidden, "pos": pos, "select": select, "seq_idx": seq,
-            "total": kv + hidden + pos + select + seq}
+    out = {"kv": kv, "hidden": hidden, "pos": pos, "select": select, "seq_idx": seq}
+    if merge:  # every row of the compact sequence read once and written once; 3 planes of pos ids
+        out["merge"] = 2 * wl.n_seg * wl.s_out * wl.hidden_row_bytes
+        out["pos_planes"] = 2 * 3 * wl.n_seg * wl.s_out * 4
+    out["total"] = sum(out.values())
+    return out
 
 
 def pick_workload(args):
@@ -171,13 +181,16 @@ class ClockSampler:
 class DeviceState:
     """Inputs and outputs of one rank, resident on its GPU."""
 
-    def __init__(self, wl, dev, rank):
+    PAGE = 16
+
+    def __init__(self, wl, dev, rank, kv_layout="token_major", merge=False):
         import torch
 
         from paper_2605_28115_b200 import civic
         from paper_2605_28115_b200 import workloads as W
 
         self.wl, self.dev = wl, dev
+        self.kv_layout, self.merge = kv_layout, merge and bool(wl.hidden_dim) and bool(wl.n_layers)
         wl_r = wl.replace(config_id=wl.config_id + 100 * rank) if rank else wl  # per-rank seeds
         self.scores_host = W.scores(wl_r)
         self.pos_host = W.pos_ids(wl)
@@ -192,11 +205,43 @@ class DeviceState:
         self.seq_idx = torch.empty((wl.n_seg, wl.s_out), dtype=torch.int32, device=dev)
         self.k_src = [W.kv_layer(wl_r, l, 0, dev) for l in range(wl.n_layers)]
         self.v_src = [W.kv_layer(wl_r, l, 1, dev) for l in range(wl.n_layers)]
-        shape = (wl.n_seg, wl.s_out, wl.kv_heads, wl.head_dim)
+        self.block_table = None
+        if kv_layout == "head_major":  # the same seeded payload read as [seq, head, token, dim]
+            self.k_src = [x.view(wl.n_seg, wl.kv_heads, wl.seq_len, wl.head_dim) for x in self.k_src]
+            self.v_src = [x.view(wl.n_seg, wl.kv_heads, wl.seq_len, wl.head_dim) for x in self.v_src]
+            shape = (wl.n_seg, wl.kv_heads, wl.s_out, wl.head_dim)
+        elif kv_layout == "paged":  # every sequence owns ceil(s_out / PAGE) pages of a shuffled pool
+            per_seq = -(-wl.s_out // self.PAGE)
+            g = torch.Generator(device="cpu")
+            g.manual_seed(wl.seed + 900 + rank)
+            self.block_table = torch.randperm(wl.n_seg * per_seq, generator=g).to(torch.int32) \
+                .view(wl.n_seg, per_seq).contiguous().to(dev)
+            shape = (wl.n_seg * per_seq, self.PAGE, wl.kv_heads, wl.head_dim)
+        else:
+            shape = (wl.n_seg, wl.s_out, wl.kv_heads, wl.head_dim)
         self.k_dst = [torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(wl.n_layers)]
         self.v_dst = [torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(wl.n_layers)]
-        self.tables = (civic.kv_tables(self.k_src, self.v_src, self.k_dst, self.v_dst)
-                       if wl.n_layers else None)
+        make = {"token_major": civic.kv_tables, "head_major": civic.kv_heads_tables,
+                "paged": civic.kv_paged_tables}[kv_layout]
+        self.tables = make(self.k_src, self.v_src, self.k_dst, self.v_dst) if wl.n_layers else None
+        if self.merge:
+            self.text = W.payload_bf16((wl.n_seg, wl.seq_len, wl.hidden_dim), wl_r.seed + 700, dev)
+            self.merged = torch.empty((wl.n_seg, wl.s_out, wl.hidden_dim), dtype=torch.bfloat16, device=dev)
+            planes = torch.arange(wl.seq_len, dtype=torch.int32).repeat(3, wl.n_seg, 1)
+            vis = torch.from_numpy(self.pos_host).permute(2, 0, 1) + wl.text_before  # (t,h,w) planes
+            planes[:, :, wl.text_before:wl.text_before + wl.n] = vis
+            self.pos_planes = planes.contiguous().to(dev)
+            self.pos_planes_out = torch.empty((3, wl.n_seg, wl.s_out), dtype=torch.int32, device=dev)
+
+    def compact_kv(self):
+        from paper_2605_28115_b200 import civic
+
+        if self.kv_layout == "head_major":
+            civic.civic_compact_kv_heads(self.tables, self.seq_idx)
+        elif self.kv_layout == "paged":
+            civic.civic_compact_kv_paged(self.tables, self.seq_idx, self.block_table)
+        else:
+            civic.civic_compact_kv(self.tables, self.seq_idx)
 
     def step(self, kv_events=None):
         """One pass of the whole path on the current stream (asynchronous)."""
@@ -209,10 +254,13 @@ class DeviceState:
         else:
             civic.civic_select(self.scores, self.desc, keep_idx=self.keep)
         civic.civic_compact(self.hidden, self.pos, self.keep, hidden_out=self.hidden_out, pos_out=self.pos_out)
+        if self.merge:
+            civic.civic_merge_embeddings(self.text, self.hidden, self.keep, wl.text_before, merged=self.merged)
+            civic.civic_compact_pos_planes(self.pos_planes, self.seq_idx, pos_out=self.pos_planes_out)
         if self.tables is not None:
             if kv_events is not None:
                 kv_events[0].record()
-            civic.civic_compact_kv(self.tables, self.seq_idx)
+            self.compact_kv()
             if kv_events is not None:
                 kv_events[1].record()
 
@@ -363,8 +411,9 @@ def run_civic(args):
     civic.load()
 
     wl = pick_workload(args)
-    st = DeviceState(wl, dev, rank)
-    nbytes = step_bytes(wl)
+    st = DeviceState(wl, dev, rank, args.kv_layout, args.merge)
+    nbytes = step_bytes(wl, st.merge)
+    default_variant = args.kv_layout == "token_major" and not st.merge
 
     def barrier():
         if world > 1:
@@ -403,15 +452,17 @@ def run_civic(args):
         kv_avg = sum(kv_ms) / len(kv_ms)
         peak, which = measured_peak()
         achieved = nbytes["kv"] / (kv_avg * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "civic_compact_kv", "achieved": achieved, "peak": peak,
+        kernel = {"token_major": "civic_compact_kv", "head_major": "civic_compact_kv_heads",
+                  "paged": "civic_compact_kv_paged"}[args.kv_layout]
+        roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                     "unit": "GB/s", "frac": achieved / peak, "peak_source": which,
-                    "traffic": NCU_DRAM_TRAFFIC_PER_LAUNCH.get(wl.name),
+                    "traffic": NCU_DRAM_TRAFFIC_PER_LAUNCH.get(wl.name) if default_variant else None,
                     "algorithmic_bytes_per_launch": nbytes["kv"], "us_per_launch": kv_avg * 1e3,
                     "us_per_launch_min": min(kv_ms) * 1e3, "launches_timed": len(kv_ms), "frac_of_8TBps_nominal": achieved / 8000.0}
 
     # end to end: pinned host inputs -> path -> pinned host results, every step
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and default_variant:
         n_e2e = max(1, args.e2e_steps)
         modes = {}
         for mode in ("zero_copy", "staged"):
@@ -446,14 +497,18 @@ def run_civic(args):
                "results_match_device_path": modes[best]["results_match_device_path"]}
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and default_variant:
         cpu = cpu_baseline(st)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-                "config": config_of(wl, {"parallelism": f"dp{world}" if world > 1 else "single"}),
+                "config": config_of(wl, {"parallelism": f"dp{world}" if world > 1 else "single",
+                                         "kv_layout": args.kv_layout, "merge": st.merge,
+                                         **({} if default_variant else {"workload": wl.name + (
+                                             "" if args.kv_layout == "token_major" else "+" + args.kv_layout)
+                                             + ("+merge" if st.merge else "")})}),
                 "bytes_per_step": nbytes, "gpu_launches": launches, "clocks": clocks,
                 "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
         print(json.dumps(line), flush=True)

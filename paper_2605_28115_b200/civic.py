@@ -307,10 +307,22 @@ def _same(ts: Sequence[torch.Tensor], what: str):
     return shape, dtype
 
 
-def civic_compact_kv_heads(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
-                           k_dst: Sequence[torch.Tensor], v_dst: Sequence[torch.Tensor],
-                           seq_idx: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
-    """Head-major caches: [n_seq, n_heads, seq_len, d] -> [n_seq, n_heads, s_out, d] per layer."""
+@dataclasses.dataclass
+class KVHeadsTables:
+    """Host pointer tables for civic_compact_kv_heads, built once per set of cache tensors."""
+    tables: tuple
+    n_layers: int
+    n_seq: int
+    n_heads: int
+    seq_len: int
+    s_out: int
+    head_bytes: int
+    keepalive: tuple
+
+
+def kv_heads_tables(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
+                    k_dst: Sequence[torch.Tensor], v_dst: Sequence[torch.Tensor]) -> KVHeadsTables:
+    """Marshal head-major per-layer tensors ([n_seq, n_heads, seq_len, d] -> [n_seq, n_heads, s_out, d])."""
     n_layers = len(k_src)
     if n_layers == 0 or not (len(v_src) == len(k_dst) == len(v_dst) == n_layers):
         raise ValueError("the four tensor lists must have one entry per layer")
@@ -320,23 +332,41 @@ def civic_compact_kv_heads(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.
             src_shape[:2] != dst_shape[:2] or src_shape[3] != dst_shape[3]:
         raise ValueError("source [n_seq, n_heads, seq_len, d] and destination [n_seq, n_heads, s_out, d] disagree")
     n_seq, n_heads, seq_len, d = src_shape
-    s_out = dst_shape[2]
-    if tuple(seq_idx.shape) != (n_seq, s_out):
+    return KVHeadsTables((_table(k_src, "k_src"), _table(v_src, "v_src"), _table(k_dst, "k_dst"),
+                          _table(v_dst, "v_dst")), n_layers, n_seq, n_heads, seq_len, dst_shape[2],
+                         d * k_src[0].element_size(),
+                         (tuple(k_src), tuple(v_src), tuple(k_dst), tuple(v_dst)))
+
+
+def civic_compact_kv_heads(tables: KVHeadsTables, seq_idx: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Head-major caches: k_dst[l][s, h, j] = k_src[l][s, h, seq_idx[s, j]] (and V), every layer."""
+    t = tables
+    if tuple(seq_idx.shape) != (t.n_seq, t.s_out):
         raise ValueError("seq_idx must be [n_seq, s_out]")
     idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
-    with torch.cuda.device(_device_of(seq_idx, k_src[0], k_dst[0])):
-        _check(load().civic_compact_kv_heads(_table(k_src, "k_src"), _table(v_src, "v_src"),
-                                             _table(k_dst, "k_dst"), _table(v_dst, "v_dst"), n_layers,
-                                             n_seq, n_heads, seq_len, s_out, d * k_src[0].element_size(),
-                                             idx_ptr, _stream_ptr(stream)), "civic_compact_kv_heads")
+    with torch.cuda.device(_device_of(seq_idx, t.keepalive[0][0], t.keepalive[2][0])):
+        _check(load().civic_compact_kv_heads(*t.tables, t.n_layers, t.n_seq, t.n_heads, t.seq_len, t.s_out,
+                                             t.head_bytes, idx_ptr, _stream_ptr(stream)),
+               "civic_compact_kv_heads")
 
 
-def civic_compact_kv_paged(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
-                           k_cache: Sequence[torch.Tensor], v_cache: Sequence[torch.Tensor],
-                           seq_idx: torch.Tensor, block_table: torch.Tensor,
-                           stream: Optional[torch.cuda.Stream] = None) -> None:
-    """Token-major sources [n_seq, seq_len, ...] into paged caches [n_pages, page_size, ...]
-    through block_table int32 [n_seq, max_pages_per_seq]."""
+@dataclasses.dataclass
+class KVPagedTables:
+    """Host pointer tables for civic_compact_kv_paged, built once per set of cache tensors."""
+    tables: tuple
+    n_layers: int
+    n_seq: int
+    seq_len: int
+    row_bytes: int
+    n_pages: int
+    page_size: int
+    keepalive: tuple
+
+
+def kv_paged_tables(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.Tensor],
+                    k_cache: Sequence[torch.Tensor], v_cache: Sequence[torch.Tensor]) -> KVPagedTables:
+    """Marshal token-major sources [n_seq, seq_len, ...] and paged caches [n_pages, page_size, ...]."""
     n_layers = len(k_src)
     if n_layers == 0 or not (len(v_src) == len(k_cache) == len(v_cache) == n_layers):
         raise ValueError("the four tensor lists must have one entry per layer")
@@ -345,24 +375,31 @@ def civic_compact_kv_paged(k_src: Sequence[torch.Tensor], v_src: Sequence[torch.
     if len(src_shape) < 3 or len(cache_shape) != len(src_shape) or cache_dtype != dtype or \
             src_shape[2:] != cache_shape[2:]:
         raise ValueError("source [n_seq, seq_len, ...] and cache [n_pages, page_size, ...] disagree")
-    n_seq, seq_len = src_shape[:2]
-    n_pages, page_size = cache_shape[:2]
     row_elems = 1
     for d in src_shape[2:]:
         row_elems *= d
-    if seq_idx.dim() != 2 or seq_idx.shape[0] != n_seq:
+    return KVPagedTables((_table(k_src, "k_src"), _table(v_src, "v_src"), _table(k_cache, "k_cache"),
+                          _table(v_cache, "v_cache")), n_layers, src_shape[0], src_shape[1],
+                         row_elems * k_src[0].element_size(), cache_shape[0], cache_shape[1],
+                         (tuple(k_src), tuple(v_src), tuple(k_cache), tuple(v_cache)))
+
+
+def civic_compact_kv_paged(tables: KVPagedTables, seq_idx: torch.Tensor, block_table: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Kept rows of every layer's K and V into the paged caches through block_table int32
+    [n_seq, max_pages_per_seq]: compact position j -> page block_table[s, j // page_size], slot j % page_size."""
+    t = tables
+    if seq_idx.dim() != 2 or seq_idx.shape[0] != t.n_seq:
         raise ValueError("seq_idx must be [n_seq, s_out]")
-    if block_table.dim() != 2 or block_table.shape[0] != n_seq:
+    if block_table.dim() != 2 or block_table.shape[0] != t.n_seq:
         raise ValueError("block_table must be [n_seq, max_pages_per_seq]")
     idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
     tab_ptr = _dev_ptr(block_table, "block_table", torch.int32)
-    with torch.cuda.device(_device_of(seq_idx, k_src[0], k_cache[0])):
-        _check(load().civic_compact_kv_paged(_table(k_src, "k_src"), _table(v_src, "v_src"),
-                                             _table(k_cache, "k_cache"), _table(v_cache, "v_cache"),
-                                             n_layers, n_seq, seq_len, seq_idx.shape[1],
-                                             row_elems * k_src[0].element_size(), idx_ptr, tab_ptr,
-                                             block_table.shape[1], page_size, n_pages,
-                                             _stream_ptr(stream)), "civic_compact_kv_paged")
+    with torch.cuda.device(_device_of(seq_idx, t.keepalive[0][0], t.keepalive[2][0])):
+        _check(load().civic_compact_kv_paged(*t.tables, t.n_layers, t.n_seq, t.seq_len, seq_idx.shape[1],
+                                             t.row_bytes, idx_ptr, tab_ptr, block_table.shape[1],
+                                             t.page_size, t.n_pages, _stream_ptr(stream)),
+               "civic_compact_kv_paged")
 
 
 def civic_merge_embeddings(text: torch.Tensor, visual: torch.Tensor, keep_idx: torch.Tensor,

@@ -87,9 +87,9 @@ def run_kv_heads(n_layers, n_seq, n_heads, seq_len, s_out, d, dtype=torch.int16,
     want_k, want_v = O.compact_kv_heads(ks, vs, idx)
     outs = [padded((n_seq, n_heads, s_out, d), dtype, 99) for _ in range(2 * n_layers)]
     kd, vd = [o[0] for o in outs[:n_layers]], [o[0] for o in outs[n_layers:]]
-    civic.civic_compact_kv_heads([torch.from_numpy(a).to(DEV) for a in ks],
-                                 [torch.from_numpy(a).to(DEV) for a in vs], kd, vd,
-                                 torch.from_numpy(idx).to(DEV))
+    tables = civic.kv_heads_tables([torch.from_numpy(a).to(DEV) for a in ks],
+                                   [torch.from_numpy(a).to(DEV) for a in vs], kd, vd)
+    civic.civic_compact_kv_heads(tables, torch.from_numpy(idx).to(DEV))
     for l in range(n_layers):
         assert np.array_equal(kd[l].cpu().numpy(), want_k[l]), f"K layer {l}"
         assert np.array_equal(vd[l].cpu().numpy(), want_v[l]), f"V layer {l}"
@@ -138,9 +138,9 @@ def run_kv_paged(n_layers, n_seq, seq_len, s_out, row_elems, page, seed=0, idx=N
     kc, vc = [o[0] for o in outs[:n_layers]], [o[0] for o in outs[n_layers:]]
     for dst, src in zip(kc + vc, old_k + old_v):
         dst.copy_(torch.from_numpy(src))
-    civic.civic_compact_kv_paged([torch.from_numpy(a).to(DEV) for a in ks],
-                                 [torch.from_numpy(a).to(DEV) for a in vs], kc, vc,
-                                 torch.from_numpy(idx).to(DEV), torch.from_numpy(table).to(DEV))
+    tables = civic.kv_paged_tables([torch.from_numpy(a).to(DEV) for a in ks],
+                                   [torch.from_numpy(a).to(DEV) for a in vs], kc, vc)
+    civic.civic_compact_kv_paged(tables, torch.from_numpy(idx).to(DEV), torch.from_numpy(table).to(DEV))
     for l in range(n_layers):
         assert np.array_equal(kc[l].cpu().numpy(), want_k[l]), f"K cache layer {l}"
         assert np.array_equal(vc[l].cpu().numpy(), want_v[l]), f"V cache layer {l}"
