@@ -41,7 +41,8 @@ typedef enum {
     CIVIC_ERR_FLOOR_EXCEEDS_K = 3, /* sum over regions of min(m, |region|) > k                    */
     CIVIC_ERR_ALIGNMENT = 4,       /* row size or pointer not a multiple of 4 bytes               */
     CIVIC_ERR_UNSUPPORTED = 5,     /* segment too large for one thread block's shared memory      */
-    CIVIC_ERR_CUDA = 6             /* a CUDA runtime call failed                                  */
+    CIVIC_ERR_CUDA = 6,            /* a CUDA runtime call failed                                  */
+    CIVIC_ERR_WORKSPACE = 7        /* scratch memory missing or smaller than required             */
 } civic_status_t;
 
 /* Selection problem of ONE segment (an image or a video); every segment of a call shares it.
@@ -92,6 +93,30 @@ civic_status_t civic_select(const float* scores, int32_t n_seg, const civic_sele
 civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_select_desc_t* desc,
                                 int32_t seq_len, int32_t vis_start, int32_t* keep_idx,
                                 int32_t* seq_idx, void* stream);
+
+/*
+ * civic_select_large -- civic_select for segments beyond one thread block (long videos).
+ *
+ * Paper: as civic_select; the paper's stated next step is long-form video (Section 5), where
+ * one segment has far more tokens than a thread block can hold.  Same definition and the same
+ * output as civic_select for any n up to 2^31 - 1, computed by many thread blocks per segment
+ * in five consecutive launches that communicate through `workspace`.
+ *
+ * workspace        dev, caller-owned scratch of at least civic_select_workspace_bytes(...)
+ *                  bytes, 256-byte aligned; contents on entry are irrelevant, contents on return
+ *                  are unspecified.  Two calls that may run concurrently need separate workspaces.
+ * chunk_tokens     tokens handled by one thread block; 0 = the library default (16384, also the
+ *                  maximum).  One "region row" (region_h token rows of w tokens) must fit into a
+ *                  chunk, otherwise CIVIC_ERR_UNSUPPORTED.
+ * CIVIC_ERR_WORKSPACE if workspace is NULL or too small.  The only allocation-free requirement
+ * on the caller is this scratch buffer; the call itself allocates nothing.
+ */
+civic_status_t civic_select_large(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                                  int32_t* keep_idx, void* workspace, size_t workspace_bytes,
+                                  int32_t chunk_tokens, void* stream);
+
+/* Scratch bytes civic_select_large needs for this shape; 0 if the shape is invalid or unsupported. */
+size_t civic_select_workspace_bytes(const civic_select_desc_t* desc, int32_t n_seg, int32_t chunk_tokens);
 
 /* Largest n = t*h*w that civic_select accepts. */
 int32_t civic_select_max_tokens(void);

@@ -20,14 +20,14 @@ LIB_PATH = os.path.join(_HERE, "libcivic.so")
 
 CIVIC_OK = 0
 STATUS_NAMES = ("CIVIC_OK", "CIVIC_ERR_INVALID_ARG", "CIVIC_ERR_K_RANGE", "CIVIC_ERR_FLOOR_EXCEEDS_K",
-                "CIVIC_ERR_ALIGNMENT", "CIVIC_ERR_UNSUPPORTED", "CIVIC_ERR_CUDA")
+                "CIVIC_ERR_ALIGNMENT", "CIVIC_ERR_UNSUPPORTED", "CIVIC_ERR_CUDA", "CIVIC_ERR_WORKSPACE")
 
 # every symbol include/civic.h declares
 EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "civic_compact",
            "civic_seq_indices", "civic_compact_kv", "civic_status_string", "civic_last_cuda_error",
            "civic_launch_count", "civic_select_seq", "civic_set_programmatic_launch",
            "civic_compact_kv_heads", "civic_compact_kv_paged", "civic_merge_embeddings",
-           "civic_compact_pos_planes")
+           "civic_compact_pos_planes", "civic_select_large", "civic_select_workspace_bytes")
 
 
 class CivicError(RuntimeError):
@@ -90,6 +90,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_merge_embeddings.restype = ctypes.c_int
     lib.civic_compact_pos_planes.argtypes = [vp, i32, i32, i32, vp, i32, vp, vp]
     lib.civic_compact_pos_planes.restype = ctypes.c_int
+    lib.civic_select_large.argtypes = [vp, i32, ctypes.POINTER(SelectDesc), vp, vp, sz, i32, vp]
+    lib.civic_select_large.restype = ctypes.c_int
+    lib.civic_select_workspace_bytes.argtypes = [ctypes.POINTER(SelectDesc), i32, i32]
+    lib.civic_select_workspace_bytes.restype = sz
     _lib = lib
     return lib
 
@@ -177,6 +181,34 @@ def civic_select_seq(scores: torch.Tensor, desc: SelectDesc, seq_len: int, vis_s
     with torch.cuda.device(_device_of(scores, keep_idx)):
         _check(load().civic_select_seq(*args, _stream_ptr(stream)), "civic_select_seq")
     return keep_idx, seq_idx
+
+
+def select_workspace_bytes(desc: SelectDesc, n_seg: int, chunk_tokens: int = 0) -> int:
+    return int(load().civic_select_workspace_bytes(ctypes.byref(desc), n_seg, chunk_tokens))
+
+
+def civic_select_large(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None, chunk_tokens: int = 0,
+                       stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """civic_select for segments of any size: many thread blocks per segment, scratch in `workspace`
+    (a uint8 CUDA tensor of at least select_workspace_bytes(...) bytes; allocated here if omitted)."""
+    if scores.dim() != 2 or scores.shape[1] != desc.t * desc.h * desc.w:
+        raise ValueError("scores must be [n_seg, t*h*w]")
+    n_seg = scores.shape[0]
+    dev = _device_of(scores)
+    if keep_idx is None:
+        keep_idx = torch.empty((n_seg, max(desc.k, 0)), dtype=torch.int32, device=dev)
+    elif tuple(keep_idx.shape) != (n_seg, desc.k):
+        raise ValueError("keep_idx must be [n_seg, k]")
+    if workspace is None:
+        workspace = torch.empty(max(select_workspace_bytes(desc, n_seg, chunk_tokens), 256),
+                                dtype=torch.uint8, device=dev)
+    args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
+            _dev_ptr(keep_idx, "keep_idx", torch.int32), _dev_ptr(workspace, "workspace", torch.uint8),
+            workspace.numel(), chunk_tokens)
+    with torch.cuda.device(dev):
+        _check(load().civic_select_large(*args, _stream_ptr(stream)), "civic_select_large")
+    return keep_idx
 
 
 def set_programmatic_launch(enable: bool) -> bool:

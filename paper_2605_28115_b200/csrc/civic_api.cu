@@ -8,6 +8,7 @@
 
 #include "gather.cuh"
 #include "select.cuh"
+#include "select_large.cuh"
 
 namespace {
 
@@ -155,6 +156,72 @@ civic_status_t launch_kv(civic::GatherParams base, const void* const* k_src, con
     return CIVIC_OK;
 }
 
+// Work split and scratch layout of the many-block selection.
+struct LargePlan {
+    int32_t n, n_rh, rows_per_chunk, n_chunks, chunk_tokens;
+    size_t hist_off, counts_off, flags_off, total;  // byte offsets into the workspace
+};
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// CIVIC_OK and a filled plan, or the reason the shape cannot be handled.
+civic_status_t plan_large(const civic_select_desc_t& d, int32_t n_seg, int32_t chunk_tokens, LargePlan& pl)
+{
+    if (reserved_count(d) < 0 || n_seg < 0 || chunk_tokens < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)d.t * d.h * d.w;
+    if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (chunk_tokens == 0 || chunk_tokens > civic::kLargeMaxChunk) chunk_tokens = civic::kLargeMaxChunk;
+    const int64_t rh = d.region_h < d.h ? d.region_h : d.h;  // tokens of the tallest region row
+    const int64_t row_tokens = rh * d.w;
+    if (row_tokens > chunk_tokens) return CIVIC_ERR_UNSUPPORTED;
+    pl.n = (int32_t)n;
+    pl.n_rh = (d.h + d.region_h - 1) / d.region_h;
+    pl.rows_per_chunk = (int32_t)(chunk_tokens / row_tokens);
+    const int64_t region_rows = (int64_t)d.t * pl.n_rh;
+    pl.n_chunks = (int32_t)((region_rows + pl.rows_per_chunk - 1) / pl.rows_per_chunk);
+    pl.chunk_tokens = (int32_t)(pl.rows_per_chunk * row_tokens);
+    if ((int64_t)pl.n_chunks * n_seg > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    pl.hist_off = 0;
+    pl.counts_off = round_up((size_t)n_seg * (3 * civic::kLargeBins + civic::kLargeSelWords) * 4, 256);
+    pl.flags_off = pl.counts_off + round_up((size_t)n_seg * pl.n_chunks * 2 * 4, 256);
+    pl.total = pl.flags_off + round_up((size_t)n_seg * (size_t)n, 256);
+    return CIVIC_OK;
+}
+
+// The five launches of the many-block selection; `ws` holds pl.total bytes of scratch.
+civic_status_t launch_large(const float* scores, int32_t n_seg, const civic_select_desc_t& d,
+                            int32_t* keep_idx, char* ws, const LargePlan& pl, int32_t k_fill,
+                            cudaStream_t stream)
+{
+    civic::LargeParams p;
+    p.scores = scores;
+    p.keep_idx = keep_idx;
+    p.n = pl.n; p.t = d.t; p.h = d.h; p.w = d.w;
+    p.region_h = d.region_h; p.region_w = d.region_w;
+    p.m = d.floor_per_region; p.k = d.k; p.k_fill = k_fill;
+    p.n_rh = pl.n_rh; p.rows_per_chunk = pl.rows_per_chunk; p.n_chunks = pl.n_chunks;
+    p.hist = (uint32_t*)(ws + pl.hist_off);
+    p.sel = p.hist + (size_t)n_seg * 3 * civic::kLargeBins;
+    p.counts = (uint32_t*)(ws + pl.counts_off);
+    p.flags = (uint8_t*)(ws + pl.flags_off);
+    // histograms and scalars start at zero
+    CIVIC_CUDA_TRY(cudaMemsetAsync(ws + pl.hist_off, 0,
+                                   (size_t)n_seg * (3 * civic::kLargeBins + civic::kLargeSelWords) * 4, stream));
+    const size_t smem = (size_t)(civic::kLargeBins + civic::kLargeMaxChunk / 32 + ((pl.chunk_tokens + 31) & ~31)) * 4;
+    if (smem > 48 * 1024)
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::large_floor_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const unsigned grid = (unsigned)(n_seg * pl.n_chunks), threads = civic::kLargeThreads;
+    const bool pdl = programmatic();
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::large_floor_kernel, grid, threads, smem, stream, p));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::large_hist_kernel<1>, grid, threads, 0, stream, p));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::large_hist_kernel<2>, grid, threads, 0, stream, p));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::large_count_kernel, grid, threads, 0, stream, p));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::large_place_kernel, grid, threads, 0, stream, p));
+    g_launches.fetch_add(5, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
 civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
                            int32_t* keep_idx, int32_t* seq_idx, int32_t seq_len, int32_t vis_start,
                            void* stream)
@@ -212,6 +279,7 @@ const char* civic_status_string(civic_status_t s)
         case CIVIC_ERR_ALIGNMENT: return "CIVIC_ERR_ALIGNMENT";
         case CIVIC_ERR_UNSUPPORTED: return "CIVIC_ERR_UNSUPPORTED";
         case CIVIC_ERR_CUDA: return "CIVIC_ERR_CUDA";
+        case CIVIC_ERR_WORKSPACE: return "CIVIC_ERR_WORKSPACE";
     }
     return "CIVIC_ERR_UNKNOWN";
 }
@@ -269,6 +337,40 @@ civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_
         return civic_seq_indices(keep_idx, n_seq, 0, seq_len, vis_start, (int32_t)n, seq_idx, stream);
     }
     return select_impl(scores, n_seq, desc, keep_idx, seq_idx, seq_len, vis_start, stream);
+}
+
+size_t civic_select_workspace_bytes(const civic_select_desc_t* desc, int32_t n_seg, int32_t chunk_tokens)
+{
+    LargePlan pl;
+    if (!desc || plan_large(*desc, n_seg, chunk_tokens, pl) != CIVIC_OK) return 0;
+    return pl.total;
+}
+
+civic_status_t civic_select_large(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                                  int32_t* keep_idx, void* workspace, size_t workspace_bytes,
+                                  int32_t chunk_tokens, void* stream)
+{
+    if (!desc || n_seg < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n_res = reserved_count(*desc);
+    if (n_res < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)desc->t * desc->h * desc->w;
+    if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (desc->k < 0 || desc->k > n) return CIVIC_ERR_K_RANGE;
+    if (n_res > desc->k) return CIVIC_ERR_FLOOR_EXCEEDS_K;
+    LargePlan pl;
+    const civic_status_t st = plan_large(*desc, n_seg, chunk_tokens, pl);
+    if (st != CIVIC_OK) return st;
+    if (n_seg == 0 || desc->k == 0) return CIVIC_OK;
+    if (!scores || !keep_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(scores, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < pl.total) return CIVIC_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return CIVIC_ERR_ALIGNMENT;
+    if (overlaps(scores, (size_t)n_seg * n * 4, keep_idx, (size_t)n_seg * desc->k * 4) ||
+        overlaps(workspace, pl.total, keep_idx, (size_t)n_seg * desc->k * 4) ||
+        overlaps(workspace, pl.total, scores, (size_t)n_seg * n * 4))
+        return CIVIC_ERR_INVALID_ARG;
+    return launch_large(scores, n_seg, *desc, keep_idx, (char*)workspace, pl, (int32_t)(desc->k - n_res),
+                        (cudaStream_t)stream);
 }
 
 civic_status_t civic_compact(const void* hidden, size_t row_bytes, const int32_t* pos_ids,

@@ -142,6 +142,33 @@ def test_compact_kv_validation(lib):
     assert f(ks, vs, kd, vd, -1, 2, 16, 8, 64, 0x10, None) == 1
 
 
+def test_select_large_validation(lib):
+    D = civic.SelectDesc
+    f = lambda d, n_seg=1, scores=0x100000, keep=0x200000, ws=0x300000, ws_bytes=1 << 30, chunk=0: \
+        lib.civic_select_large(scores, n_seg, ctypes.byref(d), keep, ws, ws_bytes, chunk, None)
+    before = lib.civic_launch_count()
+    d = D(8, 40, 40, 4, 4, 1, 4000)
+    need = lib.civic_select_workspace_bytes(ctypes.byref(d), 2, 0)
+    # 2 segments: histograms + scalars, per-chunk counts, one flag byte per token, 256-byte sections
+    assert need >= 2 * (3 * 2048 + 16) * 4 + 2 * 12800 and need % 256 == 0
+    assert lib.civic_select_workspace_bytes(ctypes.byref(D(8, 40, 40, 0, 4, 1, 4000)), 2, 0) == 0
+    assert lib.civic_select_workspace_bytes(ctypes.byref(d), 2, 100) == 0  # region row of 160 tokens
+    assert f(d, ws=None) == 7
+    assert f(d, ws_bytes=need // 2 - 1) == 7  # one segment needs about half
+    assert f(d, ws=0x300010) == 4
+    assert f(d, chunk=100) == 5
+    assert f(d, chunk=-1) == 1
+    assert f(D(8, 40, 40, 4, 4, 1, 12801)) == 2
+    assert f(D(8, 40, 40, 4, 4, 1, 799)) == 3
+    assert f(d, scores=None) == 1
+    assert f(d, keep=0x300100) == 1  # output inside the workspace
+    assert f(d, n_seg=0) == 0
+    assert f(D(8, 40, 40, 4, 4, 0, 0)) == 0
+    assert f(D(1, 4, 70000, 4, 4, 1, 70000)) == 5  # one region row holds 280000 tokens
+    assert lib.civic_launch_count() == before
+    assert lib.civic_status_string(7).decode() == "CIVIC_ERR_WORKSPACE"
+
+
 def test_adjacent_calls_validation(lib):
     P = ctypes.c_void_p * 2
     ks, vs = P(0x100000, 0x200000), P(0x300000, 0x400000)
