@@ -105,15 +105,47 @@ civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_
  * workspace        dev, caller-owned scratch of at least civic_select_workspace_bytes(...)
  *                  bytes, 256-byte aligned; contents on entry are irrelevant, contents on return
  *                  are unspecified.  Two calls that may run concurrently need separate workspaces.
- * chunk_tokens     tokens handled by one thread block; 0 = the library default (16384, also the
- *                  maximum).  One "region row" (region_h token rows of w tokens) must fit into a
- *                  chunk, otherwise CIVIC_ERR_UNSUPPORTED.
+ * chunk_tokens     tokens handled by one thread block, at most 16384; 0 = the library default
+ *                  (sized from the shapes for about one block per SM, 2048 .. 16384).  One
+ *                  "region row" (region_h token rows of w tokens) must fit into a chunk,
+ *                  otherwise CIVIC_ERR_UNSUPPORTED.  Pass the same value to
+ *                  civic_select_workspace_bytes.
  * CIVIC_ERR_WORKSPACE if workspace is NULL or too small.  The only allocation-free requirement
  * on the caller is this scratch buffer; the call itself allocates nothing.
  */
 civic_status_t civic_select_large(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
                                   int32_t* keep_idx, void* workspace, size_t workspace_bytes,
                                   int32_t chunk_tokens, void* stream);
+
+/*
+ * civic_select_ragged -- civic_select for a batch whose segments differ in shape and budget.
+ *
+ * Paper: as civic_select; instance-adaptive token budgets and mixed image/video batches are the
+ * paper's stated next steps (Section 5).  Segment s has its own descriptor descs[s] (grid,
+ * tiles, floor, k).  Scores are concatenated: segment s starts at the sum of the earlier
+ * segments' n; keep_idx likewise at the sum of the earlier k.
+ *
+ * scores    dev  [sum n] fp32
+ * descs     host [n_seg]
+ * keep_idx  dev  [sum k] int32, written: ascending segment-local token indices per segment
+ * flat_idx  dev  [sum k] int32 or NULL, written: the same tokens numbered over the concatenated
+ *           scores (keep_idx + start of the segment).  With it a ragged batch is compacted by
+ *           ONE civic_compact call: n_seg = 1, n = sum n, k = sum k, keep_idx = flat_idx.
+ * Every segment must fit one thread block (n <= civic_select_max_tokens()); sum n < 2^31.
+ * One launch per 64 segments.
+ */
+civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civic_select_desc_t* descs,
+                                   int32_t* keep_idx, int32_t* flat_idx, void* stream);
+
+/*
+ * civic_floor_from_ratio -- Table 2's "Min Keep Ratio" as a floor_per_region value.
+ *
+ * Paper: Section 4.5 / Table 2 vary the retention floor as a ratio (0.0, 0.2, 0.5) of the
+ * tokens of a spatial region.  Returns the smallest m with m >= (num / den) * region_h *
+ * region_w, in exact integer arithmetic (0/1 -> 0, i.e. plain top-K); -1 on invalid arguments
+ * (num > den, den < 1, empty tile).  Host-only helper, nothing is launched.
+ */
+int32_t civic_floor_from_ratio(int32_t region_h, int32_t region_w, int32_t num, int32_t den);
 
 /* Scratch bytes civic_select_large needs for this shape; 0 if the shape is invalid or unsupported. */
 size_t civic_select_workspace_bytes(const civic_select_desc_t* desc, int32_t n_seg, int32_t chunk_tokens);

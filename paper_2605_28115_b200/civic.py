@@ -27,7 +27,8 @@ EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "c
            "civic_seq_indices", "civic_compact_kv", "civic_status_string", "civic_last_cuda_error",
            "civic_launch_count", "civic_select_seq", "civic_set_programmatic_launch",
            "civic_compact_kv_heads", "civic_compact_kv_paged", "civic_merge_embeddings",
-           "civic_compact_pos_planes", "civic_select_large", "civic_select_workspace_bytes")
+           "civic_compact_pos_planes", "civic_select_large", "civic_select_workspace_bytes",
+           "civic_select_ragged", "civic_floor_from_ratio")
 
 
 class CivicError(RuntimeError):
@@ -94,6 +95,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_select_large.restype = ctypes.c_int
     lib.civic_select_workspace_bytes.argtypes = [ctypes.POINTER(SelectDesc), i32, i32]
     lib.civic_select_workspace_bytes.restype = sz
+    lib.civic_select_ragged.argtypes = [vp, i32, ctypes.POINTER(SelectDesc), vp, vp, vp]
+    lib.civic_select_ragged.restype = ctypes.c_int
+    lib.civic_floor_from_ratio.argtypes = [i32, i32, i32, i32]
+    lib.civic_floor_from_ratio.restype = i32
     _lib = lib
     return lib
 
@@ -209,6 +214,37 @@ def civic_select_large(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optiona
     with torch.cuda.device(dev):
         _check(load().civic_select_large(*args, _stream_ptr(stream)), "civic_select_large")
     return keep_idx
+
+
+def floor_from_ratio(region_h: int, region_w: int, num: int, den: int) -> int:
+    """Smallest floor_per_region m with m >= (num/den) * region_h * region_w; -1 on bad arguments."""
+    return int(load().civic_floor_from_ratio(region_h, region_w, num, den))
+
+
+def civic_select_ragged(scores: torch.Tensor, descs: Sequence[SelectDesc],
+                        keep_idx: Optional[torch.Tensor] = None, flat_idx: Optional[torch.Tensor] = None,
+                        want_flat: bool = True, stream: Optional[torch.cuda.Stream] = None):
+    """scores fp32 [sum n] (segments concatenated), one SelectDesc per segment ->
+    (segment-local keep indices int32 [sum k], the same tokens numbered over the concatenation or None)."""
+    total_n = sum(d.t * d.h * d.w for d in descs)
+    total_k = sum(max(d.k, 0) for d in descs)
+    if scores.dim() != 1 or scores.shape[0] != total_n:
+        raise ValueError("scores must be the 1-D concatenation of all segments")
+    dev = _device_of(scores)
+    if keep_idx is None:
+        keep_idx = torch.empty((total_k,), dtype=torch.int32, device=dev)
+    elif tuple(keep_idx.shape) != (total_k,):
+        raise ValueError("keep_idx must be [sum k]")
+    if flat_idx is None and want_flat:
+        flat_idx = torch.empty((total_k,), dtype=torch.int32, device=dev)
+    elif flat_idx is not None and tuple(flat_idx.shape) != (total_k,):
+        raise ValueError("flat_idx must be [sum k]")
+    table = (SelectDesc * max(len(descs), 1))(*descs)
+    args = (_dev_ptr(scores, "scores", torch.float32), len(descs), table,
+            _dev_ptr(keep_idx, "keep_idx", torch.int32), _dev_ptr(flat_idx, "flat_idx", torch.int32))
+    with torch.cuda.device(dev):
+        _check(load().civic_select_ragged(*args, _stream_ptr(stream)), "civic_select_ragged")
+    return keep_idx, flat_idx
 
 
 def set_programmatic_launch(enable: bool) -> bool:

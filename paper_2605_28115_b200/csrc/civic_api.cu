@@ -162,6 +162,10 @@ struct LargePlan {
     size_t hist_off, counts_off, flags_off, total;  // byte offsets into the workspace
 };
 
+// The default chunk size depends on shapes only (not on the device), so that the workspace size
+// is a pure function of the arguments: 148 = one block for each SM of a B200.
+constexpr int64_t kLargeBlocksTarget = 148;
+
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // CIVIC_OK and a filled plan, or the reason the shape cannot be handled.
@@ -170,9 +174,18 @@ civic_status_t plan_large(const civic_select_desc_t& d, int32_t n_seg, int32_t c
     if (reserved_count(d) < 0 || n_seg < 0 || chunk_tokens < 0) return CIVIC_ERR_INVALID_ARG;
     const int64_t n = (int64_t)d.t * d.h * d.w;
     if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
-    if (chunk_tokens == 0 || chunk_tokens > civic::kLargeMaxChunk) chunk_tokens = civic::kLargeMaxChunk;
     const int64_t rh = d.region_h < d.h ? d.region_h : d.h;  // tokens of the tallest region row
     const int64_t row_tokens = rh * d.w;
+    if (chunk_tokens > civic::kLargeMaxChunk) chunk_tokens = civic::kLargeMaxChunk;
+    if (chunk_tokens == 0) {
+        // default: about one block per SM over the whole launch, between 2048 tokens and the
+        // capacity (measured on B200: fewer, larger blocks leave SMs idle; many more blocks pay
+        // for their atomic flushes into the shared global histograms)
+        int64_t c = ((int64_t)n_seg * n + kLargeBlocksTarget - 1) / kLargeBlocksTarget;
+        c = c < 2048 ? 2048 : (c > civic::kLargeMaxChunk ? civic::kLargeMaxChunk : c);
+        if (c < row_tokens && row_tokens <= civic::kLargeMaxChunk) c = row_tokens;
+        chunk_tokens = (int32_t)c;
+    }
     if (row_tokens > chunk_tokens) return CIVIC_ERR_UNSUPPORTED;
     pl.n = (int32_t)n;
     pl.n_rh = (d.h + d.region_h - 1) / d.region_h;
@@ -222,6 +235,12 @@ civic_status_t launch_large(const float* scores, int32_t n_seg, const civic_sele
     return CIVIC_OK;
 }
 
+int select_threads(int64_t n)
+{
+    const int64_t threads = (n + 31) / 32 * 32;
+    return (int)(threads < 128 ? 128 : (threads > 1024 ? 1024 : threads));
+}
+
 civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
                            int32_t* keep_idx, int32_t* seq_idx, int32_t seq_len, int32_t vis_start,
                            void* stream)
@@ -243,22 +262,17 @@ civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_selec
     civic::SelectParams p;
     p.scores = scores;
     p.keep_idx = keep_idx;
-    p.n = (int32_t)n;
-    p.t = desc->t; p.h = desc->h; p.w = desc->w;
-    p.region_h = desc->region_h; p.region_w = desc->region_w;
-    p.m = desc->floor_per_region;
-    p.k = desc->k;
-    p.k_fill = (int32_t)(desc->k - n_res);
+    p.shape = civic::SegShape{(int32_t)n, desc->t, desc->h, desc->w, desc->region_h, desc->region_w,
+                              desc->floor_per_region, desc->k, (int32_t)(desc->k - n_res)};
     p.seq_idx = seq_idx;
     p.seq_len = seq_len;
     p.vis_start = vis_start;
 
-    const size_t smem = civic::select_smem_bytes(p.n);
+    const size_t smem = civic::select_smem_bytes(p.shape.n);
     if (smem > 48 * 1024)
         CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_kernel,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int threads = (p.n + 31) / 32 * 32;
-    threads = threads < 128 ? 128 : (threads > 1024 ? 1024 : threads);
+    const int threads = select_threads(p.shape.n);
     CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::select_kernel, (unsigned)n_seg, (unsigned)threads,
                                  smem, (cudaStream_t)stream, p));
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -337,6 +351,71 @@ civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_
         return civic_seq_indices(keep_idx, n_seq, 0, seq_len, vis_start, (int32_t)n, seq_idx, stream);
     }
     return select_impl(scores, n_seq, desc, keep_idx, seq_idx, seq_len, vis_start, stream);
+}
+
+civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civic_select_desc_t* descs,
+                                   int32_t* keep_idx, int32_t* flat_idx, void* stream)
+{
+    if (n_seg < 0 || (n_seg > 0 && !descs)) return CIVIC_ERR_INVALID_ARG;
+    // validate every segment before anything is launched
+    int64_t total_n = 0, total_k = 0;
+    for (int s = 0; s < n_seg; ++s) {
+        const civic_select_desc_t& d = descs[s];
+        const int64_t n_res = reserved_count(d);
+        if (n_res < 0) return CIVIC_ERR_INVALID_ARG;
+        const int64_t n = (int64_t)d.t * d.h * d.w;
+        if (n > civic_select_max_tokens()) return CIVIC_ERR_UNSUPPORTED;
+        if (d.k < 0 || d.k > n) return CIVIC_ERR_K_RANGE;
+        if (n_res > d.k) return CIVIC_ERR_FLOOR_EXCEEDS_K;
+        total_n += n;
+        total_k += d.k;
+        if (total_n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    }
+    if (total_k == 0) return CIVIC_OK;
+    if (!scores || !keep_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(scores, 4) || !aligned(keep_idx, 4) || !aligned(flat_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (overlaps(scores, (size_t)total_n * 4, keep_idx, (size_t)total_k * 4) ||
+        overlaps(scores, (size_t)total_n * 4, flat_idx, (size_t)total_k * 4) ||
+        overlaps(keep_idx, (size_t)total_k * 4, flat_idx, (size_t)total_k * 4))
+        return CIVIC_ERR_INVALID_ARG;
+
+    int32_t score_off = 0, out_off = 0;
+    for (int s0 = 0; s0 < n_seg; s0 += civic::kMaxRaggedSegs) {
+        const int ns = n_seg - s0 < civic::kMaxRaggedSegs ? n_seg - s0 : civic::kMaxRaggedSegs;
+        civic::RaggedParams p;
+        memset(&p, 0, sizeof p);
+        p.scores = scores;
+        p.keep_idx = keep_idx;
+        p.flat_idx = flat_idx;
+        int32_t n_max = 1;
+        for (int s = 0; s < ns; ++s) {
+            const civic_select_desc_t& d = descs[s0 + s];
+            const int32_t n = d.t * d.h * d.w;
+            p.shape[s] = civic::SegShape{n, d.t, d.h, d.w, d.region_h, d.region_w, d.floor_per_region, d.k,
+                                         (int32_t)(d.k - reserved_count(d))};
+            p.score_off[s] = score_off;
+            p.out_off[s] = out_off;
+            score_off += n;
+            out_off += d.k;
+            n_max = n > n_max ? n : n_max;
+        }
+        const size_t smem = civic::select_smem_bytes(n_max);
+        if (smem > 48 * 1024)
+            CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_ragged_kernel,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::select_ragged_kernel, (unsigned)ns,
+                                     (unsigned)select_threads(n_max), smem, (cudaStream_t)stream, p));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    return CIVIC_OK;
+}
+
+int32_t civic_floor_from_ratio(int32_t region_h, int32_t region_w, int32_t num, int32_t den)
+{
+    if (region_h < 1 || region_w < 1 || num < 0 || den < 1 || num > den) return -1;
+    const int64_t size = (int64_t)region_h * region_w;
+    if (size > INT32_MAX) return -1;
+    return (int32_t)((size * num + den - 1) / den);
 }
 
 size_t civic_select_workspace_bytes(const civic_select_desc_t* desc, int32_t n_seg, int32_t chunk_tokens)

@@ -20,17 +20,33 @@
 
 namespace civic {
 
+// Shape of one segment's selection problem.
+struct SegShape {
+    int32_t n, t, h, w;
+    int32_t region_h, region_w;
+    int32_t m;       // floor per region
+    int32_t k;       // kept per segment
+    int32_t k_fill;  // k - reserved count (>= 0), shape-only
+};
+
 struct SelectParams {
     const float* scores;  // [n_seg, n]
     int32_t* keep_idx;    // [n_seg, k]
-    int32_t n, t, h, w;
-    int32_t region_h, region_w;
-    int32_t m;      // floor per region
-    int32_t k;      // kept per segment
-    int32_t k_fill; // k - reserved count (>= 0), shape-only
+    SegShape shape;       // shared by all segments
     // optional fused epilogue: kept positions of the full sequence, see seq_indices_kernel
     int32_t* seq_idx;   // [n_seg, seq_len - n + k] or NULL
     int32_t seq_len, vis_start;
+};
+
+// A ragged batch: every block reads its own segment's shape and offsets from the parameters.
+constexpr int kMaxRaggedSegs = 64;
+struct RaggedParams {
+    const float* scores;  // concatenated, segment s starts at score_off[s]
+    int32_t* keep_idx;    // concatenated, segment s starts at out_off[s]; segment-local indices
+    int32_t* flat_idx;    // same layout, indices over the concatenated scores; or NULL
+    SegShape shape[kMaxRaggedSegs];
+    int32_t score_off[kMaxRaggedSegs];
+    int32_t out_off[kMaxRaggedSegs];
 };
 
 __host__ __device__ inline size_t select_smem_bytes(int n)
@@ -51,10 +67,13 @@ __device__ __forceinline__ uint32_t score_key(float s)
 // (32 warps share 4 schedulers), not by latency.  Everything that need not be done per token
 // is done by few threads: the floor with m = 1 by one thread per region, the 256-bin digit
 // scan by one warp.
-__global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
+__device__ __forceinline__ void select_block(const SegShape& d, const float* __restrict__ scores,
+                                             int32_t* __restrict__ out, int32_t* __restrict__ seq,
+                                             int seq_len, int vis_start, int32_t* __restrict__ flat,
+                                             int flat_base)
 {
     extern __shared__ __align__(16) uint32_t smem[];
-    const int n = p.n;
+    const int n = d.n;
     const int n_words = (n + 31) >> 5;
     const int n_pad = n_words << 5;
     uint32_t* hist = smem;                 // [4][256], one histogram per radix pass
@@ -65,8 +84,6 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
 
     const int tid = threadIdx.x, nt = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, n_warps = nt >> 5;
-    const float* scores = p.scores + (size_t)blockIdx.x * n;
-    int32_t* out = p.keep_idx + (size_t)blockIdx.x * p.k;
     release_next_kernel();
     wait_for_prior_kernels();
 
@@ -77,19 +94,19 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
     __syncthreads();
 
     // 2. floor
-    if (p.m == 1) {
+    if (d.m == 1) {
         // one thread per region walks its tile in index order and keeps the first maximum
-        const int n_rh = (p.h + p.region_h - 1) / p.region_h, n_rw = (p.w + p.region_w - 1) / p.region_w;
-        const int n_reg = p.t * n_rh * n_rw;
+        const int n_rh = (d.h + d.region_h - 1) / d.region_h, n_rw = (d.w + d.region_w - 1) / d.region_w;
+        const int n_reg = d.t * n_rh * n_rw;
         for (int r = tid; r < n_reg; r += nt) {
             const int tt = r / (n_rh * n_rw), rem = r - tt * (n_rh * n_rw);
             const int ry = rem / n_rw, rx = rem - ry * n_rw;
-            const int h0 = ry * p.region_h, w0 = rx * p.region_w;
-            const int h1 = min(h0 + p.region_h, p.h), w1 = min(w0 + p.region_w, p.w);
-            int best = (tt * p.h + h0) * p.w + w0;
+            const int h0 = ry * d.region_h, w0 = rx * d.region_w;
+            const int h1 = min(h0 + d.region_h, d.h), w1 = min(w0 + d.region_w, d.w);
+            int best = (tt * d.h + h0) * d.w + w0;
             uint32_t best_key = keys[best];
             for (int y = h0; y < h1; ++y) {
-                const int row = (tt * p.h + y) * p.w;
+                const int row = (tt * d.h + y) * d.w;
                 for (int x = w0; x < w1; ++x) {
                     const uint32_t key = keys[row + x];
                     if (key > best_key) { best_key = key; best = row + x; }
@@ -97,27 +114,27 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
             }
             atomicOr(&resv[best >> 5], 1u << (best & 31));
         }
-    } else if (p.m > 1) {
+    } else if (d.m > 1) {
         // general m: a token is reserved iff fewer than m tokens of its tile beat it
-        const int hw = p.h * p.w;
+        const int hw = d.h * d.w;
         for (int i = tid; i < n_pad; i += nt) {
             bool r = false;
             if (i < n) {
                 const int tt = i / hw, rem = i - tt * hw;
-                const int hh = rem / p.w, ww = rem - hh * p.w;
-                const int h0 = (hh / p.region_h) * p.region_h, w0 = (ww / p.region_w) * p.region_w;
-                const int h1 = min(h0 + p.region_h, p.h), w1 = min(w0 + p.region_w, p.w);
+                const int hh = rem / d.w, ww = rem - hh * d.w;
+                const int h0 = (hh / d.region_h) * d.region_h, w0 = (ww / d.region_w) * d.region_w;
+                const int h1 = min(h0 + d.region_h, d.h), w1 = min(w0 + d.region_w, d.w);
                 const uint32_t mine = keys[i];
                 int better = 0;
                 for (int y = h0; y < h1; ++y) {
-                    const int row = (tt * p.h + y) * p.w;
+                    const int row = (tt * d.h + y) * d.w;
                     for (int x = w0; x < w1; ++x) {
                         const int j = row + x;
                         const uint32_t other = keys[j];
                         better += (other > mine) || (other == mine && j < i);
                     }
                 }
-                r = better < p.m;
+                r = better < d.m;
             }
             const uint32_t word = __ballot_sync(0xFFFFFFFFu, r);
             if (lane == 0) resv[i >> 5] = word;
@@ -127,9 +144,9 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
 
     // 3. radix select of the k_fill-th best non-reserved key, 8 bits per pass from the top
     uint32_t prefix = 0xFFFFFFFFu, need_eq = 0;
-    if (p.k_fill > 0) {
+    if (d.k_fill > 0) {
         uint32_t mask = 0;
-        uint32_t rank = (uint32_t)p.k_fill;  // 1-based rank among the candidates still matching
+        uint32_t rank = (uint32_t)d.k_fill;  // 1-based rank among the candidates still matching
         prefix = 0;
 #pragma unroll 1
         for (int pass = 0; pass < 4; ++pass) {
@@ -153,9 +170,9 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
                 const uint32_t local = c[0] + c[1] + c[2] + c[3] + c[4] + c[5] + c[6] + c[7];
                 uint32_t incl = local;  // inclusive sum over lanes >= mine
 #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const uint32_t v = __shfl_down_sync(0xFFFFFFFFu, incl, d);
-                    if (lane + d < 32) incl += v;
+                for (int dist = 1; dist < 32; dist <<= 1) {
+                    const uint32_t v = __shfl_down_sync(0xFFFFFFFFu, incl, dist);
+                    if (lane + dist < 32) incl += v;
                 }
                 uint32_t above = incl - local;  // candidates in bins above this lane's
                 if (above < rank && rank <= incl) {
@@ -188,8 +205,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
         const int i = (wd << 5) + lane;
         const uint32_t key = keys[i];
         const bool r = (resv[wd] >> lane) & 1u;
-        const bool sure = i < n && (r || (p.k_fill > 0 && key > T));
-        const bool eq = i < n && !r && p.k_fill > 0 && key == T;
+        const bool sure = i < n && (r || (d.k_fill > 0 && key > T));
+        const bool eq = i < n && !r && d.k_fill > 0 && key == T;
         sure_cnt += __popc(__ballot_sync(0xFFFFFFFFu, sure));
         eq_cnt += __popc(__ballot_sync(0xFFFFFFFFu, eq));
     }
@@ -197,23 +214,23 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
     __syncthreads();
     uint32_t base = (lane < warp) ? warp_tot[lane] : 0u;  // n_warps <= 32
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) base += __shfl_xor_sync(0xFFFFFFFFu, base, d);
+    for (int dist = 16; dist > 0; dist >>= 1) base += __shfl_xor_sync(0xFFFFFFFFu, base, dist);
     uint32_t sure_before = base & 0xFFFFu, eq_before = base >> 16;
-    int32_t* seq = p.seq_idx ? p.seq_idx + (size_t)blockIdx.x * (p.seq_len - n + p.k) : nullptr;
     const uint32_t lt = (1u << lane) - 1u;
     for (int wd = w_begin; wd < w_end; ++wd) {
         const int i = (wd << 5) + lane;
         const uint32_t key = keys[i];
         const bool r = (resv[wd] >> lane) & 1u;
-        const bool sure = i < n && (r || (p.k_fill > 0 && key > T));
-        const bool eq = i < n && !r && p.k_fill > 0 && key == T;
+        const bool sure = i < n && (r || (d.k_fill > 0 && key > T));
+        const bool eq = i < n && !r && d.k_fill > 0 && key == T;
         const uint32_t sb = __ballot_sync(0xFFFFFFFFu, sure), eb = __ballot_sync(0xFFFFFFFFu, eq);
         const uint32_t my_eq_before = eq_before + __popc(eb & lt);
         const uint32_t my_sure_before = sure_before + __popc(sb & lt);
         if (sure || (eq && my_eq_before < need_eq)) {
             const uint32_t j = my_sure_before + min(my_eq_before, need_eq);
             out[j] = i;
-            if (seq) seq[p.vis_start + j] = p.vis_start + i;
+            if (seq) seq[vis_start + j] = vis_start + i;
+            if (flat) flat[j] = flat_base + i;
         }
         sure_before += __popc(sb);
         eq_before += __popc(eb);
@@ -221,10 +238,26 @@ __global__ void __launch_bounds__(1024) select_kernel(const SelectParams p)
     // fused sequence indices: text in front of the visual span keeps its positions, text
     // behind it moves up by the n - k dropped visual tokens
     if (seq) {
-        for (int j = tid; j < p.vis_start; j += nt) seq[j] = j;
-        const int s_out = p.seq_len - n + p.k;
-        for (int j = p.vis_start + p.k + tid; j < s_out; j += nt) seq[j] = j - p.k + n;
+        for (int j = tid; j < vis_start; j += nt) seq[j] = j;
+        const int s_out = seq_len - n + d.k;
+        for (int j = vis_start + d.k + tid; j < s_out; j += nt) seq[j] = j - d.k + n;
     }
+}
+
+__global__ void __launch_bounds__(1024) select_kernel(const __grid_constant__ SelectParams p)
+{
+    const SegShape& d = p.shape;
+    int32_t* seq = p.seq_idx ? p.seq_idx + (size_t)blockIdx.x * (p.seq_len - d.n + d.k) : nullptr;
+    select_block(d, p.scores + (size_t)blockIdx.x * d.n, p.keep_idx + (size_t)blockIdx.x * d.k, seq,
+                 p.seq_len, p.vis_start, nullptr, 0);
+}
+
+__global__ void __launch_bounds__(1024) select_ragged_kernel(const __grid_constant__ RaggedParams p)
+{
+    const SegShape& d = p.shape[blockIdx.x];
+    const int32_t out_off = p.out_off[blockIdx.x], score_off = p.score_off[blockIdx.x];
+    select_block(d, p.scores + score_off, p.keep_idx + out_off, nullptr, 0, 0,
+                 p.flat_idx ? p.flat_idx + out_off : nullptr, score_off);
 }
 
 // seq_idx[s, :] = text positions before the visual span, vis_start + kept visual indices,

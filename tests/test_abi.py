@@ -169,6 +169,29 @@ def test_select_large_validation(lib):
     assert lib.civic_status_string(7).decode() == "CIVIC_ERR_WORKSPACE"
 
 
+def test_select_ragged_validation(lib):
+    D = civic.SelectDesc
+    arr = lambda *ds: (D * len(ds))(*ds)
+    f = lambda descs, n, scores=0x100000, keep=0x200000, flat=0x300000: \
+        lib.civic_select_ragged(scores, n, descs, keep, flat, None)
+    before = lib.civic_launch_count()
+    good = arr(D(1, 4, 4, 2, 2, 1, 8), D(2, 3, 5, 1, 5, 0, 7))
+    assert f(good, 2, scores=None) == 1
+    assert f(good, 2, keep=None) == 1
+    assert f(arr(D(1, 4, 4, 2, 2, 1, 8), D(1, 4, 4, 2, 2, 1, 17)), 2) == 2
+    assert f(arr(D(1, 4, 4, 2, 2, 1, 8), D(1, 4, 4, 2, 2, 1, 3)), 2) == 3
+    assert f(arr(D(1, 4, 4, 2, 2, 1, 8), D(1, 0, 4, 2, 2, 1, 3)), 2) == 1
+    assert f(arr(D(1, 4, 4, 2, 2, 1, 8), D(1, 300, 300, 2, 2, 0, 3)), 2) == 5
+    assert f(good, 2, flat=0x200004) == 1  # flat_idx overlaps keep_idx
+    assert f(good, 2, keep=0x200002) == 4
+    assert f(None, 1) == 1
+    assert f(good, 0) == 0
+    assert f(arr(D(1, 4, 4, 2, 2, 0, 0), D(2, 3, 5, 1, 5, 0, 0)), 2) == 0  # nothing kept anywhere
+    assert lib.civic_launch_count() == before
+    assert lib.civic_floor_from_ratio(4, 4, 1, 5) == 4 and lib.civic_floor_from_ratio(4, 4, 0, 1) == 0
+    assert lib.civic_floor_from_ratio(4, 4, 1, 0) == -1
+
+
 def test_adjacent_calls_validation(lib):
     P = ctypes.c_void_p * 2
     ks, vs = P(0x100000, 0x200000), P(0x300000, 0x400000)

@@ -147,3 +147,82 @@ def test_workspace_errors_and_reuse():
     for _ in range(3):
         got = civic.civic_select_large(s, desc, workspace=ws)
         assert np.array_equal(got.cpu().numpy(), want)
+
+
+# ------------------------------------------------------------------ ragged batches
+
+def run_ragged(descs, parts):
+    scores = np.concatenate(parts).astype(np.float32)
+    want_keep, want_flat = O.select_ragged(scores, descs)
+    total_k = len(want_keep)
+    pad = 64
+    bufs = [torch.full((total_k + 2 * pad,), CANARY, dtype=torch.int32, device=DEV) for _ in range(2)]
+    keep, flat = (b[pad:pad + total_k] for b in bufs)
+    civic.civic_select_ragged(torch.from_numpy(scores).to(DEV), [civic.SelectDesc(*d) for d in descs],
+                              keep_idx=keep, flat_idx=flat)
+    assert np.array_equal(keep.cpu().numpy(), want_keep)
+    assert np.array_equal(flat.cpu().numpy(), want_flat)
+    for b in bufs:
+        host = b.cpu().numpy()
+        assert np.all(host[:pad] == CANARY) and np.all(host[pad + total_k:] == CANARY)
+    return scores, want_keep, want_flat
+
+
+def test_ragged_random_batches():
+    rng = np.random.default_rng(303)
+    for trial in range(25):
+        descs, parts = [], []
+        for _ in range(int(rng.integers(1, 9))):
+            t, h, w = int(rng.integers(1, 4)), int(rng.integers(1, 40)), int(rng.integers(1, 40))
+            rh, rw = int(rng.integers(1, min(h, 8) + 1)), int(rng.integers(1, min(w, 8) + 1))
+            m = int(rng.integers(0, 3))
+            n = t * h * w
+            k = int(rng.integers(O.reserved_count(t, h, w, rh, rw, m), n + 1))
+            descs.append((t, h, w, rh, rw, m, k))
+            parts.append(rng.integers(0, 6, n) if trial % 2 else rng.random(n))
+        run_ragged(descs, parts)
+
+
+def test_ragged_mixed_workloads_compacts_in_one_call():
+    """Images and a video of the benchmark shapes in one batch, budgets differing per segment
+    (one of them from a Min-Keep-Ratio floor); the flat indices compact the whole batch at once."""
+    m_ratio = civic.floor_from_ratio(4, 4, 1, 5)
+    assert m_ratio == O.floor_from_ratio(4, 4, 1, 5) == 4
+    shapes = [(W.C1, 65, 1), (W.C2, 341, 1), (W.C4, 1045, 1), (W.C5_THIRD, 1500, m_ratio), (W.C2, 0, 0),
+              (W.C2, 512, 2)]
+    descs = [(wl.t, wl.h, wl.w, wl.region_h, wl.region_w, m, k) for wl, k, m in shapes]
+    parts = [W.scores(wl, seg=i % wl.n_seg) for i, (wl, _, _) in enumerate(shapes)]
+    scores, keep, flat = run_ragged(descs, parts)
+    total_n, total_k = len(scores), len(keep)
+    rng = np.random.default_rng(1)
+    hidden = rng.integers(-30000, 30000, (1, total_n, 64)).astype(np.int16)
+    pos = rng.integers(0, 99, (1, total_n, 3)).astype(np.int32)
+    h_out, p_out = civic.civic_compact(torch.from_numpy(hidden).to(DEV), torch.from_numpy(pos).to(DEV),
+                                       torch.from_numpy(flat[None]).to(DEV))
+    want_h, want_p = O.compact(hidden, pos, flat[None])
+    assert np.array_equal(h_out.cpu().numpy(), want_h) and np.array_equal(p_out.cpu().numpy(), want_p)
+    assert h_out.shape == (1, total_k, 64)
+
+
+def test_ragged_more_segments_than_one_launch():
+    rng = np.random.default_rng(304)
+    descs = [(1, 6, 7, 2, 3, 1, int(rng.integers(9, 42))) for _ in range(150)]
+    run_ragged(descs, [rng.random(42) for _ in descs])
+
+
+def test_floor_from_ratio_matches_the_oracle():
+    for rh in range(1, 7):
+        for rw in range(1, 7):
+            for den in range(1, 9):
+                for num in range(0, den + 1):
+                    assert civic.floor_from_ratio(rh, rw, num, den) == O.floor_from_ratio(rh, rw, num, den)
+    assert civic.floor_from_ratio(4, 4, 3, 2) == -1
+    # Table 2's ratios on the benchmark's 4x4 tiles, run through the selection
+    wl = W.C5_HALF
+    s = W.scores(wl)
+    for num, den in [(0, 1), (1, 5), (1, 2)]:
+        m = civic.floor_from_ratio(wl.region_h, wl.region_w, num, den)
+        k = max(wl.k, m * wl.n_regions)
+        want = O.select(s, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, m, k)
+        got = civic.civic_select(torch.from_numpy(s).to(DEV), civic.SelectDesc(wl.t, wl.h, wl.w, wl.region_h, wl.region_w, m, k))
+        assert np.array_equal(got.cpu().numpy(), want)
