@@ -118,6 +118,39 @@ civic_status_t civic_select_large(const float* scores, int32_t n_seg, const civi
                                   int32_t chunk_tokens, void* stream);
 
 /*
+ * civic_select_large_static -- civic_select_large for callers that cannot allocate device memory.
+ *
+ * The paper has no counterpart to this call; it exists for the sake of its callers.  Code that
+ * runs where cudaMalloc is off limits -- inside a serving engine that handed all device memory
+ * to its own pool at start-up, in a plugin that owns no allocator, on a path that must not
+ * touch the allocator because a latency budget or a memory cap forbids it -- has nowhere to get
+ * the scratch buffer civic_select_large asks for.  This variant computes the same selection
+ * with its scratch in a fixed array built into the library, so the caller passes inputs and
+ * the output only.  The call allocates nothing, frees nothing and calls no allocating routine.
+ *
+ * Limits and sharing
+ *   - The built-in scratch is civic_select_static_scratch_bytes() = 2 MiB, held by every GPU
+ *     that loads the library until the process exits.  A shape whose
+ *     civic_select_workspace_bytes(desc, n_seg, chunk_tokens) exceeds it is rejected with
+ *     CIVIC_ERR_WORKSPACE and nothing is launched (2 MiB covers, for example, one video of about
+ *     two million tokens or eight of 200 000).
+ *   - All calls on one GPU share that one array, and it still holds the previous call's
+ *     contents: the call clears the part that must start at zero itself.  Calls in ONE stream
+ *     run one after the other and are safe; two calls of one process that can overlap on the
+ *     GPU (different streams, whichever host threads issue them) race on the scratch and give
+ *     wrong results.  Use civic_select_large with separate workspaces there.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current, as for every call).  Make that first call before starting any stream capture.
+ *
+ * Arguments, result and the other errors are those of civic_select_large.
+ */
+civic_status_t civic_select_large_static(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                                         int32_t* keep_idx, int32_t chunk_tokens, void* stream);
+
+/* Size in bytes of the scratch built into the library for civic_select_large_static. */
+size_t civic_select_static_scratch_bytes(void);
+
+/*
  * civic_select_ragged -- civic_select for a batch whose segments differ in shape and budget.
  *
  * Paper: as civic_select; instance-adaptive token budgets and mixed image/video batches are the

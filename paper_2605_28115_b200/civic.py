@@ -28,7 +28,8 @@ EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "c
            "civic_launch_count", "civic_select_seq", "civic_set_programmatic_launch",
            "civic_compact_kv_heads", "civic_compact_kv_paged", "civic_merge_embeddings",
            "civic_compact_pos_planes", "civic_select_large", "civic_select_workspace_bytes",
-           "civic_select_ragged", "civic_floor_from_ratio")
+           "civic_select_ragged", "civic_floor_from_ratio",
+           "civic_select_large_static", "civic_select_static_scratch_bytes")
 
 
 class CivicError(RuntimeError):
@@ -99,6 +100,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_select_ragged.restype = ctypes.c_int
     lib.civic_floor_from_ratio.argtypes = [i32, i32, i32, i32]
     lib.civic_floor_from_ratio.restype = i32
+    lib.civic_select_large_static.argtypes = [vp, i32, ctypes.POINTER(SelectDesc), vp, i32, vp]
+    lib.civic_select_large_static.restype = ctypes.c_int
+    lib.civic_select_static_scratch_bytes.argtypes = []
+    lib.civic_select_static_scratch_bytes.restype = sz
     _lib = lib
     return lib
 
@@ -213,6 +218,28 @@ def civic_select_large(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optiona
             workspace.numel(), chunk_tokens)
     with torch.cuda.device(dev):
         _check(load().civic_select_large(*args, _stream_ptr(stream)), "civic_select_large")
+    return keep_idx
+
+
+def select_static_scratch_bytes() -> int:
+    return int(load().civic_select_static_scratch_bytes())
+
+
+def civic_select_large_static(scores: torch.Tensor, desc: SelectDesc, keep_idx: torch.Tensor,
+                              chunk_tokens: int = 0, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """civic_select_large with the scratch built into the library (at most
+    select_static_scratch_bytes()): for callers that may not allocate device memory, so the
+    output tensor is required and nothing is allocated here either.  Calls that can overlap on
+    one GPU race on the shared scratch; keep them in one stream."""
+    if scores.dim() != 2 or scores.shape[1] != desc.t * desc.h * desc.w:
+        raise ValueError("scores must be [n_seg, t*h*w]")
+    n_seg = scores.shape[0]
+    if tuple(keep_idx.shape) != (n_seg, desc.k):
+        raise ValueError("keep_idx must be [n_seg, k]")
+    args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
+            _dev_ptr(keep_idx, "keep_idx", torch.int32), chunk_tokens)
+    with torch.cuda.device(_device_of(scores)):
+        _check(load().civic_select_large_static(*args, _stream_ptr(stream)), "civic_select_large_static")
     return keep_idx
 
 

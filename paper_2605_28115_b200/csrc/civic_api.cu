@@ -279,6 +279,33 @@ civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_selec
     return CIVIC_OK;
 }
 
+// ---- civic_select_large without any caller-provided or allocated scratch -------------------
+//
+// The scratch of the many-block selection lives in this fixed array inside the library's device
+// image: every GPU that loads the library holds it until the process exits.  In host code the
+// name g_static_scratch is only a handle for the runtime, not an address a kernel may use;
+// its device address is looked up with cudaGetSymbolAddress, once per device.
+constexpr size_t kStaticScratchBytes = (size_t)2 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of the static scratch on the CURRENT device.
+civic_status_t static_scratch_address(char** out)
+{
+    static std::atomic<char*> cached[64];
+    int dev = -1;
+    CIVIC_CUDA_TRY(cudaGetDevice(&dev));
+    const bool cacheable = dev >= 0 && dev < 64;
+    char* ptr = cacheable ? cached[dev].load(std::memory_order_acquire) : nullptr;
+    if (!ptr) {
+        void* sym = nullptr;
+        CIVIC_CUDA_TRY(cudaGetSymbolAddress(&sym, g_static_scratch));
+        ptr = (char*)sym;
+        if (cacheable) cached[dev].store(ptr, std::memory_order_release);
+    }
+    *out = ptr;
+    return CIVIC_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -351,6 +378,35 @@ civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_
         return civic_seq_indices(keep_idx, n_seq, 0, seq_len, vis_start, (int32_t)n, seq_idx, stream);
     }
     return select_impl(scores, n_seq, desc, keep_idx, seq_idx, seq_len, vis_start, stream);
+}
+
+size_t civic_select_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+civic_status_t civic_select_large_static(const float* scores, int32_t n_seg, const civic_select_desc_t* desc,
+                                         int32_t* keep_idx, int32_t chunk_tokens, void* stream)
+{
+    if (!desc || n_seg < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n_res = reserved_count(*desc);
+    if (n_res < 0) return CIVIC_ERR_INVALID_ARG;
+    const int64_t n = (int64_t)desc->t * desc->h * desc->w;
+    if (n > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (desc->k < 0 || desc->k > n) return CIVIC_ERR_K_RANGE;
+    if (n_res > desc->k) return CIVIC_ERR_FLOOR_EXCEEDS_K;
+    LargePlan pl;
+    const civic_status_t st = plan_large(*desc, n_seg, chunk_tokens, pl);
+    if (st != CIVIC_OK) return st;
+    if (pl.total > kStaticScratchBytes) return CIVIC_ERR_WORKSPACE;  // beyond the built-in scratch
+    if (n_seg == 0 || desc->k == 0) return CIVIC_OK;
+    if (!scores || !keep_idx) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(scores, 4) || !aligned(keep_idx, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (overlaps(scores, (size_t)n_seg * n * 4, keep_idx, (size_t)n_seg * desc->k * 4))
+        return CIVIC_ERR_INVALID_ARG;
+    char* scratch = nullptr;
+    const civic_status_t st2 = static_scratch_address(&scratch);
+    if (st2 != CIVIC_OK) return st2;
+    // the histograms and scalars inside the scratch are cleared by launch_large on every call
+    return launch_large(scores, n_seg, *desc, keep_idx, scratch, pl, (int32_t)(desc->k - n_res),
+                        (cudaStream_t)stream);
 }
 
 civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civic_select_desc_t* descs,
