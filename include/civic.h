@@ -318,6 +318,40 @@ civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, in
                                         int32_t seq_len, const int32_t* seq_idx, int32_t s_out,
                                         int32_t* pos_out, void* stream);
 
+/*
+ * civic_anchor_aggregate -- compact visual aggregation, the step that produces the compact
+ * visual sequence (and a per-token importance score) upstream of the selection.
+ *
+ * Paper: Eq. 8 (Section 3.3):  K_0 = Norm(LN(X_0)),  Q_A = Norm(LN(A)),
+ *        W_A = softmax(Q_A K_0^T / tau) over the dense tokens,  Z_0 = W_A X_0.
+ * LN is layer normalisation over the features without learned scale or shift (eps 1e-5), Norm
+ * the l2 normalisation of every row (eps 1e-12).  Both contractions run on the tensor cores in
+ * bf16 with fp32 accumulation; W_A is rounded to bf16 before the second one, and its rows are
+ * normalised by the sum of the rounded values, so they still add up to one.
+ *
+ * x0             dev  bf16 [n_img, t_e, d_v] dense patch embeddings, 16-byte aligned
+ * anchors        dev  fp32 [m_e, d_v], shared by all images
+ * tau            aggregation temperature, >= 0.025 (smaller: CIVIC_ERR_UNSUPPORTED)
+ * z0             dev  bf16 [n_img, m_e, d_v], written
+ * token_mass     dev  fp32 [n_img, t_e] or NULL, written: column sums of W_A, i.e. how much of
+ *                the anchors' attention each dense token receives -- usable as the `scores` of
+ *                civic_select
+ * workspace      dev  scratch of civic_anchor_aggregate_workspace_bytes(...) bytes, 256-byte
+ *                aligned (holds Q_A, the token statistics and W_A's unnormalised bf16 form)
+ * device_status  dev  int32, written: 0, or a non-zero code if a wait inside a kernel ran into
+ *                its time limit (the kernels then stop cleanly and the outputs are invalid).
+ *                Read it after synchronising the stream.
+ * d_v must be a multiple of 64 (CIVIC_ERR_UNSUPPORTED otherwise); t_e and m_e are arbitrary.
+ * Inputs must be finite.  Five launches (six with token_mass).
+ */
+civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
+                                      int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
+                                      void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                      void* stream);
+
+/* Scratch bytes civic_anchor_aggregate needs; 0 if the shape is invalid or unsupported. */
+size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d_v);
+
 /* Static, human-readable name of a status. */
 const char* civic_status_string(civic_status_t status);
 

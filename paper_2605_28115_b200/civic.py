@@ -29,7 +29,8 @@ EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "c
            "civic_compact_kv_heads", "civic_compact_kv_paged", "civic_merge_embeddings",
            "civic_compact_pos_planes", "civic_select_large", "civic_select_workspace_bytes",
            "civic_select_ragged", "civic_floor_from_ratio",
-           "civic_select_large_static", "civic_select_static_scratch_bytes")
+           "civic_select_large_static", "civic_select_static_scratch_bytes",
+           "civic_anchor_aggregate", "civic_anchor_aggregate_workspace_bytes")
 
 
 class CivicError(RuntimeError):
@@ -104,6 +105,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_select_large_static.restype = ctypes.c_int
     lib.civic_select_static_scratch_bytes.argtypes = []
     lib.civic_select_static_scratch_bytes.restype = sz
+    lib.civic_anchor_aggregate.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, sz, vp, vp]
+    lib.civic_anchor_aggregate.restype = ctypes.c_int
+    lib.civic_anchor_aggregate_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    lib.civic_anchor_aggregate_workspace_bytes.restype = sz
     _lib = lib
     return lib
 
@@ -540,3 +545,41 @@ def civic_compact_pos_planes(pos: torch.Tensor, seq_idx: torch.Tensor,
     with torch.cuda.device(_device_of(seq_idx, pos)):
         _check(load().civic_compact_pos_planes(*args, _stream_ptr(stream)), "civic_compact_pos_planes")
     return pos_out
+
+
+def anchor_aggregate_workspace_bytes(n_img: int, t_e: int, m_e: int, d_v: int) -> int:
+    return int(load().civic_anchor_aggregate_workspace_bytes(n_img, t_e, m_e, d_v))
+
+
+def civic_anchor_aggregate(x0: torch.Tensor, anchors: torch.Tensor, tau: float,
+                           z0: Optional[torch.Tensor] = None, token_mass: Optional[torch.Tensor] = None,
+                           want_mass: bool = True, workspace: Optional[torch.Tensor] = None,
+                           device_status: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None):
+    """Eq. 8: x0 bf16 [n_img, t_e, d_v], anchors fp32 [m_e, d_v] -> (z0 bf16 [n_img, m_e, d_v],
+    token mass fp32 [n_img, t_e] or None, device_status int32 [1]: 0 after a clean run)."""
+    if x0.dim() != 3 or anchors.dim() != 2 or anchors.shape[1] != x0.shape[2]:
+        raise ValueError("x0 must be [n_img, t_e, d_v] and anchors [m_e, d_v]")
+    n_img, t_e, d_v = x0.shape
+    m_e = anchors.shape[0]
+    dev = _device_of(x0)
+    if z0 is None:
+        z0 = torch.empty((n_img, m_e, d_v), dtype=torch.bfloat16, device=dev)
+    elif tuple(z0.shape) != (n_img, m_e, d_v):
+        raise ValueError("z0 must be [n_img, m_e, d_v]")
+    if token_mass is None and want_mass:
+        token_mass = torch.empty((n_img, t_e), dtype=torch.float32, device=dev)
+    elif token_mass is not None and tuple(token_mass.shape) != (n_img, t_e):
+        raise ValueError("token_mass must be [n_img, t_e]")
+    if workspace is None:
+        workspace = torch.empty(max(anchor_aggregate_workspace_bytes(n_img, t_e, m_e, d_v), 256),
+                                dtype=torch.uint8, device=dev)
+    if device_status is None:
+        device_status = torch.empty((1,), dtype=torch.int32, device=dev)
+    args = (_dev_ptr(x0, "x0", torch.bfloat16), _dev_ptr(anchors, "anchors", torch.float32), n_img, t_e, m_e, d_v,
+            ctypes.c_float(tau), _dev_ptr(z0, "z0", torch.bfloat16), _dev_ptr(token_mass, "token_mass", torch.float32),
+            _dev_ptr(workspace, "workspace", torch.uint8), workspace.numel(),
+            _dev_ptr(device_status, "device_status", torch.int32))
+    with torch.cuda.device(dev):
+        _check(load().civic_anchor_aggregate(*args, _stream_ptr(stream)), "civic_anchor_aggregate")
+    return z0, token_mass, device_status

@@ -1,0 +1,519 @@
+// Compact visual aggregation (Eq. 8 of the paper) on the 5th-generation tensor cores:
+//
+//     K_0 = Norm(LN(X_0)),  Q_A = Norm(LN(A)),  W_A = softmax(Q_A K_0^T / tau),  Z_0 = W_A X_0
+//
+// Algebra used (exact in real arithmetic): LN's 1/sqrt(var + eps) cancels under the l2
+// normalisation, so K_0[i] = r_i (x_i - mu_i 1) with r_i = 1 / ||x_i - mu_i 1||, and
+//     Q_A[m] . K_0[i] = r_i (Q_A[m] . x_i  -  mu_i * sum_j Q_A[m, j]).
+// The first contraction therefore runs on the RAW tokens; normalising them costs two scalars per
+// token (mu_i, r_i) that the epilogue applies, and one scalar per anchor (the exact sum of its
+// bf16-rounded row).  Cosines are bounded by 1, so the softmax needs no running maximum:
+// P = exp((s - 1) / tau) cannot overflow and, for tau >= 0.025, cannot underflow bf16.
+//
+// Kernels
+//   anchor_prep_kernel      A (fp32) -> Q_A (bf16) and the row sums of the rounded values
+//   token_stats_kernel      X_0 (bf16) -> (mu_i, r_i), one warp per token, HBM-bound
+//   aggregate_scores_kernel tcgen05 GEMM  S = Q_A X_0^T  (both operands K-major), epilogue
+//                           P = exp((r (S - mu qsum) - 1) / tau) as bf16 + partial row sums
+//   aggregate_values_kernel tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major)
+//   token_mass_kernel       column sums of W_A (per-token importance), HBM-bound
+//
+// GEMM skeleton (both): 192 threads.  Warp 0 = TMA producer (one elected lane), warp 1 = TMEM
+// allocation + MMA issue (one elected lane), warps 2..5 = epilogue (each reads its own quarter
+// of the 128 TMEM lanes).  Operand tiles arrive by cp.async.bulk.tensor with 128-byte swizzle
+// into a ring of stages guarded by full/empty mbarriers; accumulators live in TMEM.
+// Every wait is bounded: on a time-out the thread raises the kernel's error word, the block
+// stops issuing work, waits (bounded) for its copies in flight, frees its TMEM and returns.
+#pragma once
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "pdl.cuh"
+
+namespace civic {
+
+constexpr int kAggThreads = 192;
+constexpr int kAggBM = 128;           // anchors per tile (TMEM lanes)
+constexpr int kAggBK = 64;            // 64 bf16 = one 128-byte swizzle row
+constexpr int kScoresBN = 128;        // tokens per tile of the first GEMM
+constexpr int kScoresStages = 3;      // 3 x 32 KB: two blocks fit one SM
+constexpr int kValuesStages = 4;
+constexpr unsigned long long kWaitLimitCycles = 1ull << 31;  // about a second
+
+enum AggError { kAggOk = 0, kAggTimeoutFull = 1, kAggTimeoutEmpty = 2, kAggTimeoutAcc = 3 };
+
+// ----------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the block has been told to stop (*abort != 0) or the limit
+// ran out, in which case it also raises *abort and records `code` in the kernel's error word.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* error, int code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if ((unsigned long long)(clock64() - t0) > kWaitLimitCycles) {
+            *abort = 1;
+            atomicCAS(error, 0, code);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void fence_barrier_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols)  // whole warp
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)  // whole warp
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] B[smem], bf16 operands, fp32 accumulator, one CTA.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.u32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 consecutive fp32 columns of this warp's 32 TMEM lanes: thread t gets lane (base + t).
+__device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory operand descriptor, 128-byte swizzle, tile base 1024-byte aligned.
+//   K-major  (rows of 64 bf16 = 128 B): 8-row groups 1024 B apart (stride offset); the leading
+//             offset is unused with swizzling (set to one 16-byte unit).
+//   MN-major (the 64 contiguous elements run along M or N): 8 K-rows of 128 B form a group,
+//             groups 1024 B apart (stride offset); the next 64 elements along M/N start
+//             `leading_bytes` further on.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t leading_bytes, uint32_t stride_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((leading_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;  // descriptor version of this architecture
+    d |= 2ull << 61;  // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n; b_mn_major = 1 when B's
+// contiguous dimension is N.
+__host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major)
+{
+    return (1u << 4)                      // accumulator fp32
+           | (1u << 7) | (1u << 10)       // A, B bf16
+           | ((uint32_t)b_mn_major << 16) // B major
+           | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kAggBM >> 4) << 24);
+}
+
+// ----------------------------------------------------------------------------- small kernels
+
+// Q_A = Norm(LN(A)) rounded to bf16, and qsum[m] = sum of the ROUNDED row (what the tensor
+// core will really multiply the token mean with).  One warp per anchor; rows of any length.
+__global__ void anchor_prep_kernel(const float* __restrict__ anchors, int m_e, int d_v, float ln_eps, float norm_eps,
+                                   __nv_bfloat16* __restrict__ q, float* __restrict__ qsum)
+{
+    wait_for_prior_kernels();
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= m_e) return;
+    const float* a = anchors + (size_t)warp * d_v;
+    float s = 0.f;
+    for (int j = lane; j < d_v; j += 32) s += a[j];
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+    const float mean = s / d_v;
+    float ss = 0.f;
+    for (int j = lane; j < d_v; j += 32) { const float c = a[j] - mean; ss += c * c; }
+    for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, d);
+    const float inv_std = rsqrtf(ss / d_v + ln_eps);
+    const float norm = sqrtf(ss) * inv_std;  // l2 norm of the layer-normalised row
+    const float scale = inv_std / fmaxf(norm, norm_eps);
+    float rounded_sum = 0.f;
+    for (int j = lane; j < d_v; j += 32) {
+        const __nv_bfloat16 v = __float2bfloat16_rn((a[j] - mean) * scale);
+        q[(size_t)warp * d_v + j] = v;
+        rounded_sum += __bfloat162float(v);
+    }
+    for (int d = 16; d > 0; d >>= 1) rounded_sum += __shfl_xor_sync(0xFFFFFFFFu, rounded_sum, d);
+    if (lane == 0) qsum[warp] = rounded_sum;
+}
+
+// (mu_i, r_i) per token: K_0[i] = r_i (x_i - mu_i).  One warp per token row of d_v bf16
+// (d_v a multiple of 8: 16-byte loads).  r_i = 0 for a token whose features are all equal.
+__global__ void token_stats_kernel(const __nv_bfloat16* __restrict__ x, long long n_tokens, int d_v, float ln_eps,
+                                   float norm_eps, float2* __restrict__ stats)
+{
+    wait_for_prior_kernels();
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= n_tokens) return;
+    const uint4* row = reinterpret_cast<const uint4*>(x + warp * d_v);
+    const int vecs = d_v >> 3;
+    float s = 0.f, s2 = 0.f;  // shifted sums keep the variance accurate: shift by the row's first element
+    const float shift = __bfloat162float(x[warp * d_v]);
+    for (int v = lane; v < vecs; v += 32) {
+        const uint4 u = __ldg(row + v);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            const float a = f.x - shift, b = f.y - shift;
+            s += a + b;
+            s2 += a * a + b * b;
+        }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+        s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, d);
+    }
+    if (lane == 0) {
+        const float mean_shifted = s / d_v;
+        const float ss = fmaxf(s2 - s * mean_shifted, 0.f);  // sum (x - mu)^2
+        const float inv_std = rsqrtf(ss / d_v + ln_eps);
+        const float norm = sqrtf(ss) * inv_std;
+        const float r = ss > 0.f ? inv_std / fmaxf(norm, norm_eps) : 0.f;
+        stats[warp] = make_float2(mean_shifted + shift, r);
+    }
+}
+
+// ----------------------------------------------------------------------------- GEMM 1: scores
+
+struct ScoresParams {
+    const float2* stats;    // [n_img, t_e]  (mu, r)
+    const float* qsum;      // [m_e]
+    __nv_bfloat16* p;       // [n_img, m_e, t_ld]
+    float* lpart;           // [n_img, m_e, n_tiles_t] partial row sums of the rounded P
+    int* error;             // kernel error word (0 = fine)
+    int32_t n_img, m_e, t_e, d_v, t_ld, n_tiles_t;
+    float inv_tau_log2e;    // log2(e) / tau
+};
+
+struct alignas(1024) ScoresSmem {
+    __nv_bfloat16 a[kScoresStages][kAggBM * kAggBK];     // Q tile: 128 rows x 128 B
+    __nv_bfloat16 b[kScoresStages][kScoresBN * kAggBK];  // X tile: 128 tokens x 128 B
+    float2 stats[kScoresBN];
+    uint64_t full[kScoresStages], empty[kScoresStages], acc_full;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__global__ void __launch_bounds__(kAggThreads) aggregate_scores_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                       const __grid_constant__ CUtensorMap map_x,
+                                                                       const ScoresParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    ScoresSmem& sm = *reinterpret_cast<ScoresSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kAggBM, n0 = blockIdx.y * kScoresBN, img = blockIdx.z;
+    const int k_steps = p.d_v / kAggBK;
+    volatile int* abort = &sm.abort;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kScoresStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        mbar_init(&sm.acc_full, 1);
+        sm.abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&sm.tmem_base, kScoresBN);
+    wait_for_prior_kernels();
+    if (warp >= 2) {  // token statistics of this tile's columns
+        const int c = threadIdx.x - 64;
+        const int tok = n0 + c;
+        sm.stats[c] = tok < p.t_e ? p.stats[(size_t)img * p.t_e + tok] : make_float2(0.f, 0.f);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_acc = sm.tmem_base;
+    const bool stop = *p.error != 0;  // an earlier block of this launch already failed
+
+    if (warp == 0 && lane == 0 && !stop) {
+        // ---- producer: one box of Q and one of X per stage
+        int issued = 0;
+        for (int k = 0; k < k_steps; ++k, ++issued) {
+            const int s = k % kScoresStages;
+            if (k >= kScoresStages &&
+                !mbar_wait(&sm.empty[s], ((k / kScoresStages) - 1) & 1, abort, p.error, kAggTimeoutEmpty))
+                break;
+            mbar_expect_tx(&sm.full[s], (kAggBM + kScoresBN) * kAggBK * 2);
+            tma_load_2d(sm.a[s], &map_q, k * kAggBK, m0, &sm.full[s]);
+            tma_load_3d(sm.b[s], &map_x, k * kAggBK, n0, img, &sm.full[s]);
+        }
+        if (*abort) {  // let the copies already in flight land before the block goes away
+            for (int k = max(0, issued - kScoresStages); k < issued; ++k) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&sm.full[k % kScoresStages], (k / kScoresStages) & 1) &&
+                       (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
+            }
+        }
+    } else if (warp == 1 && lane == 0 && !stop) {
+        // ---- MMA issue: 4 instructions of K = 16 per stage
+        constexpr uint32_t idesc = umma_idesc(kScoresBN, 0);
+        bool ok = true;
+        for (int k = 0; k < k_steps && ok; ++k) {
+            const int s = k % kScoresStages;
+            ok = mbar_wait(&sm.full[s], (k / kScoresStages) & 1, abort, p.error, kAggTimeoutFull);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
+#pragma unroll
+            for (int kk = 0; kk < kAggBK / 16; ++kk)
+                umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), umma_desc(b0 + kk * 32, 16, 1024), idesc,
+                          (k | kk) != 0);
+            umma_commit(&sm.empty[s]);  // frees the stage once these MMAs have read it
+        }
+        if (ok) umma_commit(&sm.acc_full);
+    } else if (warp >= 2 && !stop) {
+        // ---- epilogue: thread = one anchor row, 4 chunks of 32 token columns
+        const int quarter = warp & 3;  // TMEM lane quarter this warp may read
+        const int m = m0 + quarter * 32 + lane;
+        // tcgen05.ld is warp-collective: the whole warp goes on, or none of it
+        if (__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full, 0, abort, p.error, kAggTimeoutAcc))) {
+            tc_fence_after_sync();
+            const float qs = m < p.m_e ? p.qsum[m] : 0.f;
+            float row_sum = 0.f;
+            __nv_bfloat16* out = p.p + ((size_t)img * p.m_e + (m < p.m_e ? m : 0)) * p.t_ld + n0;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kScoresBN; c0 += 32) {
+                uint32_t acc[32];
+                tmem_load_32cols(tmem_acc + ((uint32_t)(quarter * 32) << 16) + c0, acc);
+                uint32_t packed[16];
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                    float v[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float2 st = sm.stats[c0 + c + e];
+                        const float cosine = st.y * (__uint_as_float(acc[c + e]) - st.x * qs);
+                        v[e] = (n0 + c0 + c + e) < p.t_e ? exp2f((cosine - 1.f) * p.inv_tau_log2e) : 0.f;
+                    }
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[0], v[1]);
+                    row_sum += __low2float(h) + __high2float(h);
+                    packed[c >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                if (m < p.m_e) {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4)  // 8 columns per 16-byte store; t_ld is a multiple of 8
+                        if (n0 + c0 + q4 * 8 < p.t_ld)
+                            *reinterpret_cast<uint4*>(out + c0 + q4 * 8) =
+                                make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
+                }
+            }
+            if (m < p.m_e) p.lpart[((size_t)img * p.m_e + m) * p.n_tiles_t + blockIdx.y] = row_sum;
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_acc, kScoresBN);
+    }
+}
+
+// ----------------------------------------------------------------------------- GEMM 2: values
+
+struct ValuesParams {
+    const float* lpart;   // [n_img, m_e, n_tiles_t]
+    __nv_bfloat16* z;     // [n_img, m_e, d_v]
+    float* inv_l;         // [n_img, m_e] written by the blocks of the first feature tile
+    int* error;
+    int32_t n_img, m_e, t_e, d_v, n_tiles_t;
+};
+
+template <int BN>
+struct alignas(1024) ValuesSmem {
+    __nv_bfloat16 a[kValuesStages][kAggBM * kAggBK];  // P tile: 128 anchors x 64 tokens (K-major)
+    __nv_bfloat16 b[kValuesStages][kAggBK * BN];      // X tile: BN/64 blocks of 64 tokens x 128 B (MN-major)
+    uint64_t full[kValuesStages], empty[kValuesStages], acc_full;
+    uint32_t tmem_base;
+    int abort;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kAggThreads) aggregate_values_kernel(const __grid_constant__ CUtensorMap map_p,
+                                                                       const __grid_constant__ CUtensorMap map_x,
+                                                                       const ValuesParams p)
+{
+    constexpr uint32_t kTmemCols = BN <= 128 ? 128 : 256;
+    extern __shared__ uint8_t smem_raw[];
+    using Smem = ValuesSmem<BN>;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kAggBM, n0 = blockIdx.y * BN, img = blockIdx.z;
+    const int k_steps = (p.t_e + kAggBK - 1) / kAggBK;
+    volatile int* abort = &sm.abort;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kValuesStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        mbar_init(&sm.acc_full, 1);
+        sm.abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&sm.tmem_base, kTmemCols);
+    wait_for_prior_kernels();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_acc = sm.tmem_base;
+    const bool stop = *p.error != 0;
+
+    if (warp == 0 && lane == 0 && !stop) {
+        int issued = 0;
+        for (int k = 0; k < k_steps; ++k, ++issued) {
+            const int s = k % kValuesStages;
+            if (k >= kValuesStages &&
+                !mbar_wait(&sm.empty[s], ((k / kValuesStages) - 1) & 1, abort, p.error, kAggTimeoutEmpty))
+                break;
+            mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
+            tma_load_3d(sm.a[s], &map_p, k * kAggBK, m0, img, &sm.full[s]);
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)  // 64 features x 64 tokens per box
+                tma_load_3d(sm.b[s] + j * (kAggBK * 64), &map_x, n0 + j * 64, k * kAggBK, img, &sm.full[s]);
+        }
+        if (*abort) {
+            for (int k = max(0, issued - kValuesStages); k < issued; ++k) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&sm.full[k % kValuesStages], (k / kValuesStages) & 1) &&
+                       (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
+            }
+        }
+    } else if (warp == 1 && lane == 0 && !stop) {
+        constexpr uint32_t idesc = umma_idesc(BN, 1);
+        bool ok = true;
+        for (int k = 0; k < k_steps && ok; ++k) {
+            const int s = k % kValuesStages;
+            ok = mbar_wait(&sm.full[s], (k / kValuesStages) & 1, abort, p.error, kAggTimeoutFull);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
+#pragma unroll
+            for (int kk = 0; kk < kAggBK / 16; ++kk)  // A: 32 B per K step; B: 16 token rows of 128 B
+                umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024),
+                          umma_desc(b0 + kk * 2048, kAggBK * 128, 1024), idesc, (k | kk) != 0);
+            umma_commit(&sm.empty[s]);
+        }
+        if (ok) umma_commit(&sm.acc_full);
+    } else if (warp >= 2 && !stop) {
+        const int quarter = warp & 3;
+        const int m = m0 + quarter * 32 + lane;
+        // 1 / l[m]: the row's partial sums from the first GEMM
+        float l = 0.f;
+        if (m < p.m_e) {
+            const float* lp = p.lpart + ((size_t)img * p.m_e + m) * p.n_tiles_t;
+            for (int t = 0; t < p.n_tiles_t; ++t) l += lp[t];
+        }
+        const float inv_l = l > 0.f ? 1.f / l : 0.f;
+        if (m < p.m_e && blockIdx.y == 0) p.inv_l[(size_t)img * p.m_e + m] = inv_l;
+        if (__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full, 0, abort, p.error, kAggTimeoutAcc))) {
+            tc_fence_after_sync();
+            __nv_bfloat16* out = p.z + ((size_t)img * p.m_e + (m < p.m_e ? m : 0)) * p.d_v + n0;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t acc[32];
+                tmem_load_32cols(tmem_acc + ((uint32_t)(quarter * 32) << 16) + c0, acc);
+                if (m < p.m_e) {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        if (n0 + c0 + q4 * 8 < p.d_v) {  // d_v is a multiple of 8
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h =
+                                    __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv_l,
+                                                          __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv_l);
+                                w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                            }
+                            *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_acc, kTmemCols);
+    }
+}
+
+// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m].  Thread per token, coalesced rows.
+__global__ void token_mass_kernel(const __nv_bfloat16* __restrict__ p, const float* __restrict__ inv_l, int m_e, int t_e,
+                                  int t_ld, float* __restrict__ mass)
+{
+    wait_for_prior_kernels();
+    const int img = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= t_e) return;
+    const __nv_bfloat16* col = p + (size_t)img * m_e * t_ld + i;
+    const float* il = inv_l + (size_t)img * m_e;
+    float acc = 0.f;
+    for (int m = 0; m < m_e; ++m) acc += __bfloat162float(col[(size_t)m * t_ld]) * __ldg(il + m);
+    mass[(size_t)img * t_e + i] = acc;
+}
+
+}  // namespace civic

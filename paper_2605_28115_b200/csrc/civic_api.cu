@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstring>
 
+#include "aggregate.cuh"
 #include "gather.cuh"
 #include "select.cuh"
 #include "select_large.cuh"
@@ -306,6 +307,92 @@ civic_status_t static_scratch_address(char** out)
     return CIVIC_OK;
 }
 
+// ---- compact visual aggregation (Eq. 8) ----------------------------------------------------
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (no link against libcuda).
+civic_status_t tensor_map_encoder(EncodeTiledFn* out)
+{
+    static std::atomic<void*> cached{nullptr};
+    void* fn = cached.load(std::memory_order_acquire);
+    if (!fn) {
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        CIVIC_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || !fn) return cuda_fail(cudaErrorNotSupported, "cuTensorMapEncodeTiled");
+        cached.store(fn, std::memory_order_release);
+    }
+    *out = (EncodeTiledFn)fn;
+    return CIVIC_OK;
+}
+
+// bf16 tensor of rank 2 or 3, innermost dimension first; boxes of 64 elements (128 B, swizzled).
+civic_status_t make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                        const uint64_t* strides_bytes, uint32_t box_rows)
+{
+    cuuint64_t gdim[3] = {dims[0], dims[1], rank == 3 ? dims[2] : 1};
+    cuuint64_t gstr[2] = {strides_bytes[0], rank == 3 ? strides_bytes[1] : 0};
+    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_error, sizeof g_cuda_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return CIVIC_ERR_CUDA;
+    }
+    return CIVIC_OK;
+}
+
+struct AggPlan {
+    int32_t t_ld, n_tiles_t, values_bn;
+    size_t q_off, qsum_off, stats_off, p_off, lpart_off, invl_off, total;
+};
+
+civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d_v, AggPlan& pl)
+{
+    if (n_img < 0 || t_e < 1 || m_e < 1 || d_v < 1) return CIVIC_ERR_INVALID_ARG;
+    if (d_v % 64) return CIVIC_ERR_UNSUPPORTED;
+    pl.t_ld = (t_e + 7) / 8 * 8;
+    pl.n_tiles_t = (t_e + civic::kScoresBN - 1) / civic::kScoresBN;
+    pl.values_bn = d_v % 256 == 0 ? 256 : (d_v % 192 == 0 ? 192 : (d_v % 128 == 0 ? 128 : 256));
+    const int64_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
+    if (n_img > 65535 || pl.n_tiles_t > 65535 || m_tiles > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    size_t off = 0;
+    auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
+    pl.q_off = take((size_t)m_e * d_v * 2);
+    pl.qsum_off = take((size_t)m_e * 4);
+    pl.stats_off = take((size_t)n_img * t_e * 8);
+    pl.p_off = take((size_t)n_img * m_e * pl.t_ld * 2);
+    pl.lpart_off = take((size_t)n_img * m_e * pl.n_tiles_t * 4);
+    pl.invl_off = take((size_t)n_img * m_e * 4);
+    pl.total = off;
+    return CIVIC_OK;
+}
+
+template <int BN>
+civic_status_t launch_values(const CUtensorMap& map_p, const CUtensorMap& map_x, const civic::ValuesParams& vp,
+                             int32_t m_tiles, int32_t n_img, cudaStream_t stream)
+{
+    const size_t smem = sizeof(civic::ValuesSmem<BN>) + 1024;
+    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_values_kernel<BN>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)m_tiles, (unsigned)((vp.d_v + BN - 1) / BN), (unsigned)n_img);
+    cfg.blockDim = dim3(civic::kAggThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic() ? 1 : 0;
+    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_values_kernel<BN>, map_p, map_x, vp));
+    return CIVIC_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -407,6 +494,123 @@ civic_status_t civic_select_large_static(const float* scores, int32_t n_seg, con
     // the histograms and scalars inside the scratch are cleared by launch_large on every call
     return launch_large(scores, n_seg, *desc, keep_idx, scratch, pl, (int32_t)(desc->k - n_res),
                         (cudaStream_t)stream);
+}
+
+size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d_v)
+{
+    AggPlan pl;
+    return plan_aggregate(n_img, t_e, m_e, d_v, pl) == CIVIC_OK ? pl.total : 0;
+}
+
+civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
+                                      int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
+                                      void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                      void* stream_)
+{
+    AggPlan pl;
+    const civic_status_t st = plan_aggregate(n_img, t_e, m_e, d_v, pl);
+    if (st != CIVIC_OK) return st;
+    if (!(tau >= 0.025f) || !(tau <= 1e30f)) return CIVIC_ERR_UNSUPPORTED;  // also rejects NaN
+    if (n_img == 0) return CIVIC_OK;
+    if (!x0 || !anchors || !z0 || !device_status) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(x0, 16) || !aligned(z0, 16) || !aligned(anchors, 4) || !aligned(token_mass, 4) ||
+        !aligned(device_status, 4))
+        return CIVIC_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < pl.total) return CIVIC_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return CIVIC_ERR_ALIGNMENT;
+    const size_t x_bytes = (size_t)n_img * t_e * d_v * 2, z_bytes = (size_t)n_img * m_e * d_v * 2;
+    if (overlaps(z0, z_bytes, x0, x_bytes) || overlaps(z0, z_bytes, anchors, (size_t)m_e * d_v * 4) ||
+        overlaps(workspace, pl.total, x0, x_bytes) || overlaps(workspace, pl.total, z0, z_bytes) ||
+        overlaps(workspace, pl.total, anchors, (size_t)m_e * d_v * 4) ||
+        overlaps(token_mass, (size_t)n_img * t_e * 4, z0, z_bytes) ||
+        overlaps(token_mass, (size_t)n_img * t_e * 4, workspace, pl.total) ||
+        overlaps(device_status, 4, workspace, pl.total) || overlaps(device_status, 4, z0, z_bytes))
+        return CIVIC_ERR_INVALID_ARG;
+
+    cudaStream_t stream = (cudaStream_t)stream_;
+    char* ws = (char*)workspace;
+    __nv_bfloat16* q = (__nv_bfloat16*)(ws + pl.q_off);
+    float* qsum = (float*)(ws + pl.qsum_off);
+    float2* stats = (float2*)(ws + pl.stats_off);
+    __nv_bfloat16* p = (__nv_bfloat16*)(ws + pl.p_off);
+    float* lpart = (float*)(ws + pl.lpart_off);
+    float* inv_l = (float*)(ws + pl.invl_off);
+
+    EncodeTiledFn enc = nullptr;
+    const civic_status_t est = tensor_map_encoder(&enc);
+    if (est != CIVIC_OK) return est;
+    CUtensorMap map_q, map_x_scores, map_p, map_x_values;
+    civic_status_t ms;
+    {
+        const uint64_t dims[2] = {(uint64_t)d_v, (uint64_t)m_e}, str[1] = {(uint64_t)d_v * 2};
+        if ((ms = make_map(enc, &map_q, q, 2, dims, str, civic::kAggBM)) != CIVIC_OK) return ms;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)d_v, (uint64_t)t_e, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)d_v * 2, (uint64_t)t_e * d_v * 2};
+        if ((ms = make_map(enc, &map_x_scores, x0, 3, dims, str, civic::kScoresBN)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_x_values, x0, 3, dims, str, civic::kAggBK)) != CIVIC_OK) return ms;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)t_e, (uint64_t)m_e, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)pl.t_ld * 2, (uint64_t)m_e * pl.t_ld * 2};
+        if ((ms = make_map(enc, &map_p, p, 3, dims, str, civic::kAggBM)) != CIVIC_OK) return ms;
+    }
+
+    const bool pdl = programmatic();
+    CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::anchor_prep_kernel, (unsigned)((m_e + 7) / 8), 256u, 0, stream, anchors,
+                                 m_e, d_v, 1e-5f, 1e-12f, q, qsum));
+    const long long n_tokens = (long long)n_img * t_e;
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_stats_kernel, (unsigned)((n_tokens + 7) / 8), 256u, 0, stream,
+                                 (const __nv_bfloat16*)x0, n_tokens, d_v, 1e-5f, 1e-12f, stats));
+
+    const int32_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
+    civic::ScoresParams sp;
+    sp.stats = stats; sp.qsum = qsum; sp.p = p; sp.lpart = lpart; sp.error = device_status;
+    sp.n_img = n_img; sp.m_e = m_e; sp.t_e = t_e; sp.d_v = d_v; sp.t_ld = pl.t_ld; sp.n_tiles_t = pl.n_tiles_t;
+    sp.inv_tau_log2e = 1.4426950408889634f / tau;
+    {
+        const size_t smem = sizeof(civic::ScoresSmem) + 1024;
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_scores_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)m_tiles, (unsigned)pl.n_tiles_t, (unsigned)n_img);
+        cfg.blockDim = dim3(civic::kAggThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl ? 1 : 0;
+        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_scores_kernel, map_q, map_x_scores, sp));
+    }
+    civic::ValuesParams vp;
+    vp.lpart = lpart; vp.z = (__nv_bfloat16*)z0; vp.inv_l = inv_l; vp.error = device_status;
+    vp.n_img = n_img; vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_tiles_t = pl.n_tiles_t;
+    civic_status_t vs;
+    if (pl.values_bn == 256) vs = launch_values<256>(map_p, map_x_values, vp, m_tiles, n_img, stream);
+    else if (pl.values_bn == 192) vs = launch_values<192>(map_p, map_x_values, vp, m_tiles, n_img, stream);
+    else vs = launch_values<128>(map_p, map_x_values, vp, m_tiles, n_img, stream);
+    if (vs != CIVIC_OK) return vs;
+    int n_launched = 4;
+    if (token_mass) {
+        CIVIC_CUDA_TRY(cudaGetLastError());
+        const dim3 grid((unsigned)((t_e + 255) / 256), (unsigned)n_img);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl ? 1 : 0;
+        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::token_mass_kernel, (const __nv_bfloat16*)p, (const float*)inv_l,
+                                          m_e, t_e, pl.t_ld, token_mass));
+        ++n_launched;
+    }
+    g_launches.fetch_add(n_launched, std::memory_order_relaxed);
+    return CIVIC_OK;
 }
 
 civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civic_select_desc_t* descs,

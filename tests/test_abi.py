@@ -226,6 +226,23 @@ def test_adjacent_calls_validation(lib):
     assert lib.civic_launch_count() == before
 
 
+def test_anchor_aggregate_validation(lib):
+    f = lambda n_img=1, t_e=100, m_e=10, d_v=128, tau=0.1, x=0x100000, a=0x200000, z=0x300000, mass=None, \
+        ws=0x1000000, ws_bytes=1 << 30, status=0x400000: \
+        lib.civic_anchor_aggregate(x, a, n_img, t_e, m_e, d_v, ctypes.c_float(tau), z, mass, ws, ws_bytes, status, None)
+    before = lib.civic_launch_count()
+    assert f(d_v=100) == 5 and f(d_v=0) == 1 and f(t_e=0) == 1 and f(m_e=0) == 1
+    assert f(tau=0.01) == 5 and f(tau=float("nan")) == 5
+    assert f(x=None) == 1 and f(status=None) == 1 and f(x=0x100008) == 4
+    assert f(ws=None) == 7 and f(ws_bytes=1000) == 7 and f(ws=0x1000010) == 4
+    assert f(z=0x100100) == 1  # output overlaps the tokens
+    assert f(n_img=0) == 0
+    assert civic.anchor_aggregate_workspace_bytes(1, 100, 10, 100) == 0
+    need = civic.anchor_aggregate_workspace_bytes(2, 100, 10, 128)
+    assert need >= 10 * 128 * 2 + 2 * 100 * 8 + 2 * 10 * 104 * 2 and need % 256 == 0
+    assert lib.civic_launch_count() == before
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
 
