@@ -13,15 +13,16 @@
 // Kernels
 //   anchor_prep_kernel      A (fp32) -> Q_A (bf16) and the row sums of the rounded values
 //   token_stats_kernel      X_0 (bf16) -> (mu_i, r_i), one warp per token, HBM-bound
-//   aggregate_scores_kernel tcgen05 GEMM  S = Q_A X_0^T  (both operands K-major), epilogue
+//   aggregate_gemm_kernel<ScoresOp>   tcgen05 GEMM  S = Q_A X_0^T  (both operands K-major), epilogue
 //                           P = exp((r (S - mu qsum) - 1) / tau) as bf16 + partial row sums
-//   aggregate_values_kernel tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major)
+//   aggregate_gemm_kernel<ValuesOp>   tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major)
 //   token_mass_kernel       column sums of W_A (per-token importance), HBM-bound
 //
-// GEMM skeleton (both): 192 threads.  Warp 0 = TMA producer (one elected lane), warp 1 = TMEM
-// allocation + MMA issue (one elected lane), warps 2..5 = epilogue (each reads its own quarter
-// of the 128 TMEM lanes).  Operand tiles arrive by cp.async.bulk.tensor with 128-byte swizzle
-// into a ring of stages guarded by full/empty mbarriers; accumulators live in TMEM.
+// GEMM skeleton (both): persistent blocks of 320 threads, one per SM.  Warp 0 = TMA producer (one
+// elected lane), warp 1 = TMEM allocation + MMA issue (one elected lane), warps 2..9 = epilogue
+// (each reads its own quarter of the 128 TMEM lanes).  Operand tiles arrive by
+// cp.async.bulk.tensor with 128-byte swizzle into a ring of stages guarded by full/empty
+// mbarriers; two accumulators alternate in TMEM so the epilogue overlaps the next tile's MMAs.
 // Every wait is bounded: on a time-out the thread raises the kernel's error word, the block
 // stops issuing work, waits (bounded) for its copies in flight, frees its TMEM and returns.
 #pragma once
@@ -34,12 +35,10 @@
 
 namespace civic {
 
-constexpr int kAggThreads = 192;
+constexpr int kAggThreads = 320;      // producer warp, MMA warp, eight epilogue warps
 constexpr int kAggBM = 128;           // anchors per tile (TMEM lanes)
 constexpr int kAggBK = 64;            // 64 bf16 = one 128-byte swizzle row
-constexpr int kScoresBN = 128;        // tokens per tile of the first GEMM
-constexpr int kScoresStages = 3;      // 3 x 32 KB: two blocks fit one SM
-constexpr int kValuesStages = 4;
+constexpr int kScoresBN = 256;        // tokens per tile of the first GEMM
 constexpr unsigned long long kWaitLimitCycles = 1ull << 31;  // about a second
 
 enum AggError { kAggOk = 0, kAggTimeoutFull = 1, kAggTimeoutEmpty = 2, kAggTimeoutAcc = 3 };
@@ -129,21 +128,6 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// 32 consecutive fp32 columns of this warp's 32 TMEM lanes: thread t gets lane (base + t).
-__device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
 // Shared-memory operand descriptor, 128-byte swizzle, tile base 1024-byte aligned.
 //   K-major  (rows of 64 bf16 = 128 B): 8-row groups 1024 B apart (stride offset); the leading
 //             offset is unused with swizzling (set to one 16-byte unit).
@@ -239,281 +223,390 @@ __global__ void token_stats_kernel(const __nv_bfloat16* __restrict__ x, long lon
     }
 }
 
-// ----------------------------------------------------------------------------- GEMM 1: scores
+// ----------------------------------------------------------------------------- the two GEMMs
+//
+// One persistent kernel template: a block walks tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...
+// with the anchor tile fastest, so blocks that run at the same time share their X_0 tile in L2.
+// Two TMEM accumulators alternate between tiles: the epilogue warps drain one while the MMA thread
+// already fills the other.  `Op` supplies the tile width, how a stage is loaded, B's descriptor
+// and the epilogue.  Eight epilogue warps: two per TMEM lane quarter, each taking half of the
+// tile's columns (one warp per scheduler cannot hide its own latencies; measured 14 us per
+// 128 x 256 tile with four warps against 6.7 us of MMA time).
+
+struct TileGrid {
+    int32_t m_tiles, n_tiles, n_img, total;
+};
+
+__device__ __forceinline__ void tile_coords(const TileGrid& g, int t, int& m_tile, int& n_tile, int& img)
+{
+    m_tile = t % g.m_tiles;
+    const int rest = t / g.m_tiles;
+    n_tile = rest % g.n_tiles;
+    img = rest / g.n_tiles;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// 32 consecutive fp32 columns of this warp's 32 TMEM lanes (thread t gets lane base + t), split
+// into issue and wait, so that the next chunk's load runs under the current
+// chunk's arithmetic.  The wait names the registers as in/out operands: nothing that uses them
+// can be scheduled above it.
+__device__ __forceinline__ void tmem_load_issue(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_load_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
+}
+__device__ __forceinline__ float exp2_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Walks the `cols` (a multiple of 32) accumulator columns of one warp in chunks of 32 with two
+// register buffers; `body(acc, c0)` consumes chunk c0.
+template <class Body>
+__device__ __forceinline__ void for_each_chunk(uint32_t taddr, int cols, Body&& body)
+{
+    uint32_t even[32], odd[32];
+    tmem_load_issue(taddr, even);
+#pragma unroll 1
+    for (int c0 = 0; c0 < cols; c0 += 64) {
+        tmem_load_wait(even);
+        if (c0 + 32 < cols) tmem_load_issue(taddr + c0 + 32, odd);
+        body(even, c0);
+        if (c0 + 32 < cols) {
+            tmem_load_wait(odd);
+            if (c0 + 64 < cols) tmem_load_issue(taddr + c0 + 64, even);
+            body(odd, c0 + 32);
+        }
+    }
+}
 
 struct ScoresParams {
     const float2* stats;    // [n_img, t_e]  (mu, r)
     const float* qsum;      // [m_e]
     __nv_bfloat16* p;       // [n_img, m_e, t_ld]
-    float* lpart;           // [n_img, m_e, n_tiles_t] partial row sums of the rounded P
+    float* lpart;           // [n_img, m_e, 2 * n_tiles_t] partial row sums of the rounded P
     int* error;             // kernel error word (0 = fine)
-    int32_t n_img, m_e, t_e, d_v, t_ld, n_tiles_t;
+    TileGrid grid;
+    int32_t m_e, t_e, d_v, t_ld;
     float inv_tau_log2e;    // log2(e) / tau
 };
 
-struct alignas(1024) ScoresSmem {
-    __nv_bfloat16 a[kScoresStages][kAggBM * kAggBK];     // Q tile: 128 rows x 128 B
-    __nv_bfloat16 b[kScoresStages][kScoresBN * kAggBK];  // X tile: 128 tokens x 128 B
-    float2 stats[kScoresBN];
-    uint64_t full[kScoresStages], empty[kScoresStages], acc_full;
+struct ValuesParams {
+    const float* lpart;   // [n_img, m_e, n_parts]
+    __nv_bfloat16* z;     // [n_img, m_e, d_v]
+    float* inv_l;         // [n_img, m_e] written by the blocks of the first feature tile
+    int* error;
+    TileGrid grid;
+    int32_t m_e, t_e, d_v, n_parts;
+};
+
+constexpr int kEpilogueWarps = 8;
+
+template <int BN_, int STAGES_>
+struct alignas(1024) GemmSmem {
+    __nv_bfloat16 a[STAGES_][kAggBM * kAggBK];  // 128 rows x 128 B, K-major
+    __nv_bfloat16 b[STAGES_][BN_ * kAggBK];
+    float2 stats[kEpilogueWarps][128];          // per epilogue warp: (mu, r log2e / tau) of its columns (scores only)
+    uint64_t full[STAGES_], empty[STAGES_], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
-__global__ void __launch_bounds__(kAggThreads) aggregate_scores_kernel(const __grid_constant__ CUtensorMap map_q,
-                                                                       const __grid_constant__ CUtensorMap map_x,
-                                                                       const ScoresParams p)
+// S = Q_A X_0^T: tile of 128 anchors x 256 tokens, K = features; both operands K-major.
+struct ScoresOp {
+    static constexpr int BN = 256, STAGES = 4;
+    static constexpr bool kBMnMajor = false;
+    using Params = ScoresParams;
+    using Smem = GemmSmem<BN, STAGES>;
+    static __device__ __forceinline__ int k_steps(const Params& p) { return p.d_v / kAggBK; }
+    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
+                                                int k, int m0, int n0, int img)
+    {
+        mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
+        tma_load_2d(sm.a[s], map_a, k * kAggBK, m0, &sm.full[s]);
+        tma_load_3d(sm.b[s], map_b, k * kAggBK, n0, img, &sm.full[s]);                        // tokens n0 ..
+        tma_load_3d(sm.b[s] + 128 * kAggBK, map_b, k * kAggBK, n0 + 128, img, &sm.full[s]);  // .. + 128
+    }
+    static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 32, 16, 1024); }
+
+    // P = 2^(r' (acc - mu qsum) - c) for 32 columns of one anchor row, r' = r c, c = log2(e) / tau;
+    // MASK: columns at or beyond n_valid are tokens past the end of the image and give 0.
+    template <bool MASK>
+    static __device__ __forceinline__ void chunk(const uint32_t (&acc)[32], const float2* st, float qs, float neg_c,
+                                                 int n_valid, float& row_sum, uint32_t (&packed)[16])
+    {
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+            const float2 s0 = st[c], s1 = st[c + 1];
+            float v0 = exp2_fast(fmaf(s0.y, fmaf(-s0.x, qs, __uint_as_float(acc[c])), neg_c));
+            float v1 = exp2_fast(fmaf(s1.y, fmaf(-s1.x, qs, __uint_as_float(acc[c + 1])), neg_c));
+            if (MASK) {
+                v0 = c < n_valid ? v0 : 0.f;
+                v1 = c + 1 < n_valid ? v1 : 0.f;
+            }
+            const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+            row_sum += __low2float(h) + __high2float(h);
+            packed[c >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+    }
+
+    // thread = one anchor row of one half (128 token columns) of the tile
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, uint32_t tmem, int ewarp, int lane,
+                                                    int m0, int n0, int img, int n_tile)
+    {
+        const int quarter = ewarp & 3, half = ewarp >> 2;
+        const int nh = n0 + half * 128;  // first token of this warp's columns
+        float2* stats = sm.stats[ewarp];  // private to the warp: no barrier between warps
+        __syncwarp();
+#pragma unroll
+        for (int c = lane; c < 128; c += 32) {
+            const int tok = nh + c;
+            float2 st = tok < p.t_e ? p.stats[(size_t)img * p.t_e + tok] : make_float2(0.f, 0.f);
+            st.y *= p.inv_tau_log2e;
+            stats[c] = st;
+        }
+        __syncwarp();
+        const int m = m0 + quarter * 32 + lane;
+        const bool row_ok = m < p.m_e;
+        const float qs = row_ok ? p.qsum[m] : 0.f;
+        const float neg_c = -p.inv_tau_log2e;
+        float row_sum = 0.f;
+        __nv_bfloat16* out = p.p + ((size_t)img * p.m_e + (row_ok ? m : 0)) * p.t_ld + nh;
+        const bool full_tile = nh + 128 <= p.t_e;  // warp-uniform
+        for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * 128, 128,
+                       [&](const uint32_t (&acc)[32], int c0) {
+            uint32_t packed[16];
+            if (full_tile) chunk<false>(acc, stats + c0, qs, neg_c, 32, row_sum, packed);
+            else chunk<true>(acc, stats + c0, qs, neg_c, p.t_e - nh - c0, row_sum, packed);
+            if (row_ok) {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)  // 8 columns per 16-byte store; t_ld is a multiple of 8
+                    if (full_tile || nh + c0 + q4 * 8 < p.t_ld)
+                        *reinterpret_cast<uint4*>(out + c0 + q4 * 8) =
+                            make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
+            }
+        });
+        if (row_ok) p.lpart[((size_t)img * p.m_e + m) * (2 * p.grid.n_tiles) + 2 * n_tile + half] = row_sum;
+    }
+};
+
+// Z_0 = (P X_0) / l: tile of 128 anchors x BN features, K = tokens; A = P K-major, B = X_0
+// MN-major (BN / 64 blocks of 64 tokens x 128 B).
+template <int BN_>
+struct ValuesOp {
+    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5;
+    static constexpr bool kBMnMajor = true;
+    using Params = ValuesParams;
+    using Smem = GemmSmem<BN, STAGES>;
+    static __device__ __forceinline__ int k_steps(const Params& p) { return (p.t_e + kAggBK - 1) / kAggBK; }
+    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
+                                                int k, int m0, int n0, int img)
+    {
+        mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
+        tma_load_3d(sm.a[s], map_a, k * kAggBK, m0, img, &sm.full[s]);
+#pragma unroll
+        for (int j = 0; j < BN / 64; ++j)  // 64 features x 64 tokens per box
+            tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_b, n0 + j * 64, k * kAggBK, img, &sm.full[s]);
+    }
+    // 16 token rows of 128 B per K step; the next 64 features start one box (8 KB) further on
+    static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
+
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, uint32_t tmem, int ewarp, int lane, int m0,
+                                                    int n0, int img, int n_tile)
+    {
+        constexpr int kHalf = BN / 2;  // 64, 96 or 128 feature columns per warp
+        const int quarter = ewarp & 3, half = ewarp >> 2;
+        const int m = m0 + quarter * 32 + lane;
+        const bool row_ok = m < p.m_e;
+        float l = 0.f;  // the row's partial sums from the first GEMM
+        if (row_ok) {
+            const float* lp = p.lpart + ((size_t)img * p.m_e + m) * p.n_parts;
+            for (int t = 0; t < p.n_parts; ++t) l += lp[t];
+        }
+        const float inv_l = l > 0.f ? 1.f / l : 0.f;
+        if (row_ok && n_tile == 0 && half == 0) p.inv_l[(size_t)img * p.m_e + m] = inv_l;
+        const int nh = n0 + half * kHalf;
+        __nv_bfloat16* out = p.z + ((size_t)img * p.m_e + (row_ok ? m : 0)) * p.d_v + nh;
+        for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * kHalf, kHalf,
+                       [&](const uint32_t (&acc)[32], int c0) {
+            if (row_ok) {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    if (nh + c0 + q4 * 8 < p.d_v) {  // d_v is a multiple of 8
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 h =
+                                __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv_l,
+                                                      __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv_l);
+                            w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        });
+    }
+};
+
+template <class Op>
+__global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                     const __grid_constant__ CUtensorMap map_b,
+                                                                     const typename Op::Params p)
 {
+    constexpr int BN = Op::BN, STAGES = Op::STAGES;
+    constexpr uint32_t kAccStride = 256;  // TMEM columns between the two accumulators
     extern __shared__ uint8_t smem_raw[];
-    ScoresSmem& sm = *reinterpret_cast<ScoresSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    using Smem = typename Op::Smem;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kAggBM, n0 = blockIdx.y * kScoresBN, img = blockIdx.z;
-    const int k_steps = p.d_v / kAggBK;
+    const int k_steps = Op::k_steps(p);
     volatile int* abort = &sm.abort;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kScoresStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
-        mbar_init(&sm.acc_full, 1);
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sm.acc_full[b], 1); mbar_init(&sm.acc_empty[b], kEpilogueWarps); }
         sm.abort = 0;
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(&sm.tmem_base, kScoresBN);
+    if (warp == 1) tmem_alloc(&sm.tmem_base, 512);
     wait_for_prior_kernels();
-    if (warp >= 2) {  // token statistics of this tile's columns
-        const int c = threadIdx.x - 64;
-        const int tok = n0 + c;
-        sm.stats[c] = tok < p.t_e ? p.stats[(size_t)img * p.t_e + tok] : make_float2(0.f, 0.f);
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_acc = sm.tmem_base;
+    const uint32_t tmem_base = sm.tmem_base;
     const bool stop = *p.error != 0;  // an earlier block of this launch already failed
 
+    // A wait on the "empty" side uses the opposite parity, so the first pass over a fresh
+    // barrier falls through (nothing has to be drained yet).
     if (warp == 0 && lane == 0 && !stop) {
-        // ---- producer: one box of Q and one of X per stage
-        int issued = 0;
-        for (int k = 0; k < k_steps; ++k, ++issued) {
-            const int s = k % kScoresStages;
-            if (k >= kScoresStages &&
-                !mbar_wait(&sm.empty[s], ((k / kScoresStages) - 1) & 1, abort, p.error, kAggTimeoutEmpty))
-                break;
-            mbar_expect_tx(&sm.full[s], (kAggBM + kScoresBN) * kAggBK * 2);
-            tma_load_2d(sm.a[s], &map_q, k * kAggBK, m0, &sm.full[s]);
-            tma_load_3d(sm.b[s], &map_x, k * kAggBK, n0, img, &sm.full[s]);
+        // ---- producer
+        uint32_t it = 0;  // stages issued so far, over all tiles
+        bool ok = true;
+        for (int t = blockIdx.x; t < p.grid.total && ok; t += gridDim.x) {
+            int m_tile, n_tile, img;
+            tile_coords(p.grid, t, m_tile, n_tile, img);
+            for (int k = 0; k < k_steps; ++k, ++it) {
+                const int s = it % STAGES;
+                ok = mbar_wait(&sm.empty[s], ((it / STAGES) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty);
+                if (!ok) break;
+                Op::load(sm, s, &map_a, &map_b, k, m_tile * kAggBM, n_tile * BN, img);
+            }
         }
         if (*abort) {  // let the copies already in flight land before the block goes away
-            for (int k = max(0, issued - kScoresStages); k < issued; ++k) {
+            for (uint32_t j = it > (uint32_t)STAGES ? it - STAGES : 0; j < it; ++j) {
                 const long long t0 = clock64();
-                while (!mbar_try_wait(&sm.full[k % kScoresStages], (k / kScoresStages) & 1) &&
+                while (!mbar_try_wait(&sm.full[j % STAGES], (j / STAGES) & 1) &&
                        (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
             }
         }
     } else if (warp == 1 && lane == 0 && !stop) {
         // ---- MMA issue: 4 instructions of K = 16 per stage
-        constexpr uint32_t idesc = umma_idesc(kScoresBN, 0);
+        constexpr uint32_t idesc = umma_idesc(BN, Op::kBMnMajor ? 1 : 0);
+        uint32_t it = 0;
         bool ok = true;
-        for (int k = 0; k < k_steps && ok; ++k) {
-            const int s = k % kScoresStages;
-            ok = mbar_wait(&sm.full[s], (k / kScoresStages) & 1, abort, p.error, kAggTimeoutFull);
+        int local = 0;
+        for (int t = blockIdx.x; t < p.grid.total && ok; t += gridDim.x, ++local) {
+            const int buf = local & 1;
+            ok = mbar_wait(&sm.acc_empty[buf], ((local >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutAcc);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
+            const uint32_t tmem_acc = tmem_base + buf * kAccStride;
+            for (int k = 0; k < k_steps; ++k, ++it) {
+                const int s = it % STAGES;
+                ok = mbar_wait(&sm.full[s], (it / STAGES) & 1, abort, p.error, kAggTimeoutFull);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
 #pragma unroll
-            for (int kk = 0; kk < kAggBK / 16; ++kk)
-                umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), umma_desc(b0 + kk * 32, 16, 1024), idesc,
-                          (k | kk) != 0);
-            umma_commit(&sm.empty[s]);  // frees the stage once these MMAs have read it
-        }
-        if (ok) umma_commit(&sm.acc_full);
-    } else if (warp >= 2 && !stop) {
-        // ---- epilogue: thread = one anchor row, 4 chunks of 32 token columns
-        const int quarter = warp & 3;  // TMEM lane quarter this warp may read
-        const int m = m0 + quarter * 32 + lane;
-        // tcgen05.ld is warp-collective: the whole warp goes on, or none of it
-        if (__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full, 0, abort, p.error, kAggTimeoutAcc))) {
-            tc_fence_after_sync();
-            const float qs = m < p.m_e ? p.qsum[m] : 0.f;
-            float row_sum = 0.f;
-            __nv_bfloat16* out = p.p + ((size_t)img * p.m_e + (m < p.m_e ? m : 0)) * p.t_ld + n0;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kScoresBN; c0 += 32) {
-                uint32_t acc[32];
-                tmem_load_32cols(tmem_acc + ((uint32_t)(quarter * 32) << 16) + c0, acc);
-                uint32_t packed[16];
-#pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    float v[2];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const float2 st = sm.stats[c0 + c + e];
-                        const float cosine = st.y * (__uint_as_float(acc[c + e]) - st.x * qs);
-                        v[e] = (n0 + c0 + c + e) < p.t_e ? exp2f((cosine - 1.f) * p.inv_tau_log2e) : 0.f;
-                    }
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[0], v[1]);
-                    row_sum += __low2float(h) + __high2float(h);
-                    packed[c >> 1] = *reinterpret_cast<const uint32_t*>(&h);
-                }
-                if (m < p.m_e) {
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)  // 8 columns per 16-byte store; t_ld is a multiple of 8
-                        if (n0 + c0 + q4 * 8 < p.t_ld)
-                            *reinterpret_cast<uint4*>(out + c0 + q4 * 8) =
-                                make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
-                }
+                for (int kk = 0; kk < kAggBK / 16; ++kk)
+                    umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                umma_commit(&sm.empty[s]);  // frees the stage once these MMAs have read it
             }
-            if (m < p.m_e) p.lpart[((size_t)img * p.m_e + m) * p.n_tiles_t + blockIdx.y] = row_sum;
+            if (ok) umma_commit(&sm.acc_full[buf]);
         }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after_sync();
-        tmem_dealloc(tmem_acc, kScoresBN);
-    }
-}
-
-// ----------------------------------------------------------------------------- GEMM 2: values
-
-struct ValuesParams {
-    const float* lpart;   // [n_img, m_e, n_tiles_t]
-    __nv_bfloat16* z;     // [n_img, m_e, d_v]
-    float* inv_l;         // [n_img, m_e] written by the blocks of the first feature tile
-    int* error;
-    int32_t n_img, m_e, t_e, d_v, n_tiles_t;
-};
-
-template <int BN>
-struct alignas(1024) ValuesSmem {
-    __nv_bfloat16 a[kValuesStages][kAggBM * kAggBK];  // P tile: 128 anchors x 64 tokens (K-major)
-    __nv_bfloat16 b[kValuesStages][kAggBK * BN];      // X tile: BN/64 blocks of 64 tokens x 128 B (MN-major)
-    uint64_t full[kValuesStages], empty[kValuesStages], acc_full;
-    uint32_t tmem_base;
-    int abort;
-};
-
-template <int BN>
-__global__ void __launch_bounds__(kAggThreads) aggregate_values_kernel(const __grid_constant__ CUtensorMap map_p,
-                                                                       const __grid_constant__ CUtensorMap map_x,
-                                                                       const ValuesParams p)
-{
-    constexpr uint32_t kTmemCols = BN <= 128 ? 128 : 256;
-    extern __shared__ uint8_t smem_raw[];
-    using Smem = ValuesSmem<BN>;
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kAggBM, n0 = blockIdx.y * BN, img = blockIdx.z;
-    const int k_steps = (p.t_e + kAggBK - 1) / kAggBK;
-    volatile int* abort = &sm.abort;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kValuesStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
-        mbar_init(&sm.acc_full, 1);
-        sm.abort = 0;
-        fence_barrier_init();
-    }
-    if (warp == 1) tmem_alloc(&sm.tmem_base, kTmemCols);
-    wait_for_prior_kernels();
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_acc = sm.tmem_base;
-    const bool stop = *p.error != 0;
-
-    if (warp == 0 && lane == 0 && !stop) {
-        int issued = 0;
-        for (int k = 0; k < k_steps; ++k, ++issued) {
-            const int s = k % kValuesStages;
-            if (k >= kValuesStages &&
-                !mbar_wait(&sm.empty[s], ((k / kValuesStages) - 1) & 1, abort, p.error, kAggTimeoutEmpty))
+    } else if (warp >= 2 && !stop) {
+        // ---- epilogue: warps 2..9; a warp may read the TMEM lane quarter (warp index mod 4)
+        const int ewarp = ((warp & 3) | ((warp - 2) & 4));  // quarter in bits 0-1, column half in bit 2
+        int local = 0;
+        for (int t = blockIdx.x; t < p.grid.total; t += gridDim.x, ++local) {
+            int m_tile, n_tile, img;
+            tile_coords(p.grid, t, m_tile, n_tile, img);
+            const int buf = local & 1;
+            // tcgen05.ld is warp-collective: the whole warp goes on, or none of it
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full[buf], (local >> 1) & 1, abort, p.error, kAggTimeoutAcc)))
                 break;
-            mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
-            tma_load_3d(sm.a[s], &map_p, k * kAggBK, m0, img, &sm.full[s]);
-#pragma unroll
-            for (int j = 0; j < BN / 64; ++j)  // 64 features x 64 tokens per box
-                tma_load_3d(sm.b[s] + j * (kAggBK * 64), &map_x, n0 + j * 64, k * kAggBK, img, &sm.full[s]);
-        }
-        if (*abort) {
-            for (int k = max(0, issued - kValuesStages); k < issued; ++k) {
-                const long long t0 = clock64();
-                while (!mbar_try_wait(&sm.full[k % kValuesStages], (k / kValuesStages) & 1) &&
-                       (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
-            }
-        }
-    } else if (warp == 1 && lane == 0 && !stop) {
-        constexpr uint32_t idesc = umma_idesc(BN, 1);
-        bool ok = true;
-        for (int k = 0; k < k_steps && ok; ++k) {
-            const int s = k % kValuesStages;
-            ok = mbar_wait(&sm.full[s], (k / kValuesStages) & 1, abort, p.error, kAggTimeoutFull);
-            if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
-#pragma unroll
-            for (int kk = 0; kk < kAggBK / 16; ++kk)  // A: 32 B per K step; B: 16 token rows of 128 B
-                umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024),
-                          umma_desc(b0 + kk * 2048, kAggBK * 128, 1024), idesc, (k | kk) != 0);
-            umma_commit(&sm.empty[s]);
-        }
-        if (ok) umma_commit(&sm.acc_full);
-    } else if (warp >= 2 && !stop) {
-        const int quarter = warp & 3;
-        const int m = m0 + quarter * 32 + lane;
-        // 1 / l[m]: the row's partial sums from the first GEMM
-        float l = 0.f;
-        if (m < p.m_e) {
-            const float* lp = p.lpart + ((size_t)img * p.m_e + m) * p.n_tiles_t;
-            for (int t = 0; t < p.n_tiles_t; ++t) l += lp[t];
-        }
-        const float inv_l = l > 0.f ? 1.f / l : 0.f;
-        if (m < p.m_e && blockIdx.y == 0) p.inv_l[(size_t)img * p.m_e + m] = inv_l;
-        if (__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full, 0, abort, p.error, kAggTimeoutAcc))) {
-            tc_fence_after_sync();
-            __nv_bfloat16* out = p.z + ((size_t)img * p.m_e + (m < p.m_e ? m : 0)) * p.d_v + n0;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t acc[32];
-                tmem_load_32cols(tmem_acc + ((uint32_t)(quarter * 32) << 16) + c0, acc);
-                if (m < p.m_e) {
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        if (n0 + c0 + q4 * 8 < p.d_v) {  // d_v is a multiple of 8
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __nv_bfloat162 h =
-                                    __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv_l,
-                                                          __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv_l);
-                                w[e] = *reinterpret_cast<const uint32_t*>(&h);
-                            }
-                            *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    }
-                }
-            }
+            Op::epilogue(p, sm, tmem_base + buf * kAccStride, ewarp, lane, m_tile * kAggBM, n_tile * BN, img, n_tile);
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);  // this warp has drained its part
         }
     }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_acc, kTmemCols);
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
-// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m].  Thread per token, coalesced rows.
-__global__ void token_mass_kernel(const __nv_bfloat16* __restrict__ p, const float* __restrict__ inv_l, int m_e, int t_e,
-                                  int t_ld, float* __restrict__ mass)
+// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m].  A block owns 64 token columns of one
+// image: warp w adds rows w, w + 8, ... (one 128-byte line per row), the 8 warps' sums are added
+// in a fixed order, so the result does not depend on scheduling.
+constexpr int kMassCols = 64;
+__global__ void __launch_bounds__(256) token_mass_kernel(const __nv_bfloat16* __restrict__ p,
+                                                         const float* __restrict__ inv_l, int m_e, int t_e, int t_ld,
+                                                         float* __restrict__ mass)
 {
+    __shared__ float2 part[8][32];
     wait_for_prior_kernels();
-    const int img = blockIdx.y;
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= t_e) return;
-    const __nv_bfloat16* col = p + (size_t)img * m_e * t_ld + i;
+    const int img = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int col = blockIdx.x * kMassCols + 2 * lane;  // t_ld is even: a column pair never straddles a row
+    const __nv_bfloat16* base = p + (size_t)img * m_e * t_ld + col;
     const float* il = inv_l + (size_t)img * m_e;
-    float acc = 0.f;
-    for (int m = 0; m < m_e; ++m) acc += __bfloat162float(col[(size_t)m * t_ld]) * __ldg(il + m);
-    mass[(size_t)img * t_e + i] = acc;
+    float2 acc = make_float2(0.f, 0.f);
+    if (col < t_ld) {
+#pragma unroll 4
+        for (int m = warp; m < m_e; m += 8) {
+            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(base + (size_t)m * t_ld));
+            const float w = __ldg(il + m);
+            acc.x += v.x * w;
+            acc.y += v.y * w;
+        }
+    }
+    part[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0) {
+        float2 s = part[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) { s.x += part[w][lane].x; s.y += part[w][lane].y; }
+        float* out = mass + (size_t)img * t_e;
+        if (col < t_e) out[col] = s.x;
+        if (col + 1 < t_e) out[col + 1] = s.y;
+    }
 }
 
 }  // namespace civic

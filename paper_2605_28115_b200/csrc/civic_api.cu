@@ -359,28 +359,30 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
     pl.n_tiles_t = (t_e + civic::kScoresBN - 1) / civic::kScoresBN;
     pl.values_bn = d_v % 256 == 0 ? 256 : (d_v % 192 == 0 ? 192 : (d_v % 128 == 0 ? 128 : 256));
     const int64_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
-    if (n_img > 65535 || pl.n_tiles_t > 65535 || m_tiles > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
+    if (m_tiles * pl.n_tiles_t * n_img > INT32_MAX || m_tiles * ((d_v + 127) / 128) * n_img > INT32_MAX)
+        return CIVIC_ERR_UNSUPPORTED;
     size_t off = 0;
     auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
     pl.q_off = take((size_t)m_e * d_v * 2);
     pl.qsum_off = take((size_t)m_e * 4);
     pl.stats_off = take((size_t)n_img * t_e * 8);
     pl.p_off = take((size_t)n_img * m_e * pl.t_ld * 2);
-    pl.lpart_off = take((size_t)n_img * m_e * pl.n_tiles_t * 4);
+    pl.lpart_off = take((size_t)n_img * m_e * 2 * pl.n_tiles_t * 4);  // two column halves per token tile
     pl.invl_off = take((size_t)n_img * m_e * 4);
     pl.total = off;
     return CIVIC_OK;
 }
 
-template <int BN>
-civic_status_t launch_values(const CUtensorMap& map_p, const CUtensorMap& map_x, const civic::ValuesParams& vp,
-                             int32_t m_tiles, int32_t n_img, cudaStream_t stream)
+template <class Op>
+civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const typename Op::Params& params,
+                           int32_t total_tiles, cudaStream_t stream)
 {
-    const size_t smem = sizeof(civic::ValuesSmem<BN>) + 1024;
-    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_values_kernel<BN>,
+    const size_t smem = sizeof(typename Op::Smem) + 1024;
+    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_gemm_kernel<Op>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int sms = sm_count();
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)m_tiles, (unsigned)((vp.d_v + BN - 1) / BN), (unsigned)n_img);
+    cfg.gridDim = dim3((unsigned)(total_tiles < sms ? total_tiles : sms));  // persistent: one block per SM
     cfg.blockDim = dim3(civic::kAggThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -389,7 +391,7 @@ civic_status_t launch_values(const CUtensorMap& map_p, const CUtensorMap& map_x,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = programmatic() ? 1 : 0;
-    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_values_kernel<BN>, map_p, map_x, vp));
+    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_gemm_kernel<Op>, map_a, map_b, params));
     return CIVIC_OK;
 }
 
@@ -548,7 +550,7 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     {
         const uint64_t dims[3] = {(uint64_t)d_v, (uint64_t)t_e, (uint64_t)n_img};
         const uint64_t str[2] = {(uint64_t)d_v * 2, (uint64_t)t_e * d_v * 2};
-        if ((ms = make_map(enc, &map_x_scores, x0, 3, dims, str, civic::kScoresBN)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_x_scores, x0, 3, dims, str, 128)) != CIVIC_OK) return ms;  // two boxes per stage
         if ((ms = make_map(enc, &map_x_values, x0, 3, dims, str, civic::kAggBK)) != CIVIC_OK) return ms;
     }
     {
@@ -568,36 +570,24 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     const int32_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
     civic::ScoresParams sp;
     sp.stats = stats; sp.qsum = qsum; sp.p = p; sp.lpart = lpart; sp.error = device_status;
-    sp.n_img = n_img; sp.m_e = m_e; sp.t_e = t_e; sp.d_v = d_v; sp.t_ld = pl.t_ld; sp.n_tiles_t = pl.n_tiles_t;
+    sp.grid = civic::TileGrid{m_tiles, pl.n_tiles_t, n_img, m_tiles * pl.n_tiles_t * n_img};
+    sp.m_e = m_e; sp.t_e = t_e; sp.d_v = d_v; sp.t_ld = pl.t_ld;
     sp.inv_tau_log2e = 1.4426950408889634f / tau;
-    {
-        const size_t smem = sizeof(civic::ScoresSmem) + 1024;
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_scores_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)m_tiles, (unsigned)pl.n_tiles_t, (unsigned)n_img);
-        cfg.blockDim = dim3(civic::kAggThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = pdl ? 1 : 0;
-        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_scores_kernel, map_q, map_x_scores, sp));
-    }
+    civic_status_t gs = launch_gemm<civic::ScoresOp>(map_q, map_x_scores, sp, sp.grid.total, stream);
+    if (gs != CIVIC_OK) return gs;
     civic::ValuesParams vp;
     vp.lpart = lpart; vp.z = (__nv_bfloat16*)z0; vp.inv_l = inv_l; vp.error = device_status;
-    vp.n_img = n_img; vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_tiles_t = pl.n_tiles_t;
-    civic_status_t vs;
-    if (pl.values_bn == 256) vs = launch_values<256>(map_p, map_x_values, vp, m_tiles, n_img, stream);
-    else if (pl.values_bn == 192) vs = launch_values<192>(map_p, map_x_values, vp, m_tiles, n_img, stream);
-    else vs = launch_values<128>(map_p, map_x_values, vp, m_tiles, n_img, stream);
-    if (vs != CIVIC_OK) return vs;
+    const int32_t f_tiles = (d_v + pl.values_bn - 1) / pl.values_bn;
+    vp.grid = civic::TileGrid{m_tiles, f_tiles, n_img, m_tiles * f_tiles * n_img};
+    vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t;
+    if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, vp, vp.grid.total, stream);
+    else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, vp, vp.grid.total, stream);
+    else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, vp, vp.grid.total, stream);
+    if (gs != CIVIC_OK) return gs;
     int n_launched = 4;
     if (token_mass) {
         CIVIC_CUDA_TRY(cudaGetLastError());
-        const dim3 grid((unsigned)((t_e + 255) / 256), (unsigned)n_img);
+        const dim3 grid((unsigned)((t_e + civic::kMassCols - 1) / civic::kMassCols), (unsigned)n_img);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.stream = stream;
         cudaLaunchAttribute attr[1];
