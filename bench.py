@@ -103,6 +103,17 @@ def config_of(wl, extra=None):
     return cfg
 
 
+def measured_tensor_peak():
+    """(burst, sustained) dense bf16 TFLOP/s of this machine's B200s and where they come from."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return 1590.0, 1400.0, "fallback (1.59 PFLOP/s burst, 1.4 sustained: earlier measurement)"
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -517,6 +528,150 @@ def run_civic(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- aggregation (Eq. 8)
+
+def run_aggregate(args):
+    """`--workload agg_*`: one step = one civic_anchor_aggregate call (anchor preparation, token
+    statistics, the two tensor-core contractions, token mass) on a batch of images."""
+    import numpy as np
+    import torch
+
+    from paper_2605_28115_b200 import build as civic_build
+    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import workloads as W
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
+        raise SystemExit("the aggregation workload is benchmarked on one GPU")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    dev = "cuda:0"
+    civic_build.build()
+    civic.load()
+    w = W.AGG_BY_NAME[args.workload]
+    x0, anchors = W.agg_inputs(w, dev)
+    z0 = torch.empty((w.n_img, w.m_e, w.d_v), dtype=torch.bfloat16, device=dev)
+    mass = torch.empty((w.n_img, w.t_e), dtype=torch.float32, device=dev)
+    ws = torch.empty(civic.anchor_aggregate_workspace_bytes(w.n_img, w.t_e, w.m_e, w.d_v), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        civic.civic_anchor_aggregate(x0, anchors, w.tau, z0=z0, token_mass=mass, workspace=ws, device_status=status)
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = civic.launch_count()
+    sampler.start()
+    start.record()
+    for _ in range(args.steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = civic.launch_count() - launches0
+    ms = start.elapsed_time(end) / args.steps
+    if int(status.item()) != 0:
+        raise SystemExit(f"a wait inside the aggregation kernels timed out (status {int(status.item())})")
+    value = w.flops / (ms * 1e-3) / 1e12
+    burst, sustained, which = measured_tensor_peak()
+    timed_s = ms * 1e-3 * args.steps
+    peak = sustained if timed_s > 0.5 else burst  # a long loop runs under the power cap
+    roofline = {"bound": "tensor", "kernel": "civic_anchor_aggregate: five launches, of which the two tcgen05 "
+                "contractions carry all the flops (the other three are HBM-bound helpers and are inside the time)",
+                "achieved": value, "peak": peak, "unit": "TFLOP/s", "frac": value / peak, "peak_source": which,
+                "peak_kind": "sustained" if timed_s > 0.5 else "burst", "frac_of_burst_peak": value / burst,
+                "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
+
+    # end to end: pinned host tokens in, compact rows and token mass back out
+    e2e = None
+    if not args.no_e2e:
+        x_h = torch.empty(x0.shape, dtype=x0.dtype, pin_memory=True).copy_(x0)
+        z_h = torch.empty(z0.shape, dtype=z0.dtype, pin_memory=True)
+        m_h = torch.empty(mass.shape, dtype=mass.dtype, pin_memory=True)
+
+        def host_step():
+            x0.copy_(x_h, non_blocking=True)
+            step()
+            z_h.copy_(z0, non_blocking=True)
+            m_h.copy_(mass, non_blocking=True)
+
+        host_step()
+        torch.cuda.synchronize()
+        n_e2e = max(1, args.e2e_steps)
+        s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s2.record()
+        for _ in range(n_e2e):
+            host_step()
+        e2.record()
+        torch.cuda.synchronize()
+        ms2 = s2.elapsed_time(e2) / n_e2e
+        e2e = {"value": w.flops / (ms2 * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms2, "steps": n_e2e,
+               "h2d_bytes_per_step": x_h.numel() * 2, "d2h_bytes_per_step": z_h.numel() * 2 + m_h.numel() * 4,
+               "results_match_device_path": bool(torch.equal(z_h, z0.cpu()))}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import aggregate as OA
+
+        x64 = x0[0].double().cpu().numpy()
+        a64 = anchors.double().cpu().numpy()
+        times = []
+        t_begin = time.perf_counter()
+        while len(times) < 2 or (time.perf_counter() - t_begin < 10 and len(times) < 8):
+            t0 = time.perf_counter()
+            z_o, w_o = OA.anchor_aggregate(x64, a64, w.tau)
+            times.append(time.perf_counter() - t0)
+        med = statistics.median(times)
+        err = float(np.max(np.abs(z0[0].float().cpu().numpy() - z_o)))
+        cpu = {"value": w.flops / w.n_img / med / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": f"the fp64 numpy oracle on ONE of the {w.n_img} images, median of {len(times)} runs, "
+                         f"{med * 1e3:.0f} ms per image", "max_abs_difference_to_gpu_result": err}
+
+    line = {"metric": "aggregation_TFLOPs_eq8", "value": value, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "n_img": w.n_img, "t_e": w.t_e, "m_e": w.m_e, "d_v": w.d_v, "tau": w.tau,
+                       "l2": "the tokens (75 MB) and the weights W_A (67 MB) together exceed L2; no flush",
+                       "parallelism": "single"},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+
+
+def run_aggregate_reference(args):
+    """The fp64 numpy oracle of Eq. 8 on this machine's host cores; each step is ONE image of the
+    workload (a bounded sample), at most 10 steps."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import aggregate as OA
+    from paper_2605_28115_b200 import workloads as W
+
+    w = W.AGG_BY_NAME[args.workload]
+    x0, anchors = W.agg_inputs(w.__class__(w.name, 1, w.t_e, w.m_e, w.d_v, w.tau, w.seed), "cpu")
+    x64, a64 = x0[0].double().numpy(), anchors.double().numpy()
+    steps, warm = min(args.steps, 10), min(max(args.warmup, 1), 3)
+    for _ in range(warm):
+        OA.anchor_aggregate(x64, a64, w.tau)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        OA.anchor_aggregate(x64, a64, w.tau)
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    value = w.flops / w.n_img / (ms * 1e-3) / 1e12
+    sample = f"each step = the fp64 numpy oracle on one of the {w.n_img} images of the workload"
+    line = {"impl": "reference", "metric": "aggregation_TFLOPs_eq8", "value": value, "unit": "TFLOP/s",
+            "n_gpus": args.gpus, "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "n_img": w.n_img, "t_e": w.t_e, "m_e": w.m_e, "d_v": w.d_v, "tau": w.tau,
+                       "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
 # ----------------------------------------------------------------------------- reference arm
 
 def run_reference(args):
@@ -577,7 +732,12 @@ def run_reference(args):
 
 if __name__ == "__main__":
     a = parse_args()
-    if a.impl == "reference":
+    if a.workload.startswith("agg_"):
+        if a.impl == "reference":
+            run_aggregate_reference(a)
+        else:
+            run_aggregate(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_civic(a)

@@ -245,3 +245,60 @@ def kv_algorithmic_bytes(wl: Workload) -> int:
 
 def hidden_algorithmic_bytes(wl: Workload) -> int:
     return 2 * wl.n_seg * wl.k * (wl.hidden_row_bytes + 12)
+
+
+# ---------------------------------------------------------------- compact visual aggregation (Eq. 8)
+
+@dataclasses.dataclass(frozen=True)
+class AggWorkload:
+    """Dense patch embeddings of a batch of images and a shared set of compact anchors."""
+
+    name: str
+    n_img: int
+    t_e: int  # dense patch tokens per image (before the 2x2 merge)
+    m_e: int  # compact anchors
+    d_v: int  # vision width
+    tau: float
+    seed: int = SEED_BASE + 9000
+
+    @property
+    def flops(self) -> int:
+        """Both contractions: Q_A K_0^T and W_A X_0, 2 flops per multiply-add."""
+        return 2 * 2 * self.n_img * self.m_e * self.t_e * self.d_v
+
+
+# 8 images of 896x896: 64x64 = 4096 patches of 14x14 pixels each (they become the 32x32 merged
+# tokens of the batch-8 selection workload), vision width 1152, 1024 anchors (256 compact tokens
+# after the 2x2 merger), temperature 0.07.
+AGG_896 = AggWorkload("agg_batch8_896", 8, 4096, 1024, 1152, 0.07)
+AGG_448 = AggWorkload("agg_single_448", 1, 1024, 256, 1152, 0.07)
+AGG_BY_NAME = {w.name: w for w in (AGG_896, AGG_448)}
+
+
+def agg_inputs(w: AggWorkload, device="cpu"):
+    """(x0 bf16 [n_img, t_e, d_v] ~ 1.5 N(0,1) + 0.7, anchors fp32 [m_e, d_v] ~ N(0,1)), seeded."""
+    import torch
+
+    x0 = payload_bf16_affine((w.n_img, w.t_e, w.d_v), w.seed, device, 1.5, 0.7)
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed + 1)
+    anchors = torch.randn((w.m_e, w.d_v), generator=g, device=device, dtype=torch.float32)
+    return x0, anchors
+
+
+def payload_bf16_affine(shape, seed: int, device, scale: float, offset: float):
+    """bf16 scale * N(0,1) + offset from torch's seeded generator on `device`."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    numel = 1
+    for s in shape:
+        numel *= s
+    out = torch.empty(numel, dtype=torch.bfloat16, device=device)
+    slab = 1 << 26
+    for lo in range(0, numel, slab):
+        hi = min(numel, lo + slab)
+        out[lo:hi] = (torch.randn(hi - lo, generator=g, device=device, dtype=torch.float32) * scale
+                      + offset).to(torch.bfloat16)
+    return out.view(*shape)
