@@ -337,12 +337,13 @@ civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, in
  *                the anchors' attention each dense token receives -- usable as the `scores` of
  *                civic_select
  * workspace      dev  scratch of civic_anchor_aggregate_workspace_bytes(...) bytes, 256-byte
- *                aligned (holds Q_A, the token statistics and W_A's unnormalised bf16 form)
+ *                aligned (holds Q_A, the token statistics, W_A's unnormalised bf16 form and
+ *                partial sums)
  * device_status  dev  int32, written: 0, or a non-zero code if a wait inside a kernel ran into
  *                its time limit (the kernels then stop cleanly and the outputs are invalid).
  *                Read it after synchronising the stream.
  * d_v must be a multiple of 64 (CIVIC_ERR_UNSUPPORTED otherwise); t_e and m_e are arbitrary.
- * Inputs must be finite.  Five launches (six with token_mass).
+ * Inputs must be finite.  Three launches and one 4-byte memset (five launches with token_mass).
  */
 civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
                                       int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,

@@ -11,12 +11,12 @@
 // P = exp((s - 1) / tau) cannot overflow and, for tau >= 0.025, cannot underflow bf16.
 //
 // Kernels
-//   anchor_prep_kernel      A (fp32) -> Q_A (bf16) and the row sums of the rounded values
-//   token_stats_kernel      X_0 (bf16) -> (mu_i, r_i), one warp per token, HBM-bound
+//   aggregate_prep_kernel   A (fp32) -> Q_A (bf16) and the row sums of the rounded values; X_0 (bf16)
+//                           -> (mu_i, r_i); one warp per row, HBM-bound
 //   aggregate_gemm_kernel<ScoresOp>   tcgen05 GEMM  S = Q_A X_0^T  (both operands K-major), epilogue
 //                           P = exp((r (S - mu qsum) - 1) / tau) as bf16 + partial row sums
 //   aggregate_gemm_kernel<ValuesOp>   tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major)
-//   token_mass_kernel       column sums of W_A (per-token importance), HBM-bound
+//   token_mass_*_kernel     column sums of W_A (per-token importance), HBM-bound
 //
 // GEMM skeleton (both): persistent blocks of 320 threads, one per SM.  Warp 0 = TMA producer (one
 // elected lane), warp 1 = TMEM allocation + MMA issue (one elected lane), warps 2..9 = epilogue
@@ -156,48 +156,64 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major)
 
 // ----------------------------------------------------------------------------- small kernels
 
-// Q_A = Norm(LN(A)) rounded to bf16, and qsum[m] = sum of the ROUNDED row (what the tensor
-// core will really multiply the token mean with).  One warp per anchor; rows of any length.
-__global__ void anchor_prep_kernel(const float* __restrict__ anchors, int m_e, int d_v, float ln_eps, float norm_eps,
-                                   __nv_bfloat16* __restrict__ q, float* __restrict__ qsum)
+// Both preparations in one launch, one warp per row.  Warps [0, m_e) take an anchor each:
+// Q_A = Norm(LN(A)) rounded to bf16, and qsum[m] = sum of the ROUNDED row (what the tensor core
+// will really multiply the token mean with).  The other warps take a token each: (mu_i, r_i)
+// with K_0[i] = r_i (x_i - mu_i), r_i = 0 for a token whose features are all equal.  Few
+// registers on purpose: the token part is HBM-bound and lives on occupancy (a version that held
+// the whole row in registers measured slower).
+__device__ __forceinline__ float warp_sum(float v)
 {
-    wait_for_prior_kernels();
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (warp >= m_e) return;
-    const float* a = anchors + (size_t)warp * d_v;
-    float s = 0.f;
-    for (int j = lane; j < d_v; j += 32) s += a[j];
-    for (int d = 16; d > 0; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-    const float mean = s / d_v;
-    float ss = 0.f;
-    for (int j = lane; j < d_v; j += 32) { const float c = a[j] - mean; ss += c * c; }
-    for (int d = 16; d > 0; d >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, d);
-    const float inv_std = rsqrtf(ss / d_v + ln_eps);
-    const float norm = sqrtf(ss) * inv_std;  // l2 norm of the layer-normalised row
-    const float scale = inv_std / fmaxf(norm, norm_eps);
-    float rounded_sum = 0.f;
-    for (int j = lane; j < d_v; j += 32) {
-        const __nv_bfloat16 v = __float2bfloat16_rn((a[j] - mean) * scale);
-        q[(size_t)warp * d_v + j] = v;
-        rounded_sum += __bfloat162float(v);
-    }
-    for (int d = 16; d > 0; d >>= 1) rounded_sum += __shfl_xor_sync(0xFFFFFFFFu, rounded_sum, d);
-    if (lane == 0) qsum[warp] = rounded_sum;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    return v;
 }
 
-// (mu_i, r_i) per token: K_0[i] = r_i (x_i - mu_i).  One warp per token row of d_v bf16
-// (d_v a multiple of 8: 16-byte loads).  r_i = 0 for a token whose features are all equal.
-__global__ void token_stats_kernel(const __nv_bfloat16* __restrict__ x, long long n_tokens, int d_v, float ln_eps,
-                                   float norm_eps, float2* __restrict__ stats)
+// scale such that Norm(LN(row)) = (row - mean) * scale; 0 when the row has no direction
+__device__ __forceinline__ float normalise_scale(float ss, int d_v, float ln_eps, float norm_eps)
+{
+    const float inv_std = rsqrtf(ss / d_v + ln_eps);
+    const float norm = sqrtf(ss) * inv_std;  // l2 norm of the layer-normalised row
+    return ss > 0.f ? inv_std / fmaxf(norm, norm_eps) : 0.f;
+}
+
+__global__ void __launch_bounds__(256) aggregate_prep_kernel(const float* __restrict__ anchors, int m_e,
+                                                             const __nv_bfloat16* __restrict__ x, long long n_tokens,
+                                                             int d_v, float ln_eps, float norm_eps,
+                                                             __nv_bfloat16* __restrict__ q, float* __restrict__ qsum,
+                                                             float2* __restrict__ stats)
 {
     wait_for_prior_kernels();
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (warp >= n_tokens) return;
-    const uint4* row = reinterpret_cast<const uint4*>(x + warp * d_v);
+    if (warp < m_e) {
+        // ---- anchor row (fp32): three passes, the row stays in L1
+        const float* a = anchors + warp * d_v;
+        float s = 0.f;
+        for (int j = lane; j < d_v; j += 32) s += a[j];
+        const float mean = warp_sum(s) / d_v;
+        float ss = 0.f;
+        for (int j = lane; j < d_v; j += 32) { const float c = a[j] - mean; ss += c * c; }
+        const float scale = normalise_scale(warp_sum(ss), d_v, ln_eps, norm_eps);
+        float rounded_sum = 0.f;
+        for (int j = lane; j < d_v; j += 32) {
+            const __nv_bfloat16 v = __float2bfloat16_rn((a[j] - mean) * scale);
+            q[warp * d_v + j] = v;
+            rounded_sum += __bfloat162float(v);
+        }
+        rounded_sum = warp_sum(rounded_sum);
+        if (lane == 0) qsum[warp] = rounded_sum;
+        return;
+    }
+    const long long tok = warp - m_e;
+    if (tok >= n_tokens) return;
+    // ---- token row (bf16, d_v a multiple of 8): one pass of 16-byte loads; sums are taken
+    // relative to the row's first element so that the variance keeps its accuracy
+    const uint4* row = reinterpret_cast<const uint4*>(x + tok * d_v);
     const int vecs = d_v >> 3;
-    float s = 0.f, s2 = 0.f;  // shifted sums keep the variance accurate: shift by the row's first element
-    const float shift = __bfloat162float(x[warp * d_v]);
+    const float shift = __bfloat162float(x[tok * d_v]);
+    float s = 0.f, s2 = 0.f;
+#pragma unroll 4
     for (int v = lane; v < vecs; v += 32) {
         const uint4 u = __ldg(row + v);
         const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
@@ -209,17 +225,12 @@ __global__ void token_stats_kernel(const __nv_bfloat16* __restrict__ x, long lon
             s2 += a * a + b * b;
         }
     }
-    for (int d = 16; d > 0; d >>= 1) {
-        s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-        s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, d);
-    }
+    s = warp_sum(s);
+    s2 = warp_sum(s2);
     if (lane == 0) {
         const float mean_shifted = s / d_v;
         const float ss = fmaxf(s2 - s * mean_shifted, 0.f);  // sum (x - mu)^2
-        const float inv_std = rsqrtf(ss / d_v + ln_eps);
-        const float norm = sqrtf(ss) * inv_std;
-        const float r = ss > 0.f ? inv_std / fmaxf(norm, norm_eps) : 0.f;
-        stats[warp] = make_float2(mean_shifted + shift, r);
+        stats[tok] = make_float2(mean_shifted + shift, normalise_scale(ss, d_v, ln_eps, norm_eps));
     }
 }
 
@@ -573,40 +584,55 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
     }
 }
 
-// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m].  A block owns 64 token columns of one
-// image: warp w adds rows w, w + 8, ... (one 128-byte line per row), the 8 warps' sums are added
-// in a fixed order, so the result does not depend on scheduling.
-constexpr int kMassCols = 64;
-__global__ void __launch_bounds__(256) token_mass_kernel(const __nv_bfloat16* __restrict__ p,
-                                                         const float* __restrict__ inv_l, int m_e, int t_e, int t_ld,
-                                                         float* __restrict__ mass)
+// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m], in two deterministic steps.
+//   token_mass_partial_kernel  a block reads a panel of kMassPanel whole rows of P (contiguous
+//                              in memory, so DRAM pages are used in full) and writes the panel's
+//                              weighted column sums;
+//   token_mass_reduce_kernel   adds the panels' sums in a fixed order.
+// (One block per column slab reading all rows at an 8 KB stride measured 2.7 TB/s.)
+constexpr int kMassPanel = 16;
+__global__ void __launch_bounds__(256) token_mass_partial_kernel(const __nv_bfloat16* __restrict__ p,
+                                                                 const float* __restrict__ inv_l, int m_e, int t_e,
+                                                                 int t_ld, int n_panels, float* __restrict__ partial)
 {
-    __shared__ float2 part[8][32];
     wait_for_prior_kernels();
-    const int img = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int col = blockIdx.x * kMassCols + 2 * lane;  // t_ld is even: a column pair never straddles a row
-    const __nv_bfloat16* base = p + (size_t)img * m_e * t_ld + col;
+    const int panel = blockIdx.x, img = blockIdx.y;
+    const int m_begin = panel * kMassPanel, m_end = min(m_begin + kMassPanel, m_e);
     const float* il = inv_l + (size_t)img * m_e;
-    float2 acc = make_float2(0.f, 0.f);
-    if (col < t_ld) {
-#pragma unroll 4
-        for (int m = warp; m < m_e; m += 8) {
-            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(base + (size_t)m * t_ld));
+    float* out = partial + ((size_t)img * n_panels + panel) * t_ld;
+    // thread = 8 consecutive token columns (one 16-byte load per row); t_ld is a multiple of 8
+    for (int c = threadIdx.x * 8; c < t_ld; c += blockDim.x * 8) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        const __nv_bfloat16* col = p + ((size_t)img * m_e + m_begin) * t_ld + c;
+#pragma unroll 8
+        for (int m = m_begin; m < m_end; ++m, col += t_ld) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(col));
             const float w = __ldg(il + m);
-            acc.x += v.x * w;
-            acc.y += v.y * w;
-        }
-    }
-    part[warp][lane] = acc;
-    __syncthreads();
-    if (warp == 0) {
-        float2 s = part[0][lane];
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-        for (int w = 1; w < 8; ++w) { s.x += part[w][lane].x; s.y += part[w][lane].y; }
-        float* out = mass + (size_t)img * t_e;
-        if (col < t_e) out[col] = s.x;
-        if (col + 1 < t_e) out[col + 1] = s.y;
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __bfloat1622float2(h[e]);
+                acc[2 * e] += f.x * w;
+                acc[2 * e + 1] += f.y * w;
+            }
+        }
+        *reinterpret_cast<float4*>(out + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        *reinterpret_cast<float4*>(out + c + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
     }
+}
+
+__global__ void __launch_bounds__(64) token_mass_reduce_kernel(const float* __restrict__ partial, int t_e, int t_ld,
+                                                                int n_panels, float* __restrict__ mass)
+{
+    wait_for_prior_kernels();
+    const int img = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= t_e) return;
+    const float* col = partial + (size_t)img * n_panels * t_ld + i;
+    float acc = 0.f;
+#pragma unroll 16
+    for (int q = 0; q < n_panels; ++q) acc += col[(size_t)q * t_ld];
+    mass[(size_t)img * t_e + i] = acc;
 }
 
 }  // namespace civic

@@ -348,7 +348,8 @@ civic_status_t make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, i
 
 struct AggPlan {
     int32_t t_ld, n_tiles_t, values_bn;
-    size_t q_off, qsum_off, stats_off, p_off, lpart_off, invl_off, total;
+    int32_t n_panels;
+    size_t q_off, qsum_off, stats_off, p_off, lpart_off, invl_off, mass_off, total;
 };
 
 civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d_v, AggPlan& pl)
@@ -359,7 +360,7 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
     pl.n_tiles_t = (t_e + civic::kScoresBN - 1) / civic::kScoresBN;
     pl.values_bn = d_v % 256 == 0 ? 256 : (d_v % 192 == 0 ? 192 : (d_v % 128 == 0 ? 128 : 256));
     const int64_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
-    if (m_tiles * pl.n_tiles_t * n_img > INT32_MAX || m_tiles * ((d_v + 127) / 128) * n_img > INT32_MAX)
+    if (n_img > 65535 || m_tiles * pl.n_tiles_t * n_img > INT32_MAX || m_tiles * ((d_v + 127) / 128) * n_img > INT32_MAX)
         return CIVIC_ERR_UNSUPPORTED;
     size_t off = 0;
     auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
@@ -369,6 +370,8 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
     pl.p_off = take((size_t)n_img * m_e * pl.t_ld * 2);
     pl.lpart_off = take((size_t)n_img * m_e * 2 * pl.n_tiles_t * 4);  // two column halves per token tile
     pl.invl_off = take((size_t)n_img * m_e * 4);
+    pl.n_panels = (m_e + civic::kMassPanel - 1) / civic::kMassPanel;
+    pl.mass_off = take((size_t)n_img * pl.n_panels * pl.t_ld * 4);  // per-panel column sums of the token mass
     pl.total = off;
     return CIVIC_OK;
 }
@@ -561,11 +564,10 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
 
     const bool pdl = programmatic();
     CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
-    CIVIC_CUDA_TRY(civic::launch(pdl, civic::anchor_prep_kernel, (unsigned)((m_e + 7) / 8), 256u, 0, stream, anchors,
-                                 m_e, d_v, 1e-5f, 1e-12f, q, qsum));
     const long long n_tokens = (long long)n_img * t_e;
-    CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_stats_kernel, (unsigned)((n_tokens + 7) / 8), 256u, 0, stream,
-                                 (const __nv_bfloat16*)x0, n_tokens, d_v, 1e-5f, 1e-12f, stats));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::aggregate_prep_kernel, (unsigned)((m_e + n_tokens + 7) / 8), 256u, 0,
+                                 stream, anchors, m_e, (const __nv_bfloat16*)x0, n_tokens, d_v, 1e-5f, 1e-12f, q, qsum,
+                                 stats));
 
     const int32_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
     civic::ScoresParams sp;
@@ -584,20 +586,25 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, vp, vp.grid.total, stream);
     else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, vp, vp.grid.total, stream);
     if (gs != CIVIC_OK) return gs;
-    int n_launched = 4;
+    int n_launched = 3;
     if (token_mass) {
-        CIVIC_CUDA_TRY(cudaGetLastError());
-        const dim3 grid((unsigned)((t_e + civic::kMassCols - 1) / civic::kMassCols), (unsigned)n_img);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.stream = stream;
+        float* partial = (float*)(ws + pl.mass_off);
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.blockDim = dim3(256);
+        cfg.stream = stream;
         cfg.attrs = attr;
         cfg.numAttrs = pdl ? 1 : 0;
-        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::token_mass_kernel, (const __nv_bfloat16*)p, (const float*)inv_l,
-                                          m_e, t_e, pl.t_ld, token_mass));
-        ++n_launched;
+        cfg.gridDim = dim3((unsigned)pl.n_panels, (unsigned)n_img);
+        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::token_mass_partial_kernel, (const __nv_bfloat16*)p,
+                                          (const float*)inv_l, m_e, t_e, pl.t_ld, pl.n_panels, partial));
+        cfg.blockDim = dim3(64);
+        cfg.gridDim = dim3((unsigned)((t_e + 63) / 64), (unsigned)n_img);
+        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::token_mass_reduce_kernel, (const float*)partial, t_e, pl.t_ld,
+                                          pl.n_panels, token_mass));
+        n_launched += 2;
     }
     g_launches.fetch_add(n_launched, std::memory_order_relaxed);
     return CIVIC_OK;
