@@ -128,6 +128,82 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// ---- bulk tensor store of a shared-memory box (one thread issues; OOB parts of the box are clipped)
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(src)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the issuing thread's earlier stores have finished READING shared memory (it may be overwritten)
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
+// ---- two blocks of a cluster working as one MMA unit (cta_group::2).  Block rank 0 (the leader)
+// issues the MMAs; every block loads its half of the operands into its own shared memory, but all
+// transaction bytes are counted on the LEADER's "full" barrier; the leader's commits arrive on
+// the barriers of both blocks (multicast of the commit signal only, never of a load).
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()  // all threads of both blocks
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of `p` (a shared-memory object of this block) in the block of rank `rank`
+__device__ __forceinline__ uint32_t cluster_address(const void* p, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* slot, uint32_t cols)  // the same warp of both blocks
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D (256 rows: 128 in each block's TMEM) (+)= A (128 rows from each block) B (N / 2 columns from each block)
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.u32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// one arrival on the barrier at this shared-memory offset in BOTH blocks, once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar)
+{
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(both) : "memory");
+}
+
 // Shared-memory operand descriptor, 128-byte swizzle, tile base 1024-byte aligned.
 //   K-major  (rows of 64 bf16 = 128 B): 8-row groups 1024 B apart (stride offset); the leading
 //             offset is unused with swizzling (set to one 16-byte unit).
@@ -144,14 +220,14 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t leadi
     d |= 2ull << 61;  // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n; b_mn_major = 1 when B's
-// contiguous dimension is N.
-__host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major)
+// Instruction descriptor: bf16 x bf16 -> fp32, M = m (128, or 256 for a pair of blocks), N = n;
+// b_mn_major = 1 when B's contiguous dimension is N.
+__host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major, int m = kAggBM)
 {
     return (1u << 4)                      // accumulator fp32
            | (1u << 7) | (1u << 10)       // A, B bf16
            | ((uint32_t)b_mn_major << 16) // B major
-           | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kAggBM >> 4) << 24);
+           | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // ----------------------------------------------------------------------------- small kernels
@@ -335,30 +411,46 @@ struct ValuesParams {
 
 constexpr int kEpilogueWarps = 8;
 
-template <int BN_, int STAGES_>
+template <int BN_, int STAGES_, bool SCORES_>
 struct alignas(1024) GemmSmem {
     __nv_bfloat16 a[STAGES_][kAggBM * kAggBK];  // 128 rows x 128 B, K-major
     __nv_bfloat16 b[STAGES_][BN_ * kAggBK];
-    float2 stats[kEpilogueWarps][128];          // per epilogue warp: (mu, r log2e / tau) of its columns (scores only)
+    uint8_t out[SCORES_ ? kEpilogueWarps : 1][SCORES_ ? 32 * 128 : 1024];  // per epilogue warp: 32 rows x 64 bf16, 128-byte swizzled, for
+                                                // the bulk store of the weights (scores only)
+    float2 stats[SCORES_ ? kEpilogueWarps : 1][128];  // per epilogue warp: (mu, r log2e / tau) of its columns (scores only)
     uint64_t full[STAGES_], empty[STAGES_], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
-// S = Q_A X_0^T: tile of 128 anchors x 256 tokens, K = features; both operands K-major.
-struct ScoresOp {
-    static constexpr int BN = 256, STAGES = 4;
+// S = Q_A X_0^T, K = features, both operands K-major.
+//   PAIR = false: one block per tile of 128 anchors x 256 tokens.
+//   PAIR = true:  two blocks of a cluster share a tile of 256 anchors x 256 tokens; each loads its
+//                 own 128 anchors and HALF of the tokens, so a block moves 32 KB per K step
+//                 instead of 48 KB for the same arithmetic (the one-block kernel is bound by the
+//                 bytes it can keep in flight, not by the tensor pipe).
+template <bool PAIR>
+struct ScoresOpT {
+    static constexpr int BN = 256, STAGES = PAIR ? 5 : 3, kCtas = PAIR ? 2 : 1;
     static constexpr bool kBMnMajor = false;
     using Params = ScoresParams;
-    using Smem = GemmSmem<BN, STAGES>;
+    using Smem = GemmSmem<PAIR ? 128 : 256, STAGES, true>;
+    static constexpr uint32_t kStageBytes = (kAggBM + (PAIR ? 128 : 256)) * kAggBK * 2;  // per block
     static __device__ __forceinline__ int k_steps(const Params& p) { return p.d_v / kAggBK; }
+    // m0: this block's first anchor; n0: the tile's first token; rank: block rank in the pair
     static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, int n0, int img)
+                                                int k, int m0, int n0, int img, uint32_t rank, uint32_t leader_full)
     {
-        mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
-        tma_load_2d(sm.a[s], map_a, k * kAggBK, m0, &sm.full[s]);
-        tma_load_3d(sm.b[s], map_b, k * kAggBK, n0, img, &sm.full[s]);                        // tokens n0 ..
-        tma_load_3d(sm.b[s] + 128 * kAggBK, map_b, k * kAggBK, n0 + 128, img, &sm.full[s]);  // .. + 128
+        if constexpr (PAIR) {
+            if (rank == 0) mbar_expect_tx(&sm.full[s], 2 * kStageBytes);  // both blocks' bytes
+            tma_load_2d_pair(sm.a[s], map_a, k * kAggBK, m0, leader_full);
+            tma_load_3d_pair(sm.b[s], map_b, k * kAggBK, n0 + 128 * (int)rank, img, leader_full);
+        } else {
+            mbar_expect_tx(&sm.full[s], kStageBytes);
+            tma_load_2d(sm.a[s], map_a, k * kAggBK, m0, &sm.full[s]);
+            tma_load_3d(sm.b[s], map_b, k * kAggBK, n0, img, &sm.full[s]);                        // tokens n0 ..
+            tma_load_3d(sm.b[s] + 128 * kAggBK, map_b, k * kAggBK, n0 + 128, img, &sm.full[s]);  // .. + 128
+        }
     }
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 32, 16, 1024); }
 
@@ -383,13 +475,12 @@ struct ScoresOp {
         }
     }
 
-    // thread = one anchor row of one half (128 token columns) of the tile
-    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, uint32_t tmem, int ewarp, int lane,
-                                                    int m0, int n0, int img, int n_tile)
+    // Before the accumulator is waited for: the (mu, r log2e / tau) of this warp's 128 token
+    // columns go to the warp's private shared-memory copy (no barrier between warps).
+    static __device__ __forceinline__ void prefetch(const Params& p, Smem& sm, int ewarp, int lane, int n0, int img)
     {
-        const int quarter = ewarp & 3, half = ewarp >> 2;
-        const int nh = n0 + half * 128;  // first token of this warp's columns
-        float2* stats = sm.stats[ewarp];  // private to the warp: no barrier between warps
+        const int nh = n0 + (ewarp >> 2) * 128;
+        float2* stats = sm.stats[ewarp];
         __syncwarp();
 #pragma unroll
         for (int c = lane; c < 128; c += 32) {
@@ -399,41 +490,63 @@ struct ScoresOp {
             stats[c] = st;
         }
         __syncwarp();
+    }
+
+    // thread = one anchor row of one half (128 token columns) of the tile.  The weights leave
+    // through shared memory and a bulk tensor store, 32 rows x 64 columns at a time: whole
+    // 128-byte lines reach L2 (16-byte stores from the registers, one row per lane, measured
+    // 2.5 kcycles per 32 columns: every piece is a memory request of its own).
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap* map_c, uint32_t tmem,
+                                                    int ewarp, int lane, int m0, int n0, int img, int n_tile)
+    {
+        const int quarter = ewarp & 3, half = ewarp >> 2;
+        const int nh = n0 + half * 128;  // first token of this warp's columns
+        const float2* stats = sm.stats[ewarp];
+        uint8_t* out = sm.out[ewarp];
         const int m = m0 + quarter * 32 + lane;
         const bool row_ok = m < p.m_e;
         const float qs = row_ok ? p.qsum[m] : 0.f;
         const float neg_c = -p.inv_tau_log2e;
         float row_sum = 0.f;
-        __nv_bfloat16* out = p.p + ((size_t)img * p.m_e + (row_ok ? m : 0)) * p.t_ld + nh;
         const bool full_tile = nh + 128 <= p.t_e;  // warp-uniform
         for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * 128, 128,
                        [&](const uint32_t (&acc)[32], int c0) {
             uint32_t packed[16];
             if (full_tile) chunk<false>(acc, stats + c0, qs, neg_c, 32, row_sum, packed);
             else chunk<true>(acc, stats + c0, qs, neg_c, p.t_e - nh - c0, row_sum, packed);
-            if (row_ok) {
+            if ((c0 & 32) == 0) {  // first half of a 64-column group: the buffer must be free again
+                if (lane == 0) tma_store_wait_read();
+                __syncwarp();
+            }
+            // row `lane` of the box, 16-byte pieces j = 0..3 (or 4..7) at the swizzled position j ^ (row % 8)
+            const int j0 = (c0 & 32) >> 3;
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)  // 8 columns per 16-byte store; t_ld is a multiple of 8
-                    if (full_tile || nh + c0 + q4 * 8 < p.t_ld)
-                        *reinterpret_cast<uint4*>(out + c0 + q4 * 8) =
-                            make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
+            for (int q4 = 0; q4 < 4; ++q4)
+                *reinterpret_cast<uint4*>(out + lane * 128 + (((j0 + q4) ^ (lane & 7)) << 4)) =
+                    make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
+            if (c0 & 32) {  // the group is complete: hand it to the copy engine
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) tma_store_3d(map_c, out, nh + c0 - 32, m0 + quarter * 32, img);
             }
         });
         if (row_ok) p.lpart[((size_t)img * p.m_e + m) * (2 * p.grid.n_tiles) + 2 * n_tile + half] = row_sum;
     }
 };
+using ScoresOp = ScoresOpT<false>;
+using ScoresPairOp = ScoresOpT<true>;
 
 // Z_0 = (P X_0) / l: tile of 128 anchors x BN features, K = tokens; A = P K-major, B = X_0
 // MN-major (BN / 64 blocks of 64 tokens x 128 B).
 template <int BN_>
 struct ValuesOp {
-    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5;
+    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1;
     static constexpr bool kBMnMajor = true;
     using Params = ValuesParams;
-    using Smem = GemmSmem<BN, STAGES>;
+    using Smem = GemmSmem<BN, STAGES, false>;
     static __device__ __forceinline__ int k_steps(const Params& p) { return (p.t_e + kAggBK - 1) / kAggBK; }
     static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, int n0, int img)
+                                                int k, int m0, int n0, int img, uint32_t, uint32_t)
     {
         mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
         tma_load_3d(sm.a[s], map_a, k * kAggBK, m0, img, &sm.full[s]);
@@ -444,8 +557,10 @@ struct ValuesOp {
     // 16 token rows of 128 B per K step; the next 64 features start one box (8 KB) further on
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
 
-    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, uint32_t tmem, int ewarp, int lane, int m0,
-                                                    int n0, int img, int n_tile)
+    static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, int, int) {}
+
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, const CUtensorMap*, uint32_t tmem, int ewarp,
+                                                    int lane, int m0, int n0, int img, int n_tile)
     {
         constexpr int kHalf = BN / 2;  // 64, 96 or 128 feature columns per warp
         const int quarter = ewarp & 3, half = ewarp >> 2;
@@ -485,9 +600,11 @@ struct ValuesOp {
 template <class Op>
 __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                      const __grid_constant__ CUtensorMap map_b,
+                                                                     const __grid_constant__ CUtensorMap map_c,
                                                                      const typename Op::Params p)
 {
     constexpr int BN = Op::BN, STAGES = Op::STAGES;
+    constexpr bool kPair = Op::kCtas == 2;
     constexpr uint32_t kAccStride = 256;  // TMEM columns between the two accumulators
     extern __shared__ uint8_t smem_raw[];
     using Smem = typename Op::Smem;
@@ -495,17 +612,28 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_steps = Op::k_steps(p);
     volatile int* abort = &sm.abort;
+    // a "worker" is one block, or one pair of blocks; p.grid counts the workers' tiles
+    const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+    const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&sm.acc_full[b], 1); mbar_init(&sm.acc_empty[b], kEpilogueWarps); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.acc_full[b], 1);
+            mbar_init(&sm.acc_empty[b], kEpilogueWarps * Op::kCtas);  // the leader's collects both blocks' warps
+        }
         sm.abort = 0;
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(&sm.tmem_base, 512);
+    if (warp == 1) {
+        if (kPair) tmem_alloc_pair(&sm.tmem_base, 512);
+        else tmem_alloc(&sm.tmem_base, 512);
+    }
     wait_for_prior_kernels();
     tc_fence_before_sync();
     __syncthreads();
+    if (kPair) cluster_sync();  // the partner's barriers exist before anything is signalled on them
     tc_fence_after_sync();
     const uint32_t tmem_base = sm.tmem_base;
     const bool stop = *p.error != 0;  // an earlier block of this launch already failed
@@ -513,33 +641,40 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
     // A wait on the "empty" side uses the opposite parity, so the first pass over a fresh
     // barrier falls through (nothing has to be drained yet).
     if (warp == 0 && lane == 0 && !stop) {
-        // ---- producer
+        // ---- producer (in every block)
         uint32_t it = 0;  // stages issued so far, over all tiles
         bool ok = true;
-        for (int t = blockIdx.x; t < p.grid.total && ok; t += gridDim.x) {
+        for (int t = worker; t < p.grid.total && ok; t += n_workers) {
             int m_tile, n_tile, img;
             tile_coords(p.grid, t, m_tile, n_tile, img);
+            const int m0 = (m_tile * Op::kCtas + (int)rank) * kAggBM;
             for (int k = 0; k < k_steps; ++k, ++it) {
                 const int s = it % STAGES;
                 ok = mbar_wait(&sm.empty[s], ((it / STAGES) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty);
                 if (!ok) break;
-                Op::load(sm, s, &map_a, &map_b, k, m_tile * kAggBM, n_tile * BN, img);
+                Op::load(sm, s, &map_a, &map_b, k, m0, n_tile * BN, img, rank,
+                         kPair ? cluster_address(&sm.full[s], 0) : 0u);
             }
         }
         if (*abort) {  // let the copies already in flight land before the block goes away
-            for (uint32_t j = it > (uint32_t)STAGES ? it - STAGES : 0; j < it; ++j) {
+            if (rank == 0) {
+                for (uint32_t j = it > (uint32_t)STAGES ? it - STAGES : 0; j < it; ++j) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&sm.full[j % STAGES], (j / STAGES) & 1) &&
+                           (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
+                }
+            } else {  // the partner cannot poll the leader's barrier: give its copies ample time
                 const long long t0 = clock64();
-                while (!mbar_try_wait(&sm.full[j % STAGES], (j / STAGES) & 1) &&
-                       (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
+                while ((unsigned long long)(clock64() - t0) < (1ull << 22)) {}
             }
         }
-    } else if (warp == 1 && lane == 0 && !stop) {
-        // ---- MMA issue: 4 instructions of K = 16 per stage
-        constexpr uint32_t idesc = umma_idesc(BN, Op::kBMnMajor ? 1 : 0);
+    } else if (warp == 1 && lane == 0 && !stop && rank == 0) {
+        // ---- MMA issue (leader only): 4 instructions of K = 16 per stage
+        constexpr uint32_t idesc = umma_idesc(BN, Op::kBMnMajor ? 1 : 0, kAggBM * Op::kCtas);
         uint32_t it = 0;
         bool ok = true;
         int local = 0;
-        for (int t = blockIdx.x; t < p.grid.total && ok; t += gridDim.x, ++local) {
+        for (int t = worker; t < p.grid.total && ok; t += n_workers, ++local) {
             const int buf = local & 1;
             ok = mbar_wait(&sm.acc_empty[buf], ((local >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutAcc);
             if (!ok) break;
@@ -552,35 +687,50 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
                 tc_fence_after_sync();
                 const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
 #pragma unroll
-                for (int kk = 0; kk < kAggBK / 16; ++kk)
-                    umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
-                umma_commit(&sm.empty[s]);  // frees the stage once these MMAs have read it
+                for (int kk = 0; kk < kAggBK / 16; ++kk) {
+                    if (kPair) umma_bf16_pair(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                    else umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                }
+                // frees the stage (in both blocks) once these MMAs have read it
+                if (kPair) umma_commit_pair(&sm.empty[s]);
+                else umma_commit(&sm.empty[s]);
             }
-            if (ok) umma_commit(&sm.acc_full[buf]);
+            if (ok) {
+                if (kPair) umma_commit_pair(&sm.acc_full[buf]);
+                else umma_commit(&sm.acc_full[buf]);
+            }
         }
     } else if (warp >= 2 && !stop) {
         // ---- epilogue: warps 2..9; a warp may read the TMEM lane quarter (warp index mod 4)
         const int ewarp = ((warp & 3) | ((warp - 2) & 4));  // quarter in bits 0-1, column half in bit 2
         int local = 0;
-        for (int t = blockIdx.x; t < p.grid.total; t += gridDim.x, ++local) {
+        for (int t = worker; t < p.grid.total; t += n_workers, ++local) {
             int m_tile, n_tile, img;
             tile_coords(p.grid, t, m_tile, n_tile, img);
+            const int m0 = (m_tile * Op::kCtas + (int)rank) * kAggBM;
             const int buf = local & 1;
+            Op::prefetch(p, sm, ewarp, lane, n_tile * BN, img);
             // tcgen05.ld is warp-collective: the whole warp goes on, or none of it
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full[buf], (local >> 1) & 1, abort, p.error, kAggTimeoutAcc)))
                 break;
             tc_fence_after_sync();
-            Op::epilogue(p, sm, tmem_base + buf * kAccStride, ewarp, lane, m_tile * kAggBM, n_tile * BN, img, n_tile);
+            Op::epilogue(p, sm, &map_c, tmem_base + buf * kAccStride, ewarp, lane, m0, n_tile * BN, img, n_tile);
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);  // this warp has drained its part
+            if (lane == 0) {  // this warp has drained its part of the accumulator
+                if (kPair) mbar_arrive_cluster(cluster_address(&sm.acc_empty[buf], 0));
+                else mbar_arrive(&sm.acc_empty[buf]);
+            }
         }
+        if (lane == 0) tma_store_wait_read();  // this warp's bulk stores no longer need its shared memory
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (kPair) cluster_sync();  // neither block leaves while the other may still signal it or read its tiles
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
+        if (kPair) tmem_dealloc_pair(tmem_base, 512);
+        else tmem_dealloc(tmem_base, 512);
     }
 }
 

@@ -377,24 +377,51 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
 }
 
 template <class Op>
-civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const typename Op::Params& params,
-                           int32_t total_tiles, cudaStream_t stream)
+civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c,
+                           const typename Op::Params& params, int32_t total_tiles, cudaStream_t stream)
 {
     const size_t smem = sizeof(typename Op::Smem) + 1024;
     CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_gemm_kernel<Op>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const int sms = sm_count();
+    // persistent: one block per SM, or one pair of blocks (a cluster of two) per two SMs
+    const int workers_max = sm_count() / Op::kCtas;
+    const int workers = total_tiles < workers_max ? total_tiles : workers_max;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(total_tiles < sms ? total_tiles : sms));  // persistent: one block per SM
+    cfg.gridDim = dim3((unsigned)(workers * Op::kCtas));
     cfg.blockDim = dim3(civic::kAggThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (Op::kCtas == 2) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 2;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    if (programmatic()) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = programmatic() ? 1 : 0;
-    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_gemm_kernel<Op>, map_a, map_b, params));
+    cfg.numAttrs = n_attr;
+    if (Op::kCtas == 2) {
+        // not every SM need have a partner free: size the persistent grid to the clusters that
+        // can really be resident together (asked once per device)
+        static std::atomic<int> resident[64];
+        int dev = 0;
+        CIVIC_CUDA_TRY(cudaGetDevice(&dev));
+        int n = dev >= 0 && dev < 64 ? resident[dev].load(std::memory_order_relaxed) : 0;
+        if (n == 0) {
+            CIVIC_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, civic::aggregate_gemm_kernel<Op>, &cfg));
+            if (n < 1) return CIVIC_ERR_UNSUPPORTED;
+            if (dev >= 0 && dev < 64) resident[dev].store(n, std::memory_order_relaxed);
+        }
+        if (workers > n) cfg.gridDim = dim3((unsigned)(n * 2));
+    }
+    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_gemm_kernel<Op>, map_a, map_b, map_c, params));
     return CIVIC_OK;
 }
 
@@ -544,7 +571,7 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     EncodeTiledFn enc = nullptr;
     const civic_status_t est = tensor_map_encoder(&enc);
     if (est != CIVIC_OK) return est;
-    CUtensorMap map_q, map_x_scores, map_p, map_x_values;
+    CUtensorMap map_q, map_x_scores, map_p, map_p_store, map_x_values;
     civic_status_t ms;
     {
         const uint64_t dims[2] = {(uint64_t)d_v, (uint64_t)m_e}, str[1] = {(uint64_t)d_v * 2};
@@ -560,6 +587,7 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
         const uint64_t dims[3] = {(uint64_t)t_e, (uint64_t)m_e, (uint64_t)n_img};
         const uint64_t str[2] = {(uint64_t)pl.t_ld * 2, (uint64_t)m_e * pl.t_ld * 2};
         if ((ms = make_map(enc, &map_p, p, 3, dims, str, civic::kAggBM)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_p_store, p, 3, dims, str, 32)) != CIVIC_OK) return ms;  // 32-row boxes written by a warp
     }
 
     const bool pdl = programmatic();
@@ -572,19 +600,26 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     const int32_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
     civic::ScoresParams sp;
     sp.stats = stats; sp.qsum = qsum; sp.p = p; sp.lpart = lpart; sp.error = device_status;
-    sp.grid = civic::TileGrid{m_tiles, pl.n_tiles_t, n_img, m_tiles * pl.n_tiles_t * n_img};
     sp.m_e = m_e; sp.t_e = t_e; sp.d_v = d_v; sp.t_ld = pl.t_ld;
     sp.inv_tau_log2e = 1.4426950408889634f / tau;
-    civic_status_t gs = launch_gemm<civic::ScoresOp>(map_q, map_x_scores, sp, sp.grid.total, stream);
+    civic_status_t gs;
+    if (m_tiles >= 2) {  // pairs of blocks share tiles of 256 anchors
+        const int32_t m_pairs = (m_tiles + 1) / 2;
+        sp.grid = civic::TileGrid{m_pairs, pl.n_tiles_t, n_img, m_pairs * pl.n_tiles_t * n_img};
+        gs = launch_gemm<civic::ScoresPairOp>(map_q, map_x_scores, map_p_store, sp, sp.grid.total, stream);
+    } else {
+        sp.grid = civic::TileGrid{m_tiles, pl.n_tiles_t, n_img, m_tiles * pl.n_tiles_t * n_img};
+        gs = launch_gemm<civic::ScoresOp>(map_q, map_x_scores, map_p_store, sp, sp.grid.total, stream);
+    }
     if (gs != CIVIC_OK) return gs;
     civic::ValuesParams vp;
     vp.lpart = lpart; vp.z = (__nv_bfloat16*)z0; vp.inv_l = inv_l; vp.error = device_status;
     const int32_t f_tiles = (d_v + pl.values_bn - 1) / pl.values_bn;
     vp.grid = civic::TileGrid{m_tiles, f_tiles, n_img, m_tiles * f_tiles * n_img};
     vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t;
-    if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, vp, vp.grid.total, stream);
-    else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, vp, vp.grid.total, stream);
-    else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, vp, vp.grid.total, stream);
+    if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
+    else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
+    else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
     if (gs != CIVIC_OK) return gs;
     int n_launched = 3;
     if (token_mass) {
