@@ -23,6 +23,9 @@
 // (each reads its own quarter of the 128 TMEM lanes).  Operand tiles arrive by
 // cp.async.bulk.tensor with 128-byte swizzle into a ring of stages guarded by full/empty
 // mbarriers; two accumulators alternate in TMEM so the epilogue overlaps the next tile's MMAs.
+// The score GEMM runs on pairs of blocks (cta_group::2): with both operands in shared memory a
+// single block has to take in and hand out 187 bytes per clock for a 128 x 256 tile, more than
+// shared memory delivers; the pair halves the B traffic.
 // Every wait is bounded: on a time-out the thread raises the kernel's error word, the block
 // stops issuing work, waits (bounded) for its copies in flight, frees its TMEM and returns.
 #pragma once
@@ -332,6 +335,25 @@ __device__ __forceinline__ void tile_coords(const TileGrid& g, int t, int& m_til
     img = rest / g.n_tiles;
 }
 
+// One unit of work of a worker (a block, or a pair of blocks).
+struct Tile {
+    int m_tile;  // anchor tile of the worker: 128 anchors per block
+    int n0, n;   // first column and width of the tile (tokens for the scores, features for the values)
+    int n_tile;  // column tile number
+    int img;
+};
+
+// i-th tile of a worker, tiles of one width dealt out round-robin
+__device__ __forceinline__ bool round_robin_tile(const TileGrid& g, int width, int worker, int n_workers, int i, Tile& tl)
+{
+    const int t = worker + i * n_workers;
+    if (t >= g.total) return false;
+    tile_coords(g, t, tl.m_tile, tl.n_tile, tl.img);
+    tl.n0 = tl.n_tile * width;
+    tl.n = width;
+    return true;
+}
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -437,10 +459,15 @@ struct ScoresOpT {
     using Smem = GemmSmem<PAIR ? 128 : 256, STAGES, true>;
     static constexpr uint32_t kStageBytes = (kAggBM + (PAIR ? 128 : 256)) * kAggBK * 2;  // per block
     static __device__ __forceinline__ int k_steps(const Params& p) { return p.d_v / kAggBK; }
-    // m0: this block's first anchor; n0: the tile's first token; rank: block rank in the pair
-    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, int n0, int img, uint32_t rank, uint32_t leader_full)
+    static __device__ __forceinline__ bool tile(const Params& p, int worker, int n_workers, int i, Tile& tl)
     {
+        return round_robin_tile(p.grid, BN, worker, n_workers, i, tl);
+    }
+    // m0: this block's first anchor; rank: block rank in the pair
+    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
+                                                int k, int m0, const Tile& tl, uint32_t rank, uint32_t leader_full)
+    {
+        const int n0 = tl.n0, img = tl.img;
         if constexpr (PAIR) {
             if (rank == 0) mbar_expect_tx(&sm.full[s], 2 * kStageBytes);  // both blocks' bytes
             tma_load_2d_pair(sm.a[s], map_a, k * kAggBK, m0, leader_full);
@@ -477,9 +504,10 @@ struct ScoresOpT {
 
     // Before the accumulator is waited for: the (mu, r log2e / tau) of this warp's 128 token
     // columns go to the warp's private shared-memory copy (no barrier between warps).
-    static __device__ __forceinline__ void prefetch(const Params& p, Smem& sm, int ewarp, int lane, int n0, int img)
+    static __device__ __forceinline__ void prefetch(const Params& p, Smem& sm, int ewarp, int lane, const Tile& tl)
     {
-        const int nh = n0 + (ewarp >> 2) * 128;
+        const int img = tl.img;
+        const int nh = tl.n0 + (ewarp >> 2) * 128;
         float2* stats = sm.stats[ewarp];
         __syncwarp();
 #pragma unroll
@@ -497,10 +525,11 @@ struct ScoresOpT {
     // 128-byte lines reach L2 (16-byte stores from the registers, one row per lane, measured
     // 2.5 kcycles per 32 columns: every piece is a memory request of its own).
     static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap* map_c, uint32_t tmem,
-                                                    int ewarp, int lane, int m0, int n0, int img, int n_tile)
+                                                    int ewarp, int lane, int m0, const Tile& tl)
     {
+        const int img = tl.img, n_tile = tl.n_tile;
         const int quarter = ewarp & 3, half = ewarp >> 2;
-        const int nh = n0 + half * 128;  // first token of this warp's columns
+        const int nh = tl.n0 + half * 128;  // first token of this warp's columns
         const float2* stats = sm.stats[ewarp];
         uint8_t* out = sm.out[ewarp];
         const int m = m0 + quarter * 32 + lane;
@@ -536,8 +565,48 @@ struct ScoresOpT {
 using ScoresOp = ScoresOpT<false>;
 using ScoresPairOp = ScoresOpT<true>;
 
-// Z_0 = (P X_0) / l: tile of 128 anchors x BN features, K = tokens; A = P K-major, B = X_0
-// MN-major (BN / 64 blocks of 64 tokens x 128 B).
+// Z_0 = (P X_0) / l, K = tokens; A = P K-major, B = X_0 MN-major (blocks of 64 tokens x 128 B, one
+// per 64 features, 8 KB apart).  One block per tile of 128 anchors x BN features (BN = 128, 192 or
+// 256).  A pair version (256 anchors x 256 features, a last tile of 128, tiles dealt out widest
+// first in serpentine order) ran 15 % fewer cycles per tile but no faster in time on the
+// power-capped GPU (184.4 vs 184.8 us per call), so the simpler kernel stayed.
+__device__ __forceinline__ void values_epilogue(const ValuesParams& p, uint32_t tmem, int ewarp, int lane, int m0,
+                                                const Tile& tl)
+{
+    const int half_cols = tl.n >> 1;  // 64, 96 or 128 feature columns per warp
+    const int quarter = ewarp & 3, half = ewarp >> 2;
+    const int m = m0 + quarter * 32 + lane;
+    const bool row_ok = m < p.m_e;
+    float l = 0.f;  // the row's partial sums from the first GEMM
+    if (row_ok) {
+        const float* lp = p.lpart + ((size_t)tl.img * p.m_e + m) * p.n_parts;
+        for (int t = 0; t < p.n_parts; ++t) l += lp[t];
+    }
+    const float inv_l = l > 0.f ? 1.f / l : 0.f;
+    if (row_ok && tl.n0 == 0 && half == 0) p.inv_l[(size_t)tl.img * p.m_e + m] = inv_l;
+    const int nh = tl.n0 + half * half_cols;
+    __nv_bfloat16* out = p.z + ((size_t)tl.img * p.m_e + (row_ok ? m : 0)) * p.d_v + nh;
+    for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * half_cols, half_cols,
+                   [&](const uint32_t (&acc)[32], int c0) {
+        if (row_ok) {
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                if (nh + c0 + q4 * 8 < p.d_v) {  // d_v is a multiple of 8
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const __nv_bfloat162 h =
+                            __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv_l,
+                                                  __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv_l);
+                        w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+    });
+}
+
 template <int BN_>
 struct ValuesOp {
     static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1;
@@ -545,55 +614,26 @@ struct ValuesOp {
     using Params = ValuesParams;
     using Smem = GemmSmem<BN, STAGES, false>;
     static __device__ __forceinline__ int k_steps(const Params& p) { return (p.t_e + kAggBK - 1) / kAggBK; }
+    static __device__ __forceinline__ bool tile(const Params& p, int worker, int n_workers, int i, Tile& tl)
+    {
+        return round_robin_tile(p.grid, BN, worker, n_workers, i, tl);
+    }
     static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, int n0, int img, uint32_t, uint32_t)
+                                                int k, int m0, const Tile& tl, uint32_t, uint32_t)
     {
         mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
-        tma_load_3d(sm.a[s], map_a, k * kAggBK, m0, img, &sm.full[s]);
+        tma_load_3d(sm.a[s], map_a, k * kAggBK, m0, tl.img, &sm.full[s]);
 #pragma unroll
         for (int j = 0; j < BN / 64; ++j)  // 64 features x 64 tokens per box
-            tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_b, n0 + j * 64, k * kAggBK, img, &sm.full[s]);
+            tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_b, tl.n0 + j * 64, k * kAggBK, tl.img, &sm.full[s]);
     }
     // 16 token rows of 128 B per K step; the next 64 features start one box (8 KB) further on
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
-
-    static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, int, int) {}
-
+    static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, const Tile&) {}
     static __device__ __forceinline__ void epilogue(const Params& p, Smem&, const CUtensorMap*, uint32_t tmem, int ewarp,
-                                                    int lane, int m0, int n0, int img, int n_tile)
+                                                    int lane, int m0, const Tile& tl)
     {
-        constexpr int kHalf = BN / 2;  // 64, 96 or 128 feature columns per warp
-        const int quarter = ewarp & 3, half = ewarp >> 2;
-        const int m = m0 + quarter * 32 + lane;
-        const bool row_ok = m < p.m_e;
-        float l = 0.f;  // the row's partial sums from the first GEMM
-        if (row_ok) {
-            const float* lp = p.lpart + ((size_t)img * p.m_e + m) * p.n_parts;
-            for (int t = 0; t < p.n_parts; ++t) l += lp[t];
-        }
-        const float inv_l = l > 0.f ? 1.f / l : 0.f;
-        if (row_ok && n_tile == 0 && half == 0) p.inv_l[(size_t)img * p.m_e + m] = inv_l;
-        const int nh = n0 + half * kHalf;
-        __nv_bfloat16* out = p.z + ((size_t)img * p.m_e + (row_ok ? m : 0)) * p.d_v + nh;
-        for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * kHalf, kHalf,
-                       [&](const uint32_t (&acc)[32], int c0) {
-            if (row_ok) {
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    if (nh + c0 + q4 * 8 < p.d_v) {  // d_v is a multiple of 8
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const __nv_bfloat162 h =
-                                __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv_l,
-                                                      __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv_l);
-                            w[e] = *reinterpret_cast<const uint32_t*>(&h);
-                        }
-                        *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                }
-            }
-        });
+        values_epilogue(p, tmem, ewarp, lane, m0, tl);
     }
 };
 
@@ -603,7 +643,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
                                                                      const __grid_constant__ CUtensorMap map_c,
                                                                      const typename Op::Params p)
 {
-    constexpr int BN = Op::BN, STAGES = Op::STAGES;
+    constexpr int STAGES = Op::STAGES;
     constexpr bool kPair = Op::kCtas == 2;
     constexpr uint32_t kAccStride = 256;  // TMEM columns between the two accumulators
     extern __shared__ uint8_t smem_raw[];
@@ -644,16 +684,14 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
         // ---- producer (in every block)
         uint32_t it = 0;  // stages issued so far, over all tiles
         bool ok = true;
-        for (int t = worker; t < p.grid.total && ok; t += n_workers) {
-            int m_tile, n_tile, img;
-            tile_coords(p.grid, t, m_tile, n_tile, img);
-            const int m0 = (m_tile * Op::kCtas + (int)rank) * kAggBM;
+        Tile tl;
+        for (int i = 0; ok && Op::tile(p, worker, n_workers, i, tl); ++i) {
+            const int m0 = (tl.m_tile * Op::kCtas + (int)rank) * kAggBM;
             for (int k = 0; k < k_steps; ++k, ++it) {
                 const int s = it % STAGES;
                 ok = mbar_wait(&sm.empty[s], ((it / STAGES) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty);
                 if (!ok) break;
-                Op::load(sm, s, &map_a, &map_b, k, m0, n_tile * BN, img, rank,
-                         kPair ? cluster_address(&sm.full[s], 0) : 0u);
+                Op::load(sm, s, &map_a, &map_b, k, m0, tl, rank, kPair ? cluster_address(&sm.full[s], 0) : 0u);
             }
         }
         if (*abort) {  // let the copies already in flight land before the block goes away
@@ -670,11 +708,11 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
         }
     } else if (warp == 1 && lane == 0 && !stop && rank == 0) {
         // ---- MMA issue (leader only): 4 instructions of K = 16 per stage
-        constexpr uint32_t idesc = umma_idesc(BN, Op::kBMnMajor ? 1 : 0, kAggBM * Op::kCtas);
         uint32_t it = 0;
         bool ok = true;
-        int local = 0;
-        for (int t = worker; t < p.grid.total && ok; t += n_workers, ++local) {
+        Tile tl;
+        for (int local = 0; ok && Op::tile(p, worker, n_workers, local, tl); ++local) {
+            const uint32_t idesc = umma_idesc(tl.n, Op::kBMnMajor ? 1 : 0, kAggBM * Op::kCtas);
             const int buf = local & 1;
             ok = mbar_wait(&sm.acc_empty[buf], ((local >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutAcc);
             if (!ok) break;
@@ -703,18 +741,16 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
     } else if (warp >= 2 && !stop) {
         // ---- epilogue: warps 2..9; a warp may read the TMEM lane quarter (warp index mod 4)
         const int ewarp = ((warp & 3) | ((warp - 2) & 4));  // quarter in bits 0-1, column half in bit 2
-        int local = 0;
-        for (int t = worker; t < p.grid.total; t += n_workers, ++local) {
-            int m_tile, n_tile, img;
-            tile_coords(p.grid, t, m_tile, n_tile, img);
-            const int m0 = (m_tile * Op::kCtas + (int)rank) * kAggBM;
+        Tile tl;
+        for (int local = 0; Op::tile(p, worker, n_workers, local, tl); ++local) {
+            const int m0 = (tl.m_tile * Op::kCtas + (int)rank) * kAggBM;
             const int buf = local & 1;
-            Op::prefetch(p, sm, ewarp, lane, n_tile * BN, img);
+            Op::prefetch(p, sm, ewarp, lane, tl);
             // tcgen05.ld is warp-collective: the whole warp goes on, or none of it
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full[buf], (local >> 1) & 1, abort, p.error, kAggTimeoutAcc)))
                 break;
             tc_fence_after_sync();
-            Op::epilogue(p, sm, &map_c, tmem_base + buf * kAccStride, ewarp, lane, m0, n_tile * BN, img, n_tile);
+            Op::epilogue(p, sm, &map_c, tmem_base + buf * kAccStride, ewarp, lane, m0, tl);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {  // this warp has drained its part of the accumulator

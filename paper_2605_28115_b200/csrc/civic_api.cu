@@ -614,9 +614,9 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     if (gs != CIVIC_OK) return gs;
     civic::ValuesParams vp;
     vp.lpart = lpart; vp.z = (__nv_bfloat16*)z0; vp.inv_l = inv_l; vp.error = device_status;
+    vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t;
     const int32_t f_tiles = (d_v + pl.values_bn - 1) / pl.values_bn;
     vp.grid = civic::TileGrid{m_tiles, f_tiles, n_img, m_tiles * f_tiles * n_img};
-    vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t;
     if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
     else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
     else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);

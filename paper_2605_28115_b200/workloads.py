@@ -271,8 +271,9 @@ class AggWorkload:
 # tokens of the batch-8 selection workload), vision width 1152, 1024 anchors (256 compact tokens
 # after the 2x2 merger), temperature 0.07.
 AGG_896 = AggWorkload("agg_batch8_896", 8, 4096, 1024, 1152, 0.07)
+AGG_896_X2 = AggWorkload("agg_batch2_896", 2, 4096, 1024, 1152, 0.07)  # a quarter of it, for profiler captures
 AGG_448 = AggWorkload("agg_single_448", 1, 1024, 256, 1152, 0.07)
-AGG_BY_NAME = {w.name: w for w in (AGG_896, AGG_448)}
+AGG_BY_NAME = {w.name: w for w in (AGG_896, AGG_896_X2, AGG_448)}
 
 
 def agg_inputs(w: AggWorkload, device="cpu"):
