@@ -59,6 +59,9 @@ def parse_args():
     ap.add_argument("--merge", action="store_true",
                     help="also build the compact prefill sequence (Eq. 13 merge of text and kept visual "
                          "rows) and its plane-major position ids in every step")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one step in a CUDA graph and time its replays: the GPU-side latency of the "
+                         "step without the Python binding's per-call host time (for the small workloads)")
     ap.add_argument("--layers", type=int, default=0,
                     help="shrink the workload to this many K/V layers (profiling a small case); "
                          "the JSON line then names the reduced workload")
@@ -97,7 +100,8 @@ def config_of(wl, extra=None):
            "scores": wl.score_kind, "hidden_dim": wl.hidden_dim, "layers": wl.n_layers,
            "kv_row_bytes": wl.kv_row_bytes, "seq_len": wl.seq_len, "s_out": wl.s_out,
            "text_tokens": [wl.text_before, wl.text_after],
-           "l2": "inputs larger than L2: each step streams the whole K/V set through it, no flush"}
+           "l2": ("inputs larger than L2: each step streams the whole K/V set through it, no flush" if wl.n_layers
+                  else "working set smaller than L2 and not flushed: a latency figure, not a bandwidth figure")}
     if extra:
         cfg.update(extra)
     return cfg
@@ -442,6 +446,20 @@ def run_civic(args):
     stride = max(1, min(KV_EVENT_STRIDE, args.steps // 20))
     kv_ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
              for i in range(0, args.steps, stride)} if wl.n_layers else None
+    graph, launches_per_replay = None, 0
+    if args.graph:
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            st.step()
+            torch.cuda.synchronize()
+            before_capture = civic.launch_count()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                st.step()
+            launches_per_replay = civic.launch_count() - before_capture
+        for _ in range(3):
+            graph.replay()
+        kv_ev = None  # no events inside a graph: the roofline object needs the plain mode
     sampler = ClockSampler(local_rank)
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = civic.launch_count()
@@ -449,11 +467,14 @@ def run_civic(args):
     barrier()
     start.record()
     for i in range(args.steps):
-        st.step(kv_ev.get(i) if kv_ev else None)
+        if graph is not None:
+            graph.replay()
+        else:
+            st.step(kv_ev.get(i) if kv_ev else None)
     end.record()
     barrier()
     clocks = sampler.stop()
-    launches = civic.launch_count() - launches0
+    launches = launches_per_replay * args.steps if graph is not None else civic.launch_count() - launches0
     ms_per_step = sharding.max_over_ranks(start.elapsed_time(end), dev) / args.steps
     value = sharding.job_throughput_gbs(nbytes["total"], world, ms_per_step)
 
@@ -516,6 +537,7 @@ def run_civic(args):
                 "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "u8", "data": "synthetic",
                 "config": config_of(wl, {"parallelism": f"dp{world}" if world > 1 else "single",
+                                         "cuda_graph": graph is not None,
                                          "kv_layout": args.kv_layout, "merge": st.merge,
                                          **({} if default_variant else {"workload": wl.name + (
                                              "" if args.kv_layout == "token_major" else "+" + args.kv_layout)
