@@ -68,3 +68,47 @@ def anchor_aggregate_batch(x0: np.ndarray, anchors: np.ndarray, tau: float):
         z.append(z_i)
         mass.append(w_i.sum(axis=0))
     return np.stack(z), np.stack(mass)
+
+
+# ---------------------------------------------------------------------------------------------
+# Compact visual encoding layer: KV-compressed attention (Eq. 9)
+#
+#     Q = H W_Q,  K = H W_K,  V = H W_V
+#     K_c = Rbar^T K,  V_c = Rbar^T V           Rbar = R with every column normalised
+#     Attn_c = softmax(Q K_c^T / sqrt(d)) V_c   per head, d the per-head dimension
+#
+# H [M_e, D_v] are the compact hidden states, R [M_e, S] the KV assignment matrix onto S memory
+# anchors.  Readings where the paper is silent: R is non-negative and "column-normalised" means
+# every column is divided by its sum, so a row of K_c is a weighted average of the rows of K;
+# heads split the feature dimension into n_heads contiguous blocks of d = D_v / n_heads, K_c and
+# V_c are compressed over the whole feature dimension at once (R does not depend on the head);
+# the softmax runs over the S memory anchors; no output projection (Eq. 9 has none).
+
+def column_normalize(r: np.ndarray) -> np.ndarray:
+    r = np.asarray(r, dtype=np.float64)
+    return r / r.sum(axis=0, keepdims=True)
+
+
+def kv_compressed_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, r: np.ndarray, n_heads: int):
+    """q, k, v [M_e, D] (already projected), r [M_e, S] -> (Attn_c [M_e, D], K_c [S, D], V_c [S, D])."""
+    q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
+    m_e, dim = q.shape
+    d = dim // n_heads
+    rbar = column_normalize(r)
+    k_c = rbar.T @ k
+    v_c = rbar.T @ v
+    out = np.empty_like(q)
+    for h in range(n_heads):
+        cols = slice(h * d, (h + 1) * d)
+        logits = q[:, cols] @ k_c[:, cols].T / np.sqrt(d)
+        logits = logits - logits.max(axis=1, keepdims=True)  # softmax over the S memory anchors
+        e = np.exp(logits)
+        out[:, cols] = (e / e.sum(axis=1, keepdims=True)) @ v_c[:, cols]
+    return out, k_c, v_c
+
+
+def compact_visual_layer(h: np.ndarray, w_q: np.ndarray, w_k: np.ndarray, w_v: np.ndarray, r: np.ndarray,
+                         n_heads: int) -> np.ndarray:
+    """Eq. 9 from the hidden states: projections, then the KV-compressed attention."""
+    h = np.asarray(h, dtype=np.float64)
+    return kv_compressed_attention(h @ w_q, h @ w_k, h @ w_v, r, n_heads)[0]

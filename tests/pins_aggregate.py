@@ -115,3 +115,84 @@ def pin_batch_and_mass(agg):
 
 ALL_AGGREGATE_PINS = [pin_two_feature_closed_form, pin_library_routines, pin_convexity_and_limits,
                       pin_invariances, pin_layer_norm_and_norm, pin_batch_and_mass]
+
+
+# ---------------------------------------------------------------- KV-compressed attention (Eq. 9)
+
+def _dense_attention(q, k, v, n_heads):
+    """Ordinary multi-head attention from library routines (scipy softmax)."""
+    from scipy.special import softmax
+
+    d = q.shape[1] // n_heads
+    out = np.empty_like(q)
+    for h in range(n_heads):
+        c = slice(h * d, (h + 1) * d)
+        out[:, c] = softmax(q[:, c] @ k[:, c].T / np.sqrt(d), axis=1) @ v[:, c]
+    return out
+
+
+def pin_identity_assignment_is_dense_attention(agg):
+    """S = M_e and R = identity (or any permutation of it, or a positive diagonal): nothing is
+    compressed, Eq. 9 is ordinary attention over the compact tokens themselves."""
+    rng = np.random.default_rng(81)
+    m_e, dim, heads = 12, 8, 2
+    q, k, v = (rng.standard_normal((m_e, dim)) for _ in range(3))
+    want = _dense_attention(q, k, v, heads)
+    out, k_c, v_c = agg.kv_compressed_attention(q, k, v, np.eye(m_e), heads)
+    assert np.allclose(out, want, rtol=1e-12, atol=1e-14) and np.allclose(k_c, k) and np.allclose(v_c, v)
+    perm = rng.permutation(m_e)
+    out_p, k_p, _ = agg.kv_compressed_attention(q, k, v, np.eye(m_e)[:, perm], heads)
+    assert np.allclose(out_p, want, rtol=1e-12, atol=1e-14) and np.allclose(k_p, k[perm])
+    out_d, _, _ = agg.kv_compressed_attention(q, k, v, np.diag(rng.uniform(0.5, 3.0, m_e)), heads)
+    assert np.allclose(out_d, want, rtol=1e-12, atol=1e-14), "column normalisation removes a column's scale"
+
+
+def pin_compression_closed_forms(agg):
+    rng = np.random.default_rng(83)
+    m_e, dim, heads, s = 10, 6, 3, 4
+    q, k, v = (rng.standard_normal((m_e, dim)) for _ in range(3))
+    # one memory anchor that every token feeds equally: K_c, V_c are the means, every query returns mean(V)
+    out, k_c, v_c = agg.kv_compressed_attention(q, k, v, np.ones((m_e, 1)), heads)
+    assert np.allclose(k_c[0], k.mean(axis=0)) and np.allclose(v_c[0], v.mean(axis=0))
+    assert np.allclose(out, np.tile(v.mean(axis=0), (m_e, 1)))
+    # hard assignment: anchor j averages exactly the tokens assigned to it
+    assign = rng.integers(0, s, m_e)
+    assign[:s] = np.arange(s)  # no empty anchor
+    r = np.zeros((m_e, s))
+    r[np.arange(m_e), assign] = 1.0
+    out, k_c, v_c = agg.kv_compressed_attention(q, k, v, r, heads)
+    for j in range(s):
+        assert np.allclose(k_c[j], k[assign == j].mean(axis=0)) and np.allclose(v_c[j], v[assign == j].mean(axis=0))
+    assert np.allclose(out, _dense_attention(q, k_c, v_c, heads), rtol=1e-12, atol=1e-14)
+    # the columns of the normalised assignment sum to one; outputs are convex combinations of V_c rows
+    rbar = agg.column_normalize(rng.uniform(0.1, 1.0, (m_e, s)))
+    assert np.allclose(rbar.sum(axis=0), 1.0)
+    assert np.all(out <= v_c.max(axis=0) + 1e-12) and np.all(out >= v_c.min(axis=0) - 1e-12)
+    # hand-worked: two tokens, one head of size 1, two anchors with R = [[1, 1], [0, 1]]
+    q1, k1, v1 = np.array([[1.0], [0.0]]), np.array([[2.0], [4.0]]), np.array([[10.0], [20.0]])
+    out1, kc1, vc1 = agg.kv_compressed_attention(q1, k1, v1, np.array([[1.0, 1.0], [0.0, 1.0]]), 1)
+    assert np.allclose(kc1[:, 0], [2.0, 3.0]) and np.allclose(vc1[:, 0], [10.0, 15.0])
+    w = np.exp([2.0, 3.0]) / np.exp([2.0, 3.0]).sum()  # query 1 . K_c / sqrt(1)
+    assert np.allclose(out1[:, 0], [w @ [10.0, 15.0], 12.5])  # the zero query weighs both anchors equally
+
+
+def pin_layer_composition(agg):
+    """Eq. 9 from the hidden states is the attention of the three projections; heads do not mix."""
+    rng = np.random.default_rng(87)
+    m_e, dim, heads, s = 9, 8, 4, 3
+    h = rng.standard_normal((m_e, dim))
+    w_q, w_k, w_v = (rng.standard_normal((dim, dim)) for _ in range(3))
+    r = rng.uniform(0.1, 1.0, (m_e, s))
+    full = agg.compact_visual_layer(h, w_q, w_k, w_v, r, heads)
+    want, _, _ = agg.kv_compressed_attention(h @ w_q, h @ w_k, h @ w_v, r, heads)
+    assert np.allclose(full, want)
+    d = dim // heads
+    q, k, v = h @ w_q, h @ w_k, h @ w_v
+    k2 = k.copy()
+    k2[:, d:2 * d] *= -2.0  # changing head 1's keys leaves the other heads' outputs untouched
+    out2, _, _ = agg.kv_compressed_attention(q, k2, v, r, heads)
+    assert np.allclose(out2[:, :d], want[:, :d]) and np.allclose(out2[:, 2 * d:], want[:, 2 * d:])
+    assert not np.allclose(out2[:, d:2 * d], want[:, d:2 * d])
+
+
+ALL_ATTENTION_PINS = [pin_identity_assignment_is_dense_attention, pin_compression_closed_forms, pin_layer_composition]
