@@ -353,6 +353,37 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
 /* Scratch bytes civic_anchor_aggregate needs; 0 if the shape is invalid or unsupported. */
 size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d_v);
 
+/*
+ * civic_kv_compressed_attention -- attention of the compact visual encoder with compressed keys
+ * and values.
+ *
+ * Paper: Eq. 9 (Section 3.4), for already projected Q = H W_Q, K = H W_K, V = H W_V (the three
+ * projections are plain GEMMs and are left to the caller's BLAS):
+ *     K_c = Rbar^T K,  V_c = Rbar^T V,  Attn_c = softmax(Q K_c^T / sqrt(d)) V_c   per head,
+ * R [m_e, s] the KV assignment matrix onto s memory anchors (non-negative, every column with a
+ * positive sum), Rbar = R with every column divided by its sum, d = head_dim.  Heads split the
+ * feature dimension into n_heads contiguous blocks of head_dim; the softmax runs over the s
+ * anchors.  bf16 tensor-core products with fp32 accumulation; K_c, V_c and the softmax weights
+ * are rounded to bf16 on the way.
+ *
+ * q, k, v        dev  bf16 [n_img, m_e, n_heads * head_dim], 16-byte aligned
+ * r              dev  fp32 [m_e, s], shared by the images
+ * out            dev  bf16 [n_img, m_e, n_heads * head_dim], written
+ * workspace      dev  scratch of civic_kv_compressed_attention_workspace_bytes(...) bytes,
+ *                256-byte aligned (R in bf16, its column sums, K_c and V_c)
+ * device_status  dev  int32, written: 0, or non-zero if a wait inside a kernel hit its time limit
+ * head_dim must be 64 or 128 and s a multiple of 64 up to 256: CIVIC_ERR_UNSUPPORTED otherwise.
+ * Four launches and a 4-byte memset.
+ */
+civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const void* v, const float* r,
+                                             int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                             int32_t s, void* out, void* workspace, size_t workspace_bytes,
+                                             int32_t* device_status, void* stream);
+
+/* Scratch bytes civic_kv_compressed_attention needs; 0 if the shape is invalid or unsupported. */
+size_t civic_kv_compressed_attention_workspace_bytes(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                                     int32_t s);
+
 /* Static, human-readable name of a status. */
 const char* civic_status_string(civic_status_t status);
 

@@ -30,7 +30,8 @@ EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "c
            "civic_compact_pos_planes", "civic_select_large", "civic_select_workspace_bytes",
            "civic_select_ragged", "civic_floor_from_ratio",
            "civic_select_large_static", "civic_select_static_scratch_bytes",
-           "civic_anchor_aggregate", "civic_anchor_aggregate_workspace_bytes")
+           "civic_anchor_aggregate", "civic_anchor_aggregate_workspace_bytes",
+           "civic_kv_compressed_attention", "civic_kv_compressed_attention_workspace_bytes")
 
 
 class CivicError(RuntimeError):
@@ -109,6 +110,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_anchor_aggregate.restype = ctypes.c_int
     lib.civic_anchor_aggregate_workspace_bytes.argtypes = [i32, i32, i32, i32]
     lib.civic_anchor_aggregate_workspace_bytes.restype = sz
+    lib.civic_kv_compressed_attention.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.civic_kv_compressed_attention.restype = ctypes.c_int
+    lib.civic_kv_compressed_attention_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.civic_kv_compressed_attention_workspace_bytes.restype = sz
     _lib = lib
     return lib
 
@@ -583,3 +588,38 @@ def civic_anchor_aggregate(x0: torch.Tensor, anchors: torch.Tensor, tau: float,
     with torch.cuda.device(dev):
         _check(load().civic_anchor_aggregate(*args, _stream_ptr(stream)), "civic_anchor_aggregate")
     return z0, token_mass, device_status
+
+
+def kv_compressed_attention_workspace_bytes(n_img: int, m_e: int, n_heads: int, head_dim: int, s: int) -> int:
+    return int(load().civic_kv_compressed_attention_workspace_bytes(n_img, m_e, n_heads, head_dim, s))
+
+
+def civic_kv_compressed_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, r: torch.Tensor, n_heads: int,
+                                  out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                  device_status: Optional[torch.Tensor] = None,
+                                  stream: Optional[torch.cuda.Stream] = None):
+    """Eq. 9 for projected q, k, v bf16 [n_img, m_e, n_heads * d] and the assignment r fp32 [m_e, s] ->
+    (attention output bf16 [n_img, m_e, n_heads * d], device_status int32 [1]: 0 after a clean run)."""
+    if q.dim() != 3 or q.shape != k.shape or q.shape != v.shape or r.dim() != 2 or r.shape[0] != q.shape[1]:
+        raise ValueError("q, k, v must be [n_img, m_e, D] and r [m_e, s]")
+    n_img, m_e, dim = q.shape
+    if dim % n_heads:
+        raise ValueError("the feature dimension must be a multiple of n_heads")
+    head_dim, s = dim // n_heads, r.shape[1]
+    dev = _device_of(q)
+    if out is None:
+        out = torch.empty_like(q)
+    elif out.shape != q.shape:
+        raise ValueError("out must have q's shape")
+    if workspace is None:
+        workspace = torch.empty(max(kv_compressed_attention_workspace_bytes(n_img, m_e, n_heads, head_dim, s), 256),
+                                dtype=torch.uint8, device=dev)
+    if device_status is None:
+        device_status = torch.empty((1,), dtype=torch.int32, device=dev)
+    args = (_dev_ptr(q, "q", torch.bfloat16), _dev_ptr(k, "k", torch.bfloat16), _dev_ptr(v, "v", torch.bfloat16),
+            _dev_ptr(r, "r", torch.float32), n_img, m_e, n_heads, head_dim, s, _dev_ptr(out, "out", torch.bfloat16),
+            _dev_ptr(workspace, "workspace", torch.uint8), workspace.numel(),
+            _dev_ptr(device_status, "device_status", torch.int32))
+    with torch.cuda.device(dev):
+        _check(load().civic_kv_compressed_attention(*args, _stream_ptr(stream)), "civic_kv_compressed_attention")
+    return out, device_status

@@ -224,11 +224,12 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr, uint32_t leadi
     return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = m (128, or 256 for a pair of blocks), N = n;
-// b_mn_major = 1 when B's contiguous dimension is N.
-__host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major, int m = kAggBM)
+// a_mn_major / b_mn_major = 1 when the operand's contiguous dimension is M / N rather than K.
+__host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major, int m = kAggBM, int a_mn_major = 0)
 {
     return (1u << 4)                      // accumulator fp32
            | (1u << 7) | (1u << 10)       // A, B bf16
+           | ((uint32_t)a_mn_major << 15) // A major
            | ((uint32_t)b_mn_major << 16) // B major
            | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
@@ -454,7 +455,7 @@ struct alignas(1024) GemmSmem {
 template <bool PAIR>
 struct ScoresOpT {
     static constexpr int BN = 256, STAGES = PAIR ? 5 : 3, kCtas = PAIR ? 2 : 1;
-    static constexpr bool kBMnMajor = false;
+    static constexpr bool kAMnMajor = false, kBMnMajor = false;
     using Params = ScoresParams;
     using Smem = GemmSmem<PAIR ? 128 : 256, STAGES, true>;
     static constexpr uint32_t kStageBytes = (kAggBM + (PAIR ? 128 : 256)) * kAggBK * 2;  // per block
@@ -479,6 +480,7 @@ struct ScoresOpT {
             tma_load_3d(sm.b[s] + 128 * kAggBK, map_b, k * kAggBK, n0 + 128, img, &sm.full[s]);  // .. + 128
         }
     }
+    static __device__ __forceinline__ uint64_t a_desc(uint32_t a0, int kk) { return umma_desc(a0 + kk * 32, 16, 1024); }
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 32, 16, 1024); }
 
     // P = 2^(r' (acc - mu qsum) - c) for 32 columns of one anchor row, r' = r c, c = log2(e) / tau;
@@ -610,7 +612,7 @@ __device__ __forceinline__ void values_epilogue(const ValuesParams& p, uint32_t 
 template <int BN_>
 struct ValuesOp {
     static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1;
-    static constexpr bool kBMnMajor = true;
+    static constexpr bool kAMnMajor = false, kBMnMajor = true;
     using Params = ValuesParams;
     using Smem = GemmSmem<BN, STAGES, false>;
     static __device__ __forceinline__ int k_steps(const Params& p) { return (p.t_e + kAggBK - 1) / kAggBK; }
@@ -627,6 +629,7 @@ struct ValuesOp {
         for (int j = 0; j < BN / 64; ++j)  // 64 features x 64 tokens per box
             tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_b, tl.n0 + j * 64, k * kAggBK, tl.img, &sm.full[s]);
     }
+    static __device__ __forceinline__ uint64_t a_desc(uint32_t a0, int kk) { return umma_desc(a0 + kk * 32, 16, 1024); }
     // 16 token rows of 128 B per K step; the next 64 features start one box (8 KB) further on
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
     static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, const Tile&) {}
@@ -634,6 +637,74 @@ struct ValuesOp {
                                                     int lane, int m0, const Tile& tl)
     {
         values_epilogue(p, tmem, ewarp, lane, m0, tl);
+    }
+};
+
+// K_c = Rbar^T K (and V_c = Rbar^T V) of the KV-compressed attention: tile of 128 memory anchors x
+// BN features, K = compact tokens.  A = R [m_e, s] read as R^T, i.e. MN-major (two blocks of 64
+// tokens x 64 anchors); B = K or V [m_e, d] MN-major as above.  The epilogue divides row s by the
+// column sum of R.
+struct CompressParams {
+    const float* colsum;  // [s] column sums of the bf16-rounded assignment matrix
+    __nv_bfloat16* out;   // [n_img, s, d_v]
+    int* error;
+    TileGrid grid;
+    int32_t s, m_e, d_v;
+};
+
+template <int BN_>
+struct CompressOp {
+    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1;
+    static constexpr bool kAMnMajor = true, kBMnMajor = true;
+    using Params = CompressParams;
+    using Smem = GemmSmem<BN, STAGES, false>;
+    static __device__ __forceinline__ int k_steps(const Params& p) { return (p.m_e + kAggBK - 1) / kAggBK; }
+    static __device__ __forceinline__ bool tile(const Params& p, int worker, int n_workers, int i, Tile& tl)
+    {
+        return round_robin_tile(p.grid, BN, worker, n_workers, i, tl);
+    }
+    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
+                                                int k, int m0, const Tile& tl, uint32_t, uint32_t)
+    {
+        mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
+        tma_load_2d(sm.a[s], map_a, m0, k * kAggBK, &sm.full[s]);                       // anchors m0 .. + 64
+        tma_load_2d(sm.a[s] + kAggBK * 64, map_a, m0 + 64, k * kAggBK, &sm.full[s]);    // .. + 128
+#pragma unroll
+        for (int j = 0; j < BN / 64; ++j)
+            tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_b, tl.n0 + j * 64, k * kAggBK, tl.img, &sm.full[s]);
+    }
+    static __device__ __forceinline__ uint64_t a_desc(uint32_t a0, int kk) { return umma_desc(a0 + kk * 2048, kAggBK * 128, 1024); }
+    static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
+    static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, const Tile&) {}
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, const CUtensorMap*, uint32_t tmem, int ewarp,
+                                                    int lane, int m0, const Tile& tl)
+    {
+        const int half_cols = tl.n >> 1;
+        const int quarter = ewarp & 3, half = ewarp >> 2;
+        const int row = m0 + quarter * 32 + lane;  // memory anchor
+        const bool row_ok = row < p.s;
+        const float sum = row_ok ? p.colsum[row] : 0.f;
+        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        const int nh = tl.n0 + half * half_cols;
+        __nv_bfloat16* out = p.out + ((size_t)tl.img * p.s + (row_ok ? row : 0)) * p.d_v + nh;
+        for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * half_cols, half_cols,
+                       [&](const uint32_t (&acc)[32], int c0) {
+            if (row_ok) {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    if (nh + c0 + q4 * 8 < p.d_v) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv,
+                                                                           __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv);
+                            w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        });
     }
 };
 
@@ -712,7 +783,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
         bool ok = true;
         Tile tl;
         for (int local = 0; ok && Op::tile(p, worker, n_workers, local, tl); ++local) {
-            const uint32_t idesc = umma_idesc(tl.n, Op::kBMnMajor ? 1 : 0, kAggBM * Op::kCtas);
+            const uint32_t idesc = umma_idesc(tl.n, Op::kBMnMajor ? 1 : 0, kAggBM * Op::kCtas, Op::kAMnMajor ? 1 : 0);
             const int buf = local & 1;
             ok = mbar_wait(&sm.acc_empty[buf], ((local >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutAcc);
             if (!ok) break;
@@ -726,8 +797,8 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
                 const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
 #pragma unroll
                 for (int kk = 0; kk < kAggBK / 16; ++kk) {
-                    if (kPair) umma_bf16_pair(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
-                    else umma_bf16(tmem_acc, umma_desc(a0 + kk * 32, 16, 1024), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                    if (kPair) umma_bf16_pair(tmem_acc, Op::a_desc(a0, kk), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                    else umma_bf16(tmem_acc, Op::a_desc(a0, kk), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
                 }
                 // frees the stage (in both blocks) once these MMAs have read it
                 if (kPair) umma_commit_pair(&sm.empty[s]);

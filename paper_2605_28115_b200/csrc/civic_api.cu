@@ -8,6 +8,7 @@
 
 #include "aggregate.cuh"
 #include "gather.cuh"
+#include "kv_attention.cuh"
 #include "select.cuh"
 #include "select_large.cuh"
 
@@ -642,6 +643,136 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
         n_launched += 2;
     }
     g_launches.fetch_add(n_launched, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+// ---- KV-compressed visual attention (Eq. 9) -------------------------------------------------
+
+struct KvAttnPlan {
+    int32_t dim, compress_bn;
+    size_t r16_off, colsum_off, kc_off, vc_off, total, attn_smem;
+};
+
+static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim, int32_t s,
+                                        KvAttnPlan& pl)
+{
+    if (n_img < 0 || m_e < 1 || n_heads < 1 || head_dim < 1 || s < 1) return CIVIC_ERR_INVALID_ARG;
+    if ((head_dim != 64 && head_dim != 128) || s % 64 || s > 256 || n_img > 65535 || n_heads > 65535)
+        return CIVIC_ERR_UNSUPPORTED;
+    const int64_t dim = (int64_t)n_heads * head_dim;
+    if (dim > (1 << 20)) return CIVIC_ERR_UNSUPPORTED;
+    pl.dim = (int32_t)dim;
+    pl.attn_smem = civic::attn_smem_bytes(head_dim, s);
+    if (pl.attn_smem > kMaxDynamicSmem) return CIVIC_ERR_UNSUPPORTED;
+    pl.compress_bn = dim % 256 == 0 ? 256 : (dim % 192 == 0 ? 192 : 128);
+    size_t off = 0;
+    auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
+    pl.r16_off = take((size_t)m_e * s * 2);
+    pl.colsum_off = take((size_t)s * 4);
+    pl.kc_off = take((size_t)n_img * s * dim * 2);
+    pl.vc_off = take((size_t)n_img * s * dim * 2);
+    pl.total = off;
+    return CIVIC_OK;
+}
+
+size_t civic_kv_compressed_attention_workspace_bytes(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                                     int32_t s)
+{
+    KvAttnPlan pl;
+    return plan_kv_attention(n_img, m_e, n_heads, head_dim, s, pl) == CIVIC_OK ? pl.total : 0;
+}
+
+civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const void* v, const float* r,
+                                             int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                             int32_t s, void* out, void* workspace, size_t workspace_bytes,
+                                             int32_t* device_status, void* stream_)
+{
+    KvAttnPlan pl;
+    const civic_status_t st = plan_kv_attention(n_img, m_e, n_heads, head_dim, s, pl);
+    if (st != CIVIC_OK) return st;
+    if (n_img == 0) return CIVIC_OK;
+    if (!q || !k || !v || !r || !out || !device_status) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16) || !aligned(r, 4) ||
+        !aligned(device_status, 4))
+        return CIVIC_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < pl.total) return CIVIC_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return CIVIC_ERR_ALIGNMENT;
+    const size_t x_bytes = (size_t)n_img * m_e * pl.dim * 2;
+    if (overlaps(out, x_bytes, q, x_bytes) || overlaps(out, x_bytes, k, x_bytes) || overlaps(out, x_bytes, v, x_bytes) ||
+        overlaps(out, x_bytes, r, (size_t)m_e * s * 4) || overlaps(workspace, pl.total, out, x_bytes) ||
+        overlaps(workspace, pl.total, q, x_bytes) || overlaps(workspace, pl.total, k, x_bytes) ||
+        overlaps(workspace, pl.total, v, x_bytes) || overlaps(workspace, pl.total, r, (size_t)m_e * s * 4) ||
+        overlaps(device_status, 4, workspace, pl.total) || overlaps(device_status, 4, out, x_bytes))
+        return CIVIC_ERR_INVALID_ARG;
+
+    cudaStream_t stream = (cudaStream_t)stream_;
+    char* ws = (char*)workspace;
+    __nv_bfloat16* r16 = (__nv_bfloat16*)(ws + pl.r16_off);
+    float* colsum = (float*)(ws + pl.colsum_off);
+    __nv_bfloat16* kc = (__nv_bfloat16*)(ws + pl.kc_off);
+    __nv_bfloat16* vc = (__nv_bfloat16*)(ws + pl.vc_off);
+
+    EncodeTiledFn enc = nullptr;
+    civic_status_t ms = tensor_map_encoder(&enc);
+    if (ms != CIVIC_OK) return ms;
+    CUtensorMap map_r, map_k_in, map_v_in, map_q, map_kc, map_vc;
+    {
+        const uint64_t dims[2] = {(uint64_t)s, (uint64_t)m_e}, str[1] = {(uint64_t)s * 2};
+        if ((ms = make_map(enc, &map_r, r16, 2, dims, str, 64)) != CIVIC_OK) return ms;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
+        if ((ms = make_map(enc, &map_k_in, k, 3, dims, str, 64)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_v_in, v, 3, dims, str, 64)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_q, q, 3, dims, str, civic::kAggBM)) != CIVIC_OK) return ms;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)s, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)s * pl.dim * 2};
+        if ((ms = make_map(enc, &map_kc, kc, 3, dims, str, 64)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_vc, vc, 3, dims, str, 64)) != CIVIC_OK) return ms;
+    }
+
+    const bool pdl = programmatic();
+    CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::assign_prep_kernel, 1u, (unsigned)s, 0, stream, r, m_e, s, r16, colsum));
+
+    civic::CompressParams cp;
+    cp.colsum = colsum; cp.error = device_status; cp.s = s; cp.m_e = m_e; cp.d_v = pl.dim;
+    const int32_t s_tiles = (s + civic::kAggBM - 1) / civic::kAggBM;
+    const int32_t f_tiles = (pl.dim + pl.compress_bn - 1) / pl.compress_bn;
+    cp.grid = civic::TileGrid{s_tiles, f_tiles, n_img, s_tiles * f_tiles * n_img};
+    for (int which = 0; which < 2; ++which) {
+        cp.out = which ? vc : kc;
+        const CUtensorMap& map_x = which ? map_v_in : map_k_in;
+        civic_status_t gs;
+        if (pl.compress_bn == 256) gs = launch_gemm<civic::CompressOp<256>>(map_r, map_x, map_r, cp, cp.grid.total, stream);
+        else if (pl.compress_bn == 192) gs = launch_gemm<civic::CompressOp<192>>(map_r, map_x, map_r, cp, cp.grid.total, stream);
+        else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_x, map_r, cp, cp.grid.total, stream);
+        if (gs != CIVIC_OK) return gs;
+    }
+
+    civic::AttnParams ap;
+    ap.out = (__nv_bfloat16*)out; ap.error = device_status;
+    ap.m_e = m_e; ap.n_heads = n_heads; ap.d = head_dim; ap.s = s;
+    ap.scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
+    {
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)pl.attn_smem));
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((m_e + civic::kAggBM - 1) / civic::kAggBM), (unsigned)n_heads, (unsigned)n_img);
+        cfg.blockDim = dim3(civic::kAttnThreads);
+        cfg.dynamicSmemBytes = pl.attn_smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl ? 1 : 0;
+        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::kv_attention_kernel, map_q, map_kc, map_vc, ap));
+    }
+    g_launches.fetch_add(4, std::memory_order_relaxed);
     return CIVIC_OK;
 }
 

@@ -243,6 +243,23 @@ def test_anchor_aggregate_validation(lib):
     assert lib.civic_launch_count() == before
 
 
+def test_kv_compressed_attention_validation(lib):
+    f = lambda n_img=1, m_e=100, heads=2, d=64, s=128, q=0x100000, k=0x200000, v=0x300000, r=0x400000, \
+        out=0x500000, ws=0x1000000, ws_bytes=1 << 30, status=0x600000: \
+        lib.civic_kv_compressed_attention(q, k, v, r, n_img, m_e, heads, d, s, out, ws, ws_bytes, status, None)
+    before = lib.civic_launch_count()
+    assert f(d=72) == 5 and f(s=100) == 5 and f(s=320) == 5 and f(d=256) == 5
+    assert f(m_e=0) == 1 and f(heads=0) == 1 and f(q=None) == 1 and f(status=None) == 1
+    assert f(k=0x200008) == 4 and f(ws=0x1000010) == 4
+    assert f(ws=None) == 7 and f(ws_bytes=100) == 7
+    assert f(out=0x100040) == 1  # output overlaps q
+    assert f(n_img=0) == 0
+    assert lib.civic_kv_compressed_attention_workspace_bytes(1, 100, 2, 72, 128) == 0
+    need = lib.civic_kv_compressed_attention_workspace_bytes(2, 100, 2, 64, 128)
+    assert need >= 100 * 128 * 2 + 128 * 4 + 2 * 2 * 128 * 128 * 2 and need % 256 == 0
+    assert lib.civic_launch_count() == before
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
 
