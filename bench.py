@@ -662,6 +662,80 @@ def run_aggregate(args):
     print(json.dumps(line), flush=True)
 
 
+def run_kv_attention(args):
+    """`--workload kvattn_*`: one step = one civic_kv_compressed_attention call (Eq. 9)."""
+    import numpy as np
+    import torch
+
+    from paper_2605_28115_b200 import build as civic_build
+    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import workloads as W
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
+        raise SystemExit("this workload is benchmarked on one GPU")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    dev = "cuda:0"
+    civic_build.build()
+    civic.load()
+    w = W.KVATTN_BY_NAME[args.workload]
+    q, k, v, r = W.kvattn_inputs(w, dev)
+    out = torch.empty_like(q)
+    ws = torch.empty(civic.kv_compressed_attention_workspace_bytes(w.n_img, w.m_e, w.n_heads, w.head_dim, w.s),
+                     dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        civic.civic_kv_compressed_attention(q, k, v, r, w.n_heads, out=out, workspace=ws, device_status=status)
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = civic.launch_count()
+    sampler.start()
+    start.record()
+    for _ in range(args.steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = civic.launch_count() - launches0
+    ms = start.elapsed_time(end) / args.steps
+    if int(status.item()) != 0:
+        raise SystemExit(f"a wait inside the kernels timed out (status {int(status.item())})")
+    value = w.flops / (ms * 1e-3) / 1e12
+    burst, sustained, which = measured_tensor_peak()
+    roofline = {"bound": "tensor", "kernel": "civic_kv_compressed_attention (four launches; latency-bound at this size)",
+                "achieved": value, "peak": burst, "unit": "TFLOP/s", "frac": value / burst, "peak_source": which,
+                "peak_kind": "burst", "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import aggregate as OA
+
+        q64, k64, v64 = (a[0].double().cpu().numpy() for a in (q, k, v))
+        r64 = r.double().cpu().numpy()
+        times = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            want, _, _ = OA.kv_compressed_attention(q64, k64, v64, r64, w.n_heads)
+            times.append(time.perf_counter() - t0)
+        med = statistics.median(times)
+        cpu = {"value": w.flops / w.n_img / med / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": f"the fp64 numpy oracle on ONE of the {w.n_img} images, median of 3 runs, {med * 1e3:.0f} ms",
+               "max_abs_difference_to_gpu_result": float(np.max(np.abs(out[0].float().cpu().numpy() - want)))}
+    line = {"metric": "kv_compressed_attention_TFLOPs_eq9", "value": value, "unit": "TFLOP/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "n_img": w.n_img, "m_e": w.m_e, "n_heads": w.n_heads, "head_dim": w.head_dim,
+                       "s": w.s, "l2": "working set (50 MB) smaller than L2 and not flushed: a latency figure",
+                       "parallelism": "single"},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": None, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+
+
 def run_aggregate_reference(args):
     """The fp64 numpy oracle of Eq. 8 on this machine's host cores; each step is ONE image of the
     workload (a bounded sample), at most 10 steps."""
@@ -754,7 +828,11 @@ def run_reference(args):
 
 if __name__ == "__main__":
     a = parse_args()
-    if a.workload.startswith("agg_"):
+    if a.workload.startswith("kvattn_"):
+        if a.impl == "reference":
+            raise SystemExit("the reference arm covers the select + compact + KV and the aggregation workloads")
+        run_kv_attention(a)
+    elif a.workload.startswith("agg_"):
         if a.impl == "reference":
             run_aggregate_reference(a)
         else:

@@ -645,7 +645,8 @@ struct ValuesOp {
 // tokens x 64 anchors); B = K or V [m_e, d] MN-major as above.  The epilogue divides row s by the
 // column sum of R.
 struct CompressParams {
-    const float* colsum;  // [s] column sums of the bf16-rounded assignment matrix
+    const float* colsum_parts;  // [n_parts, s] column sums of the bf16-rounded assignment matrix, by row panel
+    int32_t n_parts;
     __nv_bfloat16* out;   // [n_img, s, d_v]
     int* error;
     TileGrid grid;
@@ -683,7 +684,9 @@ struct CompressOp {
         const int quarter = ewarp & 3, half = ewarp >> 2;
         const int row = m0 + quarter * 32 + lane;  // memory anchor
         const bool row_ok = row < p.s;
-        const float sum = row_ok ? p.colsum[row] : 0.f;
+        float sum = 0.f;  // fixed order of additions: every tile gets the same divisor
+        if (row_ok)
+            for (int q = 0; q < p.n_parts; ++q) sum += p.colsum_parts[(size_t)q * p.s + row];
         const float inv = sum > 0.f ? 1.f / sum : 0.f;
         const int nh = tl.n0 + half * half_cols;
         __nv_bfloat16* out = p.out + ((size_t)tl.img * p.s + (row_ok ? row : 0)) * p.d_v + nh;

@@ -650,7 +650,8 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
 
 struct KvAttnPlan {
     int32_t dim, compress_bn;
-    size_t r16_off, colsum_off, kc_off, vc_off, total, attn_smem;
+    int32_t n_parts;
+    size_t r16_off, colsum_off, partial_off, kc_off, vc_off, total, attn_smem;
 };
 
 static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim, int32_t s,
@@ -669,6 +670,8 @@ static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_he
     auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
     pl.r16_off = take((size_t)m_e * s * 2);
     pl.colsum_off = take((size_t)s * 4);
+    pl.n_parts = (m_e + civic::kAssignRows - 1) / civic::kAssignRows;
+    pl.partial_off = take((size_t)pl.n_parts * s * 4);
     pl.kc_off = take((size_t)n_img * s * dim * 2);
     pl.vc_off = take((size_t)n_img * s * dim * 2);
     pl.total = off;
@@ -708,7 +711,6 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
     cudaStream_t stream = (cudaStream_t)stream_;
     char* ws = (char*)workspace;
     __nv_bfloat16* r16 = (__nv_bfloat16*)(ws + pl.r16_off);
-    float* colsum = (float*)(ws + pl.colsum_off);
     __nv_bfloat16* kc = (__nv_bfloat16*)(ws + pl.kc_off);
     __nv_bfloat16* vc = (__nv_bfloat16*)(ws + pl.vc_off);
 
@@ -736,10 +738,12 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
 
     const bool pdl = programmatic();
     CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
-    CIVIC_CUDA_TRY(civic::launch(pdl, civic::assign_prep_kernel, 1u, (unsigned)s, 0, stream, r, m_e, s, r16, colsum));
+    float* partial = (float*)(ws + pl.partial_off);
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::assign_convert_kernel, (unsigned)pl.n_parts, (unsigned)s, 0, stream, r, m_e,
+                                 s, r16, partial));
 
     civic::CompressParams cp;
-    cp.colsum = colsum; cp.error = device_status; cp.s = s; cp.m_e = m_e; cp.d_v = pl.dim;
+    cp.colsum_parts = partial; cp.n_parts = pl.n_parts; cp.error = device_status; cp.s = s; cp.m_e = m_e; cp.d_v = pl.dim;
     const int32_t s_tiles = (s + civic::kAggBM - 1) / civic::kAggBM;
     const int32_t f_tiles = (pl.dim + pl.compress_bn - 1) / pl.compress_bn;
     cp.grid = civic::TileGrid{s_tiles, f_tiles, n_img, s_tiles * f_tiles * n_img};

@@ -12,7 +12,7 @@
 //   MMA 1    S = Q K_c^T -> TMEM columns [0, s)
 //   softmax  thread per query row: maximum, exp2, row sum; P as bf16 into 128-byte-swizzled
 //            shared memory (the A operand of the second chain)
-//   MMA 2    O = P V_c -> TMEM columns [s, s + d)
+//   MMA 2    O = P V_c -> TMEM columns [0, d) again
 //   store    O / row sum as bf16
 // Every wait is bounded as in aggregate.cuh.
 #pragma once
@@ -21,22 +21,25 @@
 namespace civic {
 
 // R (fp32) -> bf16 copy and the column sums of the ROUNDED values (what the tensor core will
-// multiply with).  One block; thread = one column.
-__global__ void assign_prep_kernel(const float* __restrict__ r, int m_e, int s, __nv_bfloat16* __restrict__ r16,
-                                   float* __restrict__ colsum)
+// multiply with): a block converts kAssignRows rows and writes their column sums; the compression
+// GEMM's epilogue adds the panels' sums in a fixed order.
+constexpr int kAssignRows = 16;
+__global__ void assign_convert_kernel(const float* __restrict__ r, int m_e, int s, __nv_bfloat16* __restrict__ r16,
+                                      float* __restrict__ partial)
 {
     wait_for_prior_kernels();
+    const int m_begin = blockIdx.x * kAssignRows, m_end = min(m_begin + kAssignRows, m_e);
     for (int c = threadIdx.x; c < s; c += blockDim.x) {
         float sum = 0.f;
-        for (int m = 0; m < m_e; ++m) {
+#pragma unroll 4
+        for (int m = m_begin; m < m_end; ++m) {
             const __nv_bfloat16 v = __float2bfloat16_rn(r[(size_t)m * s + c]);
             r16[(size_t)m * s + c] = v;
             sum += __bfloat162float(v);
         }
-        colsum[c] = sum;
+        partial[(size_t)blockIdx.x * s + c] = sum;
     }
 }
-
 constexpr int kAttnThreads = 192;  // warp 0: TMA, warp 1: TMEM + MMA, warps 2..5: one query row per thread
 
 struct AttnParams {
@@ -46,12 +49,18 @@ struct AttnParams {
     float scale_log2e;   // log2(e) / sqrt(d)
 };
 
-// Shared memory: q [d/64][128 x 128 B] | k [d/64][s x 128 B] | v [s/64][d/64][64 x 128 B] |
-// p [s/64][128 x 128 B], every block 1024-byte aligned; then the barriers.
+// Shared memory: region A = q [d/64][128 x 128 B] | k [d/64][s x 128 B], later overwritten by
+// p [s/64][128 x 128 B] (Q and K_c are dead once the first MMA chain has completed); then
+// v [s/64][d/64][64 x 128 B]; then the barriers.  Every block of data is 1024-byte aligned.
+// 96 KB for 64-wide heads and 256 anchors: two blocks per SM.
+__host__ __device__ constexpr size_t attn_region_a_bytes(int d, int s)
+{
+    const size_t qk = (size_t)(d / 64) * 16384 + (size_t)(d / 64) * s * 128, pr = (size_t)(s / 64) * 16384;
+    return qk > pr ? qk : pr;
+}
 __host__ __device__ constexpr size_t attn_smem_bytes(int d, int s)
 {
-    return (size_t)(d / 64) * 16384 + (size_t)(d / 64) * s * 128 + (size_t)(s / 64) * (d / 64) * 8192 +
-           (size_t)(s / 64) * 16384 + 1024 /* barriers */ + 1024 /* alignment slack */;
+    return attn_region_a_bytes(d, s) + (size_t)(s / 64) * (d / 64) * 8192 + 1024 /* barriers */ + 1024 /* alignment slack */;
 }
 
 __global__ void __launch_bounds__(kAttnThreads) kv_attention_kernel(const __grid_constant__ CUtensorMap map_q,
@@ -64,18 +73,19 @@ __global__ void __launch_bounds__(kAttnThreads) kv_attention_kernel(const __grid
     const int d = p.d, s = p.s, d_blocks = d >> 6, s_blocks = s >> 6;
     uint8_t* q_sm = base;
     uint8_t* k_sm = q_sm + d_blocks * 16384;
-    uint8_t* v_sm = k_sm + d_blocks * s * 128;
-    uint8_t* p_sm = v_sm + s_blocks * d_blocks * 8192;
+    uint8_t* p_sm = base;  // takes over the Q / K_c region after the first MMA chain
+    uint8_t* v_sm = base + attn_region_a_bytes(d, s);
     struct Sync {
         uint64_t loaded, scores_done, probs_ready, out_done;
         uint32_t tmem_base;
         int abort;
     };
-    Sync& sy = *reinterpret_cast<Sync*>(p_sm + s_blocks * 16384);
+    Sync& sy = *reinterpret_cast<Sync*>(v_sm + s_blocks * d_blocks * 8192);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * kAggBM, head = blockIdx.y, img = blockIdx.z;
     volatile int* abort = &sy.abort;
-    const uint32_t tmem_cols = (s + d) <= 128 ? 128u : ((s + d) <= 256 ? 256u : 512u);
+    // O takes over the first d columns of S (S is dead once every softmax warp has read it)
+    const uint32_t tmem_cols = max(s, d) <= 64 ? 64u : (max(s, d) <= 128 ? 128u : 256u);
 
     if (threadIdx.x == 0) {
         mbar_init(&sy.loaded, 1);
@@ -90,7 +100,7 @@ __global__ void __launch_bounds__(kAttnThreads) kv_attention_kernel(const __grid
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_s = sy.tmem_base, tmem_o = sy.tmem_base + s;
+    const uint32_t tmem_s = sy.tmem_base, tmem_o = sy.tmem_base;
     const bool stop = *p.error != 0;
 
     if (warp == 0 && lane == 0 && !stop) {

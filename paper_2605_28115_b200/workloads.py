@@ -303,3 +303,43 @@ def payload_bf16_affine(shape, seed: int, device, scale: float, offset: float):
         out[lo:hi] = (torch.randn(hi - lo, generator=g, device=device, dtype=torch.float32) * scale
                       + offset).to(torch.bfloat16)
     return out.view(*shape)
+
+
+# ---------------------------------------------------------------- KV-compressed attention (Eq. 9)
+
+@dataclasses.dataclass(frozen=True)
+class KvAttnWorkload:
+    """Projected Q, K, V of one compact vision layer for a batch of images, and a shared assignment."""
+
+    name: str
+    n_img: int
+    m_e: int      # compact tokens
+    n_heads: int
+    head_dim: int
+    s: int        # memory anchors
+    seed: int = SEED_BASE + 9500
+
+    @property
+    def dim(self) -> int:
+        return self.n_heads * self.head_dim
+
+    @property
+    def flops(self) -> int:
+        """Compression of K and V (2 GEMMs) and the two contractions of the attention."""
+        return 2 * 2 * self.n_img * self.s * self.m_e * self.dim * 2
+
+
+# 8 images, 1024 compact tokens, 16 heads of 64 (vision width 1024), 256 memory anchors
+KVATTN_896 = KvAttnWorkload("kvattn_batch8_896", 8, 1024, 16, 64, 256)
+KVATTN_BY_NAME = {w.name: w for w in (KVATTN_896,)}
+
+
+def kvattn_inputs(w: KvAttnWorkload, device="cpu"):
+    """(q, k, v bf16 [n_img, m_e, dim] ~ 1.2 N(0,1); r fp32 [m_e, s]: row-wise softmax of 3 N(0,1)), seeded."""
+    import torch
+
+    q, k, v = (payload_bf16_affine((w.n_img, w.m_e, w.dim), w.seed + i, device, 1.2, 0.0) for i in range(3))
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed + 3)
+    r = torch.softmax(torch.randn((w.m_e, w.s), generator=g, device=device, dtype=torch.float32) * 3.0, dim=1)
+    return q, k, v, r
