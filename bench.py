@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used when MEASURE
 # profiles/; keyed by workload name.  None = not captured for that workload.
 NCU_DRAM_TRAFFIC_PER_LAUNCH = {
     # profiles/gather_rows_kernel_c3_kv.md: 8-layer capture, reads x4.5, writes = algorithmic minus
-    # the 50.6 MB that were still dirty in L2 when the kernel ended
-    "c3_kv_qwen3vl8b": 1_860_600_000,
+    # the 52.0 MB that were still dirty in L2 when the kernel ended
+    "c3_kv_qwen3vl8b": 1_859_200_000,
 }
 
 

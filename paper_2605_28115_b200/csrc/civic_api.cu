@@ -625,21 +625,11 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     int n_launched = 3;
     if (token_mass) {
         float* partial = (float*)(ws + pl.mass_off);
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cudaLaunchConfig_t cfg = {};
-        cfg.blockDim = dim3(256);
-        cfg.stream = stream;
-        cfg.attrs = attr;
-        cfg.numAttrs = pdl ? 1 : 0;
-        cfg.gridDim = dim3((unsigned)pl.n_panels, (unsigned)n_img);
-        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::token_mass_partial_kernel, (const __nv_bfloat16*)p,
-                                          (const float*)inv_l, m_e, t_e, pl.t_ld, pl.n_panels, partial));
-        cfg.blockDim = dim3(64);
-        cfg.gridDim = dim3((unsigned)((t_e + 63) / 64), (unsigned)n_img);
-        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::token_mass_reduce_kernel, (const float*)partial, t_e, pl.t_ld,
-                                          pl.n_panels, token_mass));
+        CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_partial_kernel, dim3((unsigned)pl.n_panels, (unsigned)n_img),
+                                     256u, 0, stream, (const __nv_bfloat16*)p, (const float*)inv_l, m_e, t_e, pl.t_ld,
+                                     pl.n_panels, partial));
+        CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_reduce_kernel, dim3((unsigned)((t_e + 63) / 64), (unsigned)n_img),
+                                     64u, 0, stream, (const float*)partial, t_e, pl.t_ld, pl.n_panels, token_mass));
         n_launched += 2;
     }
     g_launches.fetch_add(n_launched, std::memory_order_relaxed);
@@ -761,21 +751,11 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
     ap.out = (__nv_bfloat16*)out; ap.error = device_status;
     ap.m_e = m_e; ap.n_heads = n_heads; ap.d = head_dim; ap.s = s;
     ap.scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
-    {
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)pl.attn_smem));
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)((m_e + civic::kAggBM - 1) / civic::kAggBM), (unsigned)n_heads, (unsigned)n_img);
-        cfg.blockDim = dim3(civic::kAttnThreads);
-        cfg.dynamicSmemBytes = pl.attn_smem;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = pdl ? 1 : 0;
-        CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::kv_attention_kernel, map_q, map_kc, map_vc, ap));
-    }
+    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)pl.attn_smem));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel,
+                                 dim3((unsigned)((m_e + civic::kAggBM - 1) / civic::kAggBM), (unsigned)n_heads, (unsigned)n_img),
+                                 (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, ap));
     g_launches.fetch_add(4, std::memory_order_relaxed);
     return CIVIC_OK;
 }

@@ -25,11 +25,11 @@ __device__ __forceinline__ void release_next_kernel()
 }
 
 template <typename... KArgs, typename... Args>
-cudaError_t launch(bool programmatic, void (*kernel)(KArgs...), unsigned grid, unsigned block,
-                   size_t smem, cudaStream_t stream, Args&&... args)
+cudaError_t launch(bool programmatic, void (*kernel)(KArgs...), dim3 grid, unsigned block, size_t smem,
+                   cudaStream_t stream, Args&&... args)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
+    cfg.gridDim = grid;
     cfg.blockDim = dim3(block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
