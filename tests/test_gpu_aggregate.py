@@ -94,6 +94,12 @@ def test_benchmark_shape_one_image():
     check(x, a, 0.07)
 
 
+def test_many_tiles_ragged_everywhere():
+    """More pair tiles than resident pairs in the anchor direction, ragged token and anchor edges."""
+    x, a = inputs(2, 9001, 1500, 320, seed=13)
+    check(x, a, 0.05)
+
+
 def test_structure_and_degenerate_tokens():
     x, a = inputs(2, 300, 40, 128, seed=9)
     x[0, 17] = 2.5        # a token with all features equal has no direction: logit 0, as in the oracle
