@@ -145,8 +145,36 @@ def _device_of(*tensors) -> torch.device:
     return torch.device("cuda", torch.cuda.current_device())
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
-    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+    """cudaStream_t of `stream`, or of torch's current stream on the current device."""
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_stream is not None:  # same value as current_stream().cuda_stream without building a Stream object
+        return _raw_stream(torch.cuda.current_device())
+    return torch.cuda.current_stream().cuda_stream
+
+
+class _on_device:
+    """Makes `device` current for the duration of a call; does nothing when it already is (the
+    common case, and several microseconds cheaper than torch.cuda.device)."""
+
+    __slots__ = ("index", "ctx")
+
+    def __init__(self, device: torch.device):
+        self.index = device.index if device.index is not None else torch.cuda.current_device()
+        self.ctx = None
+
+    def __enter__(self):
+        if torch.cuda.current_device() != self.index:
+            self.ctx = torch.cuda.device(self.index)
+            self.ctx.__enter__()
+
+    def __exit__(self, *exc):
+        if self.ctx is not None:
+            self.ctx.__exit__(*exc)
 
 
 def launch_count() -> int:
@@ -173,7 +201,7 @@ def civic_select(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optional[torc
         raise ValueError("keep_idx must be [n_seg, k]")
     args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
             _dev_ptr(keep_idx, "keep_idx", torch.int32))
-    with torch.cuda.device(_device_of(scores, keep_idx)):
+    with _on_device(_device_of(scores, keep_idx)):
         _check(load().civic_select(*args, _stream_ptr(stream)), "civic_select")
     return keep_idx
 
@@ -198,7 +226,7 @@ def civic_select_seq(scores: torch.Tensor, desc: SelectDesc, seq_len: int, vis_s
         raise ValueError("seq_idx must be [n_seq, seq_len - n + k]")
     args = (_dev_ptr(scores, "scores", torch.float32), n_seq, ctypes.byref(desc), seq_len, vis_start,
             _dev_ptr(keep_idx, "keep_idx", torch.int32), _dev_ptr(seq_idx, "seq_idx", torch.int32))
-    with torch.cuda.device(_device_of(scores, keep_idx)):
+    with _on_device(_device_of(scores, keep_idx)):
         _check(load().civic_select_seq(*args, _stream_ptr(stream)), "civic_select_seq")
     return keep_idx, seq_idx
 
@@ -226,7 +254,7 @@ def civic_select_large(scores: torch.Tensor, desc: SelectDesc, keep_idx: Optiona
     args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
             _dev_ptr(keep_idx, "keep_idx", torch.int32), _dev_ptr(workspace, "workspace", torch.uint8),
             workspace.numel(), chunk_tokens)
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         _check(load().civic_select_large(*args, _stream_ptr(stream)), "civic_select_large")
     return keep_idx
 
@@ -248,7 +276,7 @@ def civic_select_large_static(scores: torch.Tensor, desc: SelectDesc, keep_idx: 
         raise ValueError("keep_idx must be [n_seg, k]")
     args = (_dev_ptr(scores, "scores", torch.float32), n_seg, ctypes.byref(desc),
             _dev_ptr(keep_idx, "keep_idx", torch.int32), chunk_tokens)
-    with torch.cuda.device(_device_of(scores)):
+    with _on_device(_device_of(scores)):
         _check(load().civic_select_large_static(*args, _stream_ptr(stream)), "civic_select_large_static")
     return keep_idx
 
@@ -279,7 +307,7 @@ def civic_select_ragged(scores: torch.Tensor, descs: Sequence[SelectDesc],
     table = (SelectDesc * max(len(descs), 1))(*descs)
     args = (_dev_ptr(scores, "scores", torch.float32), len(descs), table,
             _dev_ptr(keep_idx, "keep_idx", torch.int32), _dev_ptr(flat_idx, "flat_idx", torch.int32))
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         _check(load().civic_select_ragged(*args, _stream_ptr(stream)), "civic_select_ragged")
     return keep_idx, flat_idx
 
@@ -320,7 +348,7 @@ def civic_compact(hidden: Optional[torch.Tensor], pos_ids: Optional[torch.Tensor
     args = (_dev_ptr(hidden, "hidden"), row_bytes, _dev_ptr(pos_ids, "pos_ids", torch.int32),
             _dev_ptr(keep_idx, "keep_idx", torch.int32), n_seg, n, k,
             _dev_ptr(hidden_out, "hidden_out"), _dev_ptr(pos_out, "pos_out", torch.int32))
-    with torch.cuda.device(_device_of(keep_idx, hidden, pos_ids)):
+    with _on_device(_device_of(keep_idx, hidden, pos_ids)):
         _check(load().civic_compact(*args, _stream_ptr(stream)), "civic_compact")
     return hidden_out, pos_out
 
@@ -337,7 +365,7 @@ def civic_seq_indices(keep_idx: torch.Tensor, seq_len: int, vis_start: int, n_vi
         raise ValueError("seq_idx must be [n_seq, seq_len - n_vis + k]")
     args = (_dev_ptr(keep_idx, "keep_idx", torch.int32), n_seq, k, seq_len, vis_start, n_vis,
             _dev_ptr(seq_idx, "seq_idx", torch.int32))
-    with torch.cuda.device(_device_of(keep_idx, seq_idx)):
+    with _on_device(_device_of(keep_idx, seq_idx)):
         _check(load().civic_seq_indices(*args, _stream_ptr(stream)), "civic_seq_indices")
     return seq_idx
 
@@ -393,7 +421,7 @@ def civic_compact_kv(tables: KVTables, seq_idx: torch.Tensor,
     if tuple(seq_idx.shape) != (tables.n_seq, tables.s_out):
         raise ValueError("seq_idx must be [n_seq, s_out]")
     idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
-    with torch.cuda.device(_device_of(seq_idx, *tables.keepalive[0], *tables.keepalive[2])):
+    with _on_device(_device_of(seq_idx, *tables.keepalive[0], *tables.keepalive[2])):
         _check(load().civic_compact_kv(tables.k_src, tables.v_src, tables.k_dst, tables.v_dst,
                                        tables.n_layers, tables.n_seq, tables.seq_len, tables.s_out,
                                        tables.row_bytes, idx_ptr, _stream_ptr(stream)),
@@ -450,7 +478,7 @@ def civic_compact_kv_heads(tables: KVHeadsTables, seq_idx: torch.Tensor,
     if tuple(seq_idx.shape) != (t.n_seq, t.s_out):
         raise ValueError("seq_idx must be [n_seq, s_out]")
     idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
-    with torch.cuda.device(_device_of(seq_idx, t.keepalive[0][0], t.keepalive[2][0])):
+    with _on_device(_device_of(seq_idx, t.keepalive[0][0], t.keepalive[2][0])):
         _check(load().civic_compact_kv_heads(*t.tables, t.n_layers, t.n_seq, t.n_heads, t.seq_len, t.s_out,
                                              t.head_bytes, idx_ptr, _stream_ptr(stream)),
                "civic_compact_kv_heads")
@@ -500,7 +528,7 @@ def civic_compact_kv_paged(tables: KVPagedTables, seq_idx: torch.Tensor, block_t
         raise ValueError("block_table must be [n_seq, max_pages_per_seq]")
     idx_ptr = _dev_ptr(seq_idx, "seq_idx", torch.int32)
     tab_ptr = _dev_ptr(block_table, "block_table", torch.int32)
-    with torch.cuda.device(_device_of(seq_idx, t.keepalive[0][0], t.keepalive[2][0])):
+    with _on_device(_device_of(seq_idx, t.keepalive[0][0], t.keepalive[2][0])):
         _check(load().civic_compact_kv_paged(*t.tables, t.n_layers, t.n_seq, t.seq_len, seq_idx.shape[1],
                                              t.row_bytes, idx_ptr, tab_ptr, block_table.shape[1],
                                              t.page_size, t.n_pages, _stream_ptr(stream)),
@@ -528,7 +556,7 @@ def civic_merge_embeddings(text: torch.Tensor, visual: torch.Tensor, keep_idx: t
     args = (_dev_ptr(text, "text"), _dev_ptr(visual, "visual"), dim * text.element_size(),
             _dev_ptr(keep_idx, "keep_idx", torch.int32), n_seq, seq_len, vis_start, n_vis, k,
             _dev_ptr(merged, "merged"))
-    with torch.cuda.device(_device_of(keep_idx, text, visual)):
+    with _on_device(_device_of(keep_idx, text, visual)):
         _check(load().civic_merge_embeddings(*args, _stream_ptr(stream)), "civic_merge_embeddings")
     return merged
 
@@ -547,7 +575,7 @@ def civic_compact_pos_planes(pos: torch.Tensor, seq_idx: torch.Tensor,
         raise ValueError("pos_out must be [n_planes, n_seq, s_out]")
     args = (_dev_ptr(pos, "pos", torch.int32), n_planes, n_seq, seq_len,
             _dev_ptr(seq_idx, "seq_idx", torch.int32), s_out, _dev_ptr(pos_out, "pos_out", torch.int32))
-    with torch.cuda.device(_device_of(seq_idx, pos)):
+    with _on_device(_device_of(seq_idx, pos)):
         _check(load().civic_compact_pos_planes(*args, _stream_ptr(stream)), "civic_compact_pos_planes")
     return pos_out
 
@@ -585,7 +613,7 @@ def civic_anchor_aggregate(x0: torch.Tensor, anchors: torch.Tensor, tau: float,
             ctypes.c_float(tau), _dev_ptr(z0, "z0", torch.bfloat16), _dev_ptr(token_mass, "token_mass", torch.float32),
             _dev_ptr(workspace, "workspace", torch.uint8), workspace.numel(),
             _dev_ptr(device_status, "device_status", torch.int32))
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         _check(load().civic_anchor_aggregate(*args, _stream_ptr(stream)), "civic_anchor_aggregate")
     return z0, token_mass, device_status
 
@@ -620,6 +648,6 @@ def civic_kv_compressed_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Ten
             _dev_ptr(r, "r", torch.float32), n_img, m_e, n_heads, head_dim, s, _dev_ptr(out, "out", torch.bfloat16),
             _dev_ptr(workspace, "workspace", torch.uint8), workspace.numel(),
             _dev_ptr(device_status, "device_status", torch.int32))
-    with torch.cuda.device(dev):
+    with _on_device(dev):
         _check(load().civic_kv_compressed_attention(*args, _stream_ptr(stream)), "civic_kv_compressed_attention")
     return out, device_status
