@@ -6,9 +6,10 @@
 //                      IEEE-754 totalOrder on the scores;
 //   2. floor           a token is reserved iff fewer than m tokens of its region beat it
 //                      (higher key, or equal key and lower index);
-//   3. radix select    over the non-reserved tokens, 4 passes of 8 bits from the top:
-//                      the exact key T of the k'-th best and how many tokens with key == T
-//                      are still needed (k' = k - number reserved);
+//   3. radix select    over the non-reserved tokens, up to 4 passes of 8 bits from the top:
+//                      the key T of the k'-th best (as many leading bits as are needed to tell
+//                      it apart) and how many tokens equal to T in those bits are still
+//                      needed (k' = k - number reserved);
 //   4. mask + scan     keep = reserved | key > T | (key == T and fewer than `need_eq`
 //                      equal-keyed non-reserved tokens precede it); destinations come from
 //                      a ballot/popc scan in index order, so the output is ascending.
@@ -78,7 +79,7 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
     const int n_pad = n_words << 5;
     uint32_t* hist = smem;                 // [4][256], one histogram per radix pass
     uint32_t* warp_tot = hist + 4 * 256;   // [32]
-    uint32_t* scal = warp_tot + 32;        // [0] chosen digit, [1] rank inside its bin
+    uint32_t* scal = warp_tot + 32;        // [0] chosen digit, [1] rank inside its bin, [2] whole bin wanted
     uint32_t* resv = scal + 4;             // [n_words] bit i%32 of word i/32
     uint32_t* keys = resv + n_words;       // [n_pad]
 
@@ -143,9 +144,9 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
     __syncthreads();
 
     // 3. radix select of the k_fill-th best non-reserved key, 8 bits per pass from the top
-    uint32_t prefix = 0xFFFFFFFFu, need_eq = 0;
+    uint32_t prefix = 0xFFFFFFFFu, mask = 0xFFFFFFFFu, need_eq = 0;
     if (d.k_fill > 0) {
-        uint32_t mask = 0;
+        mask = 0;
         uint32_t rank = (uint32_t)d.k_fill;  // 1-based rank among the candidates still matching
         prefix = 0;
 #pragma unroll 1
@@ -181,6 +182,7 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
                         if (above < rank && rank <= above + c[q]) {
                             scal[0] = 8 * lane + 7 - q;
                             scal[1] = rank - above;
+                            scal[2] = rank - above == c[q];  // the whole bin is wanted
                         }
                         above += c[q];
                     }
@@ -190,10 +192,14 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
             prefix |= scal[0] << shift;
             mask |= 0xFFu << shift;
             rank = scal[1];
+            // Every candidate that still matches the prefix is wanted: the lower bits cannot change
+            // the outcome, so the remaining passes are skipped (with continuous scores the bin of
+            // the threshold usually holds a single token after two passes).
+            if (scal[2]) break;
         }
         need_eq = rank;
     }
-    const uint32_t T = prefix;
+    const uint32_t T = prefix;  // compared under `mask`: the key bits decided so far
 
     // 4. keep mask and ascending destinations.  Each warp owns a contiguous run of 32-token
     // words; pass A counts, pass B places.
@@ -205,8 +211,8 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
         const int i = (wd << 5) + lane;
         const uint32_t key = keys[i];
         const bool r = (resv[wd] >> lane) & 1u;
-        const bool sure = i < n && (r || (d.k_fill > 0 && key > T));
-        const bool eq = i < n && !r && d.k_fill > 0 && key == T;
+        const bool sure = i < n && (r || (d.k_fill > 0 && (key & mask) > T));
+        const bool eq = i < n && !r && d.k_fill > 0 && (key & mask) == T;
         sure_cnt += __popc(__ballot_sync(0xFFFFFFFFu, sure));
         eq_cnt += __popc(__ballot_sync(0xFFFFFFFFu, eq));
     }
@@ -221,8 +227,8 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
         const int i = (wd << 5) + lane;
         const uint32_t key = keys[i];
         const bool r = (resv[wd] >> lane) & 1u;
-        const bool sure = i < n && (r || (d.k_fill > 0 && key > T));
-        const bool eq = i < n && !r && d.k_fill > 0 && key == T;
+        const bool sure = i < n && (r || (d.k_fill > 0 && (key & mask) > T));
+        const bool eq = i < n && !r && d.k_fill > 0 && (key & mask) == T;
         const uint32_t sb = __ballot_sync(0xFFFFFFFFu, sure), eb = __ballot_sync(0xFFFFFFFFu, eq);
         const uint32_t my_eq_before = eq_before + __popc(eb & lt);
         const uint32_t my_sure_before = sure_before + __popc(sb & lt);
