@@ -708,7 +708,7 @@ def run_kv_attention(args):
         raise SystemExit(f"a wait inside the kernels timed out (status {int(status.item())})")
     value = w.flops / (ms * 1e-3) / 1e12
     burst, sustained, which = measured_tensor_peak()
-    roofline = {"bound": "tensor", "kernel": "civic_kv_compressed_attention (four launches; latency-bound at this size)",
+    roofline = {"bound": "tensor", "kernel": "civic_kv_compressed_attention (three launches; latency-bound at this size)",
                 "achieved": value, "peak": burst, "unit": "TFLOP/s", "frac": value / burst, "peak_source": which,
                 "peak_kind": "burst", "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
     cpu = None

@@ -465,8 +465,9 @@ struct ScoresOpT {
         return round_robin_tile(p.grid, BN, worker, n_workers, i, tl);
     }
     // m0: this block's first anchor; rank: block rank in the pair
-    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, const Tile& tl, uint32_t rank, uint32_t leader_full)
+    static __device__ __forceinline__ void load(const Params&, Smem& sm, int s, const CUtensorMap* map_a,
+                                                const CUtensorMap* map_b, const CUtensorMap*, int k, int m0,
+                                                const Tile& tl, uint32_t rank, uint32_t leader_full)
     {
         const int n0 = tl.n0, img = tl.img;
         if constexpr (PAIR) {
@@ -620,8 +621,9 @@ struct ValuesOp {
     {
         return round_robin_tile(p.grid, BN, worker, n_workers, i, tl);
     }
-    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, const Tile& tl, uint32_t, uint32_t)
+    static __device__ __forceinline__ void load(const Params&, Smem& sm, int s, const CUtensorMap* map_a,
+                                                const CUtensorMap* map_b, const CUtensorMap*, int k, int m0,
+                                                const Tile& tl, uint32_t, uint32_t)
     {
         mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
         tma_load_3d(sm.a[s], map_a, k * kAggBK, m0, tl.img, &sm.full[s]);
@@ -647,10 +649,11 @@ struct ValuesOp {
 struct CompressParams {
     const float* colsum_parts;  // [n_parts, s] column sums of the bf16-rounded assignment matrix, by row panel
     int32_t n_parts;
-    __nv_bfloat16* out;   // [n_img, s, d_v]
+    __nv_bfloat16* out;    // [n_img, s, d_v]  K_c
+    __nv_bfloat16* out_v;  // [n_img, s, d_v]  V_c
     int* error;
-    TileGrid grid;
-    int32_t s, m_e, d_v;
+    TileGrid grid;         // over 2 n_img "images": K of every image, then V
+    int32_t s, m_e, d_v, n_img;
 };
 
 template <int BN_>
@@ -664,15 +667,20 @@ struct CompressOp {
     {
         return round_robin_tile(p.grid, BN, worker, n_workers, i, tl);
     }
-    static __device__ __forceinline__ void load(Smem& sm, int s, const CUtensorMap* map_a, const CUtensorMap* map_b,
-                                                int k, int m0, const Tile& tl, uint32_t, uint32_t)
+    // "Images" [0, n_img) of the tile grid compress K (map_b), [n_img, 2 n_img) compress V (map_v).
+    static __device__ __forceinline__ void load(const Params& p, Smem& sm, int s, const CUtensorMap* map_a,
+                                                const CUtensorMap* map_b, const CUtensorMap* map_v, int k, int m0,
+                                                const Tile& tl, uint32_t, uint32_t)
     {
+        const bool second = tl.img >= p.n_img;
+        const CUtensorMap* map_x = second ? map_v : map_b;
+        const int img = second ? tl.img - p.n_img : tl.img;
         mbar_expect_tx(&sm.full[s], (kAggBM + BN) * kAggBK * 2);
         tma_load_2d(sm.a[s], map_a, m0, k * kAggBK, &sm.full[s]);                       // anchors m0 .. + 64
         tma_load_2d(sm.a[s] + kAggBK * 64, map_a, m0 + 64, k * kAggBK, &sm.full[s]);    // .. + 128
 #pragma unroll
         for (int j = 0; j < BN / 64; ++j)
-            tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_b, tl.n0 + j * 64, k * kAggBK, tl.img, &sm.full[s]);
+            tma_load_3d(sm.b[s] + j * (kAggBK * 64), map_x, tl.n0 + j * 64, k * kAggBK, img, &sm.full[s]);
     }
     static __device__ __forceinline__ uint64_t a_desc(uint32_t a0, int kk) { return umma_desc(a0 + kk * 2048, kAggBK * 128, 1024); }
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
@@ -689,7 +697,9 @@ struct CompressOp {
             for (int q = 0; q < p.n_parts; ++q) sum += p.colsum_parts[(size_t)q * p.s + row];
         const float inv = sum > 0.f ? 1.f / sum : 0.f;
         const int nh = tl.n0 + half * half_cols;
-        __nv_bfloat16* out = p.out + ((size_t)tl.img * p.s + (row_ok ? row : 0)) * p.d_v + nh;
+        const bool second = tl.img >= p.n_img;
+        __nv_bfloat16* out = (second ? p.out_v : p.out) +
+                             ((size_t)(second ? tl.img - p.n_img : tl.img) * p.s + (row_ok ? row : 0)) * p.d_v + nh;
         for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * half_cols, half_cols,
                        [&](const uint32_t (&acc)[32], int c0) {
             if (row_ok) {
@@ -765,7 +775,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
                 const int s = it % STAGES;
                 ok = mbar_wait(&sm.empty[s], ((it / STAGES) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty);
                 if (!ok) break;
-                Op::load(sm, s, &map_a, &map_b, k, m0, tl, rank, kPair ? cluster_address(&sm.full[s], 0) : 0u);
+                Op::load(p, sm, s, &map_a, &map_b, &map_c, k, m0, tl, rank, kPair ? cluster_address(&sm.full[s], 0) : 0u);
             }
         }
         if (*abort) {  // let the copies already in flight land before the block goes away

@@ -736,14 +736,14 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
     cp.colsum_parts = partial; cp.n_parts = pl.n_parts; cp.error = device_status; cp.s = s; cp.m_e = m_e; cp.d_v = pl.dim;
     const int32_t s_tiles = (s + civic::kAggBM - 1) / civic::kAggBM;
     const int32_t f_tiles = (pl.dim + pl.compress_bn - 1) / pl.compress_bn;
-    cp.grid = civic::TileGrid{s_tiles, f_tiles, n_img, s_tiles * f_tiles * n_img};
-    for (int which = 0; which < 2; ++which) {
-        cp.out = which ? vc : kc;
-        const CUtensorMap& map_x = which ? map_v_in : map_k_in;
+    // K and V in one launch: the tile grid runs over 2 n_img "images"
+    cp.grid = civic::TileGrid{s_tiles, f_tiles, 2 * n_img, s_tiles * f_tiles * 2 * n_img};
+    cp.out = kc; cp.out_v = vc; cp.n_img = n_img;
+    {
         civic_status_t gs;
-        if (pl.compress_bn == 256) gs = launch_gemm<civic::CompressOp<256>>(map_r, map_x, map_r, cp, cp.grid.total, stream);
-        else if (pl.compress_bn == 192) gs = launch_gemm<civic::CompressOp<192>>(map_r, map_x, map_r, cp, cp.grid.total, stream);
-        else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_x, map_r, cp, cp.grid.total, stream);
+        if (pl.compress_bn == 256) gs = launch_gemm<civic::CompressOp<256>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
+        else if (pl.compress_bn == 192) gs = launch_gemm<civic::CompressOp<192>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
+        else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
         if (gs != CIVIC_OK) return gs;
     }
 
@@ -756,7 +756,7 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel,
                                  dim3((unsigned)((m_e + civic::kAggBM - 1) / civic::kAggBM), (unsigned)n_heads, (unsigned)n_img),
                                  (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, ap));
-    g_launches.fetch_add(4, std::memory_order_relaxed);
+    g_launches.fetch_add(3, std::memory_order_relaxed);
     return CIVIC_OK;
 }
 
