@@ -372,8 +372,10 @@ size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_
  * workspace      dev  scratch of civic_kv_compressed_attention_workspace_bytes(...) bytes,
  *                256-byte aligned (R in bf16, its column sums, K_c and V_c)
  * device_status  dev  int32, written: 0, or non-zero if a wait inside a kernel hit its time limit
+ *                or a kernel found its shared memory misplaced (the kernels then stop cleanly and
+ *                `out` is invalid).  Read it after synchronising the stream.
  * head_dim must be 64 or 128 and s a multiple of 64 up to 256: CIVIC_ERR_UNSUPPORTED otherwise.
- * Four launches and a 4-byte memset.
+ * Three launches and a 4-byte memset.
  */
 civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const void* v, const float* r,
                                              int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,

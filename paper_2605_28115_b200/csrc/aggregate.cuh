@@ -44,7 +44,7 @@ constexpr int kAggBK = 64;            // 64 bf16 = one 128-byte swizzle row
 constexpr int kScoresBN = 256;        // tokens per tile of the first GEMM
 constexpr unsigned long long kWaitLimitCycles = 1ull << 31;  // about a second
 
-enum AggError { kAggOk = 0, kAggTimeoutFull = 1, kAggTimeoutEmpty = 2, kAggTimeoutAcc = 3 };
+enum AggError { kAggOk = 0, kAggTimeoutFull = 1, kAggTimeoutEmpty = 2, kAggTimeoutAcc = 3, kAggMisaligned = 4 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
 
@@ -125,6 +125,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
         "}\n"
         ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// One lane of a converged warp (the same one every time).
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t chosen;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "elect.sync _|p, 0xFFFFFFFF;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(chosen));
+    return chosen != 0;
 }
 // The mbarrier gets one arrival once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar)

@@ -2,6 +2,7 @@
 // for the contract of every entry point.
 #include "../../include/civic.h"
 
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
@@ -644,6 +645,22 @@ struct KvAttnPlan {
     size_t r16_off, colsum_off, partial_off, kc_off, vc_off, total, attn_smem;
 };
 
+// Query tiles per block of the attention kernel: the split that needs the fewest rounds of
+// resident blocks, a block's cost being its tiles plus about a tile and a half of set-up
+// (barriers, tensor memory, the head's K_c and V_c).
+static int32_t attention_tiles_per_block(int32_t q_tiles, int64_t pairs, int blocks_per_sm)
+{
+    const int64_t resident = (int64_t)std::max(1, blocks_per_sm) * sm_count();
+    int32_t best = q_tiles;
+    double best_cost = 0.0;
+    for (int32_t per = q_tiles; per >= 1; --per) {
+        const int64_t blocks = (int64_t)((q_tiles + per - 1) / per) * pairs;
+        const double cost = (double)((blocks + resident - 1) / resident) * (per + 1.5);
+        if (per == q_tiles || cost < best_cost) { best = per; best_cost = cost; }
+    }
+    return best;
+}
+
 static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim, int32_t s,
                                         KvAttnPlan& pl)
 {
@@ -747,15 +764,42 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
         if (gs != CIVIC_OK) return gs;
     }
 
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
+    const int32_t q_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
+    CUtensorMap map_o;  // boxes of 32 rows x 64 features: one softmax warp's share of a tile
+    {
+        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
+        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32)) != CIVIC_OK) return ms;
+    }
     civic::AttnParams ap;
-    ap.out = (__nv_bfloat16*)out; ap.error = device_status;
-    ap.m_e = m_e; ap.n_heads = n_heads; ap.d = head_dim; ap.s = s;
-    ap.scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
+    ap.error = device_status; ap.m_e = m_e; ap.d = head_dim; ap.s = s;
+    ap.scale_log2e = scale_log2e;
     CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)pl.attn_smem));
+    // all of the SM's memory as shared memory, so that two blocks of 113 KB can be resident
+    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        (int)cudaSharedmemCarveoutMaxShared));
+    // Blocks that fit on an SM together, by shared memory, registers, threads and tensor memory
+    // columns.  (The runtime's occupancy query answers 1 for this kernel whatever its shared
+    // memory, while two blocks were measured running side by side on the SMs.)
+    int dev = 0, smem_per_sm = 0, reserved = 0, regs_per_sm = 0;
+    CIVIC_CUDA_TRY(cudaGetDevice(&dev));
+    CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
+    CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev));
+    CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&regs_per_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev));
+    cudaFuncAttributes fattr;
+    CIVIC_CUDA_TRY(cudaFuncGetAttributes(&fattr, civic::kv_attention_kernel));
+    const int regs_per_block = ((fattr.numRegs + 7) / 8 * 8) * civic::kAttnThreads;
+    int blocks_per_sm = (int)((size_t)smem_per_sm / (pl.attn_smem + (size_t)reserved));
+    blocks_per_sm = std::min(blocks_per_sm, regs_per_sm / std::max(regs_per_block, 1));
+    blocks_per_sm = std::min(blocks_per_sm, 2048 / civic::kAttnThreads);
+    blocks_per_sm = std::min(blocks_per_sm, (int)(512 / civic::attn_tmem_cols(head_dim, s)));
+    ap.tiles_per_block = attention_tiles_per_block(q_tiles, (int64_t)n_heads * n_img, blocks_per_sm);
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel,
-                                 dim3((unsigned)((m_e + civic::kAggBM - 1) / civic::kAggBM), (unsigned)n_heads, (unsigned)n_img),
-                                 (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, ap));
+                                 dim3((unsigned)((q_tiles + ap.tiles_per_block - 1) / ap.tiles_per_block),
+                                      (unsigned)n_heads, (unsigned)n_img),
+                                 (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, map_o, ap));
     g_launches.fetch_add(3, std::memory_order_relaxed);
     return CIVIC_OK;
 }

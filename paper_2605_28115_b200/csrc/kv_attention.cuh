@@ -4,17 +4,23 @@
 //
 // R [m_e, s] assigns the m_e compact tokens to s memory anchors; Rbar is R with every column
 // divided by its sum.  The compression is a GEMM of the persistent template (CompressOp in
-// aggregate.cuh), run once for K and once for V.  This file holds the preparation of R and the
-// attention itself: one block per (128 queries, head, image).  With at most 256 memory anchors a
-// head's whole K_c and V_c fit in shared memory, so the block issues two MMAs chains and one
-// softmax between them, with no running maximum to maintain:
-//   TMA      Q tile [128, d], K_c[:, head] [s, d] (K-major) and V_c[:, head] [s, d] (MN-major)
+// aggregate.cuh), one launch for K and V together.  This file holds the preparation of R and the
+// attention itself: one block per (range of query tiles, head, image).  With at most 256 memory
+// anchors a head's whole K_c and V_c fit in shared memory and stay there while the block walks
+// its tiles of 128 queries; per tile there are two MMA chains and one softmax between them,
+// with no running maximum to maintain:
+//   TMA      K_c[:, head] [s, d] (K-major) and V_c[:, head] [s, d] (MN-major) once; Q tiles
+//            [128, d] into a ring of two
 //   MMA 1    S = Q K_c^T -> TMEM columns [0, s)
-//   softmax  thread per query row: maximum, exp2, row sum; P as bf16 into 128-byte-swizzled
-//            shared memory (the A operand of the second chain)
-//   MMA 2    O = P V_c -> TMEM columns [0, d) again
-//   store    O / row sum as bf16
-// Every wait is bounded as in aggregate.cuh.
+//   softmax  thread per query row: maximum, exp2, row sum; P as packed bf16 straight back into
+//            TMEM, columns [0, s / 2), behind the thread's own reads of S
+//   MMA 2    O = P V_c with the A operand read from TMEM -> TMEM columns [s / 2, s / 2 + d).
+//            (With P in shared memory this chain was bound by shared-memory reads: 4 KB of P
+//            for every 2 KB of V_c and only 64 or 128 output columns to amortise them.)
+//   store    O / row sum as bf16, staged in swizzled shared memory, one bulk tensor store of
+//            32 rows per warp
+// A block is a serial chain; two blocks share an SM (shared memory and tensor memory allow it
+// for 64-wide heads) and fill each other's waits.  Every wait is bounded as in aggregate.cuh.
 #pragma once
 #include "aggregate.cuh"
 
@@ -43,55 +49,129 @@ __global__ void assign_convert_kernel(const float* __restrict__ r, int m_e, int 
 constexpr int kAttnThreads = 192;  // warp 0: TMA, warp 1: TMEM + MMA, warps 2..5: one query row per thread
 
 struct AttnParams {
-    __nv_bfloat16* out;  // [n_img, m_e, n_heads * d]
     int* error;
-    int32_t m_e, n_heads, d, s;
-    float scale_log2e;   // log2(e) / sqrt(d)
+    int32_t m_e, d, s;
+    int32_t tiles_per_block;  // query tiles of 128 rows walked by one block
+    float scale_log2e;        // log2(e) / sqrt(d)
 };
 
-// Shared memory: region A = q [d/64][128 x 128 B] | k [d/64][s x 128 B], later overwritten by
-// p [s/64][128 x 128 B] (Q and K_c are dead once the first MMA chain has completed); then
-// v [s/64][d/64][64 x 128 B]; then the barriers.  Every block of data is 1024-byte aligned.
-// 96 KB for 64-wide heads and 256 anchors: two blocks per SM.
-__host__ __device__ constexpr size_t attn_region_a_bytes(int d, int s)
+// D[tmem] (+)= A[tmem] B[smem]: A's row i on TMEM lane i, two bf16 of consecutive k per 32-bit column.
+__device__ __forceinline__ void umma_bf16_a_tmem(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate)
 {
-    const size_t qk = (size_t)(d / 64) * 16384 + (size_t)(d / 64) * s * 128, pr = (size_t)(s / 64) * 16384;
-    return qk > pr ? qk : pr;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.u32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__host__ __device__ constexpr size_t attn_smem_bytes(int d, int s)
+// 8 consecutive 32-bit columns of this warp's 32 TMEM lanes (thread t writes lane base + t)
+__device__ __forceinline__ void tmem_store8(uint32_t taddr, const uint32_t (&r)[8])
 {
-    return attn_region_a_bytes(d, s) + (size_t)(s / 64) * (d / 64) * 8192 + 1024 /* barriers */ + 1024 /* alignment slack */;
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_store_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 16 fp32 columns at a time (the exponential pass keeps its register count down with these),
+// issue and wait split as for the 32-column loads
+__device__ __forceinline__ void tmem_load_issue16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_load_wait16(uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 :: "memory");
+}
+// `cols` (a multiple of 32) columns in chunks of 16 with two register buffers
+template <class Body>
+__device__ __forceinline__ void for_each_chunk16(uint32_t taddr, int cols, Body&& body)
+{
+    uint32_t even[16], odd[16];
+    tmem_load_issue16(taddr, even);
+#pragma unroll 1
+    for (int c0 = 0; c0 < cols; c0 += 32) {
+        tmem_load_wait16(even);
+        tmem_load_issue16(taddr + c0 + 16, odd);
+        body(even, c0);
+        tmem_load_wait16(odd);
+        if (c0 + 32 < cols) tmem_load_issue16(taddr + c0 + 32, even);
+        body(odd, c0 + 16);
+    }
 }
 
-__global__ void __launch_bounds__(kAttnThreads) kv_attention_kernel(const __grid_constant__ CUtensorMap map_q,
+// Shared memory: k [d/64][s x 128 B] | v [s/64][d/64][64 x 128 B] | q [2][d/64][128 x 128 B] |
+// o [4 warps][d/64][32 x 128 B] | barriers.  Every block of data is 1024-byte aligned; the
+// kernel has no static shared memory, so the dynamic window itself starts on such a boundary
+// (checked at run time) and no slack is set aside: 113 KB for 64-wide heads and 256 anchors is
+// exactly what lets two blocks share an SM; 225 KB for 128-wide heads.
+__host__ __device__ constexpr size_t attn_smem_bytes(int d, int s)
+{
+    return (size_t)(d / 64) * s * 128 + (size_t)(s / 64) * (d / 64) * 8192 + 2 * (size_t)(d / 64) * 16384 +
+           4 * (size_t)(d / 64) * 4096 + 1024 /* barriers */;
+}
+// TMEM columns of a block: S in [0, s), later P in [0, s / 2) and O in [s / 2, s / 2 + d)
+__host__ __device__ constexpr uint32_t attn_tmem_cols(int d, int s)
+{
+    const int need = s > s / 2 + d ? s : s / 2 + d;
+    return need <= 32 ? 32u : (need <= 64 ? 64u : (need <= 128 ? 128u : 256u));
+}
+
+// Registers are handed out per group of four warps, so a block of six warps is charged for eight:
+// bounding the kernel as if it had 256 threads, two blocks per SM, keeps it at 128 registers.
+__global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                     const __grid_constant__ CUtensorMap map_k,
                                                                     const __grid_constant__ CUtensorMap map_v,
+                                                                    const __grid_constant__ CUtensorMap map_o,
                                                                     const AttnParams p)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t attn_smem[];
+    uint8_t* base = attn_smem;
+    if (smem_u32(base) & 1023u) {  // the swizzled tiles would be misplaced: refuse, before anything is set up
+        if (threadIdx.x == 0) atomicCAS(p.error, 0, kAggMisaligned);
+        return;
+    }
     const int d = p.d, s = p.s, d_blocks = d >> 6, s_blocks = s >> 6;
-    uint8_t* q_sm = base;
-    uint8_t* k_sm = q_sm + d_blocks * 16384;
-    uint8_t* p_sm = base;  // takes over the Q / K_c region after the first MMA chain
-    uint8_t* v_sm = base + attn_region_a_bytes(d, s);
+    uint8_t* k_sm = base;
+    uint8_t* v_sm = k_sm + d_blocks * s * 128;
+    uint8_t* q_sm = v_sm + s_blocks * d_blocks * 8192;
+    uint8_t* o_sm = q_sm + 2 * d_blocks * 16384;
     struct Sync {
-        uint64_t loaded, scores_done, probs_ready, out_done;
+        uint64_t k_loaded, v_loaded, q_full[2], q_empty[2], s_full, s_free, p_ready, o_done;
         uint32_t tmem_base;
         int abort;
     };
-    Sync& sy = *reinterpret_cast<Sync*>(v_sm + s_blocks * d_blocks * 8192);
+    Sync& sy = *reinterpret_cast<Sync*>(o_sm + 4 * d_blocks * 4096);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kAggBM, head = blockIdx.y, img = blockIdx.z;
+    const int head = blockIdx.y, img = blockIdx.z;
+    const int tiles_total = (p.m_e + kAggBM - 1) / kAggBM;
+    const int first = blockIdx.x * p.tiles_per_block;
+    const int n_tiles = min(p.tiles_per_block, tiles_total - first);
     volatile int* abort = &sy.abort;
-    // O takes over the first d columns of S (S is dead once every softmax warp has read it)
-    const uint32_t tmem_cols = max(s, d) <= 64 ? 64u : (max(s, d) <= 128 ? 128u : 256u);
+    const uint32_t tmem_cols = attn_tmem_cols(d, s);
+    const uint32_t o_col = (uint32_t)(s >> 1);
 
     if (threadIdx.x == 0) {
-        mbar_init(&sy.loaded, 1);
-        mbar_init(&sy.scores_done, 1);
-        mbar_init(&sy.probs_ready, 4);  // one arrival per softmax warp
-        mbar_init(&sy.out_done, 1);
+        mbar_init(&sy.k_loaded, 1);
+        mbar_init(&sy.v_loaded, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sy.q_full[b], 1);
+            mbar_init(&sy.q_empty[b], 1);
+        }
+        mbar_init(&sy.s_full, 1);
+        mbar_init(&sy.s_free, 4);   // one arrival per softmax warp
+        mbar_init(&sy.p_ready, 4);
+        mbar_init(&sy.o_done, 1);
         sy.abort = 0;
         fence_barrier_init();
     }
@@ -100,112 +180,143 @@ __global__ void __launch_bounds__(kAttnThreads) kv_attention_kernel(const __grid
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_s = sy.tmem_base, tmem_o = sy.tmem_base;
-    const bool stop = *p.error != 0;
+    const uint32_t tmem_base = sy.tmem_base;
+    const bool stop = *p.error != 0 || n_tiles <= 0;
 
+    // A wait on a "free / empty" barrier uses the opposite parity, so the first pass over a
+    // fresh barrier falls through.
     if (warp == 0 && lane == 0 && !stop) {
-        // ---- all operands of this block, one barrier
-        const uint32_t bytes = d_blocks * 16384 + d_blocks * s * 128 + s_blocks * d_blocks * 8192;
-        mbar_expect_tx(&sy.loaded, bytes);
-        for (int db = 0; db < d_blocks; ++db) {
-            tma_load_3d(q_sm + db * 16384, &map_q, head * d + db * 64, m0, img, &sy.loaded);
+        // ---- producer
+        mbar_expect_tx(&sy.k_loaded, d_blocks * s * 128);
+        for (int db = 0; db < d_blocks; ++db)
             for (int r0 = 0; r0 < s; r0 += 64)  // boxes of 64 anchors
-                tma_load_3d(k_sm + db * s * 128 + r0 * 128, &map_k, head * d + db * 64, r0, img, &sy.loaded);
-        }
-        for (int sb = 0; sb < s_blocks; ++sb)
+                tma_load_3d(k_sm + db * s * 128 + r0 * 128, &map_k, head * d + db * 64, r0, img, &sy.k_loaded);
+        for (int t = 0; t < n_tiles; ++t) {
+            const int st = t & 1;
+            if (!mbar_wait(&sy.q_empty[st], ((t >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) break;
+            mbar_expect_tx(&sy.q_full[st], d_blocks * 16384);
             for (int db = 0; db < d_blocks; ++db)
-                tma_load_3d(v_sm + (sb * d_blocks + db) * 8192, &map_v, head * d + db * 64, sb * 64, img, &sy.loaded);
-    } else if (warp == 1 && lane == 0 && !stop) {
-        // ---- MMA 1: S[128, s] = Q K_c^T, K = d
-        if (mbar_wait(&sy.loaded, 0, abort, p.error, kAggTimeoutFull)) {
-            tc_fence_after_sync();
-            const uint32_t idesc1 = umma_idesc(s, 0);
-            for (int db = 0; db < d_blocks; ++db)
-                for (int kk = 0; kk < 4; ++kk)
-                    umma_bf16(tmem_s, umma_desc(smem_u32(q_sm + db * 16384) + kk * 32, 16, 1024),
-                              umma_desc(smem_u32(k_sm + db * s * 128) + kk * 32, 16, 1024), idesc1, (db | kk) != 0);
-            umma_commit(&sy.scores_done);
-            // ---- MMA 2: O[128, d] = P V_c, K = s; B blocks of 64 features are 8 KB apart
-            if (mbar_wait(&sy.probs_ready, 0, abort, p.error, kAggTimeoutAcc)) {
-                tc_fence_after_sync();
-                const uint32_t idesc2 = umma_idesc(d, 1);
+                tma_load_3d(q_sm + (st * d_blocks + db) * 16384, &map_q, head * d + db * 64, (first + t) * kAggBM, img,
+                            &sy.q_full[st]);
+            if (t == 0) {  // V_c is not needed before the second chain of the first tile
+                mbar_expect_tx(&sy.v_loaded, s_blocks * d_blocks * 8192);
                 for (int sb = 0; sb < s_blocks; ++sb)
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma_bf16(tmem_o, umma_desc(smem_u32(p_sm + sb * 16384) + kk * 32, 16, 1024),
-                                  umma_desc(smem_u32(v_sm + sb * d_blocks * 8192) + kk * 2048, 8192, 1024), idesc2,
-                                  (sb | kk) != 0);
-                umma_commit(&sy.out_done);
+                    for (int db = 0; db < d_blocks; ++db)
+                        tma_load_3d(v_sm + (sb * d_blocks + db) * 8192, &map_v, head * d + db * 64, sb * 64, img,
+                                    &sy.v_loaded);
             }
+        }
+        if (*abort) {  // copies still in flight after a time-out: give them ample time to land
+            const long long t0 = clock64();
+            while ((unsigned long long)(clock64() - t0) < (1ull << 22)) {}
+        }
+    } else if (warp == 1 && lane == 0 && !stop) {
+        // ---- MMA issue.  One descriptor per shared-memory operand, built once; a tile or K step
+        // further on only moves the start-address field (16-byte units in the low bits; shared
+        // memory addresses never carry out of it).
+        const uint32_t idesc1 = umma_idesc(s, 0), idesc2 = umma_idesc(d, 1);
+        const uint64_t desc_q = umma_desc(smem_u32(q_sm), 16, 1024), desc_k = umma_desc(smem_u32(k_sm), 16, 1024);
+        const uint64_t desc_v = umma_desc(smem_u32(v_sm), 8192, 1024);
+        bool ok = mbar_wait(&sy.k_loaded, 0, abort, p.error, kAggTimeoutFull);
+        for (int t = 0; ok && t < n_tiles; ++t) {
+            const int st = t & 1;
+            // S[128, s] = Q(t) K_c^T, K = d; the previous tile's O has been read out of these columns
+            if (!(ok = mbar_wait(&sy.q_full[st], (t >> 1) & 1, abort, p.error, kAggTimeoutFull))) break;
+            if (!(ok = mbar_wait(&sy.s_free, (t & 1) ^ 1, abort, p.error, kAggTimeoutAcc))) break;
+            tc_fence_after_sync();
+            for (int db = 0; db < d_blocks; ++db) {
+                const uint64_t a = desc_q + (uint64_t)(((st * d_blocks + db) * 16384) >> 4);
+                const uint64_t b = desc_k + (uint64_t)((db * s * 128) >> 4);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base, a + 2 * kk, b + 2 * kk, idesc1, (db | kk) != 0);
+            }
+            umma_commit(&sy.q_empty[st]);
+            umma_commit(&sy.s_full);
+            if (t == 0 && !(ok = mbar_wait(&sy.v_loaded, 0, abort, p.error, kAggTimeoutFull))) break;
+            // O[128, d] = P V_c, K = s: A from TMEM (8 columns per K step of 16), B blocks of 64
+            // anchors are d_blocks x 8 KB apart, K steps inside a block 2 KB
+            if (!(ok = mbar_wait(&sy.p_ready, t & 1, abort, p.error, kAggTimeoutAcc))) break;
+            tc_fence_after_sync();
+            for (int sb = 0; sb < s_blocks; ++sb) {
+                const uint64_t b = desc_v + (uint64_t)((sb * d_blocks * 8192) >> 4);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_bf16_a_tmem(tmem_base + o_col, tmem_base + (uint32_t)(sb * 32 + kk * 8), b + 128 * kk, idesc2,
+                                     (sb | kk) != 0);
+            }
+            umma_commit(&sy.o_done);
         }
     } else if (warp >= 2 && !stop) {
         // ---- softmax and output: thread = query row (TMEM lane) 32 * (warp % 4) + lane
         const int quarter = warp & 3;
-        const int row = quarter * 32 + lane;
-        const int m = m0 + row;
-        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        if (__all_sync(0xFFFFFFFFu, mbar_wait(&sy.scores_done, 0, abort, p.error, kAggTimeoutAcc))) {
+        const uint32_t tm = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        uint8_t* o_stage = o_sm + (warp - 2) * d_blocks * 4096;  // [d/64][32 rows x 128 B], swizzled
+        for (int t = 0; t < n_tiles; ++t) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.s_full, t & 1, abort, p.error, kAggTimeoutAcc))) break;
             tc_fence_after_sync();
-            float mx = -3.0e38f;
-            for_each_chunk(tmem_s + lane_addr, s, [&](const uint32_t (&acc)[32], int) {
+            float mx4[4] = {-3.0e38f, -3.0e38f, -3.0e38f, -3.0e38f};  // four chains instead of one
+            for_each_chunk(tm, s, [&](const uint32_t (&acc)[32], int) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(acc[c]));
+                for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(acc[c]));
             });
-            const float shift = mx * p.scale_log2e;
+            const float shift = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;
+            // P(row, c) for the 16 columns of a chunk -> 8 packed columns at c / 2: always behind
+            // the columns of S this thread has already taken into registers
             float row_sum = 0.f;
-            for_each_chunk(tmem_s + lane_addr, s, [&](const uint32_t (&acc)[32], int c0) {
-                uint8_t* blk = p_sm + (c0 >> 6) * 16384 + row * 128;  // this row in the 64-column block
-                const int j0 = (c0 & 32) >> 3;                        // first 16-byte piece of the chunk
+            for_each_chunk16(tm, s, [&](const uint32_t (&acc)[16], int c0) {
+                uint32_t w[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float x0 = exp2_fast(fmaf(__uint_as_float(acc[2 * e]), p.scale_log2e, -shift));
+                    const float x1 = exp2_fast(fmaf(__uint_as_float(acc[2 * e + 1]), p.scale_log2e, -shift));
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);  // x0 in the low half
+                    row_sum += __low2float(h) + __high2float(h);
+                    w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                tmem_store8(tm + (uint32_t)(c0 >> 1), w);
+            });
+            tmem_store_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sy.p_ready);
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.o_done, t & 1, abort, p.error, kAggTimeoutAcc))) break;
+            tc_fence_after_sync();
+            const float inv = 1.f / row_sum;  // at least one term is exp2(0) = 1
+            if (lane == 0) tma_store_wait_read();  // the previous tile's store has read the staging rows
+            __syncwarp();
+            for_each_chunk(tm + o_col, d, [&](const uint32_t (&acc)[32], int c0) {
+                uint8_t* blk = o_stage + (c0 >> 6) * 4096 + lane * 128;  // this row in the 64-column block
+                const int j0 = (c0 & 32) >> 3;                           // first 16-byte piece of the chunk
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     uint32_t w[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float a = exp2_fast(fmaf(__uint_as_float(acc[q4 * 8 + 2 * e]), p.scale_log2e, -shift));
-                        const float b = exp2_fast(fmaf(__uint_as_float(acc[q4 * 8 + 2 * e + 1]), p.scale_log2e, -shift));
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-                        row_sum += __low2float(h) + __high2float(h);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv,
+                                                                       __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv);
                         w[e] = *reinterpret_cast<const uint32_t*>(&h);
                     }
-                    *reinterpret_cast<uint4*>(blk + (((j0 + q4) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(blk + (((j0 + q4) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             });
-            fence_async_smem();      // the MMA reads P through the async proxy
-            tc_fence_before_sync();  // and S has been read out of TMEM
+            fence_async_smem();      // the bulk store reads the staging rows through the async proxy
+            tc_fence_before_sync();  // and O has been read out of TMEM
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sy.probs_ready);
-            if (__all_sync(0xFFFFFFFFu, mbar_wait(&sy.out_done, 0, abort, p.error, kAggTimeoutAcc))) {
-                tc_fence_after_sync();
-                const float inv = 1.f / row_sum;  // at least one term is exp2(0) = 1
-                const bool row_ok = m < p.m_e;
-                __nv_bfloat16* out = p.out + ((size_t)img * p.m_e + (row_ok ? m : 0)) * (p.n_heads * d) + head * d;
-                for_each_chunk(tmem_o + lane_addr, d, [&](const uint32_t (&acc)[32], int c0) {
-                    if (row_ok) {
-#pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv,
-                                                                               __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv);
-                                w[e] = *reinterpret_cast<const uint32_t*>(&h);
-                            }
-                            *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    }
-                });
+            if (lane == 0) {
+                const int m_first = (first + t) * kAggBM + quarter * 32;
+                if (m_first < p.m_e)  // rows past m_e are clipped by the store
+                    for (int db = 0; db < d_blocks; ++db)
+                        tma_store_3d(&map_o, o_stage + db * 4096, head * d + db * 64, m_first, img);
+                mbar_arrive(&sy.s_free);
             }
         }
-    }
-    // copies still in flight after a time-out: give them ample time before the block goes away
-    if (*abort && warp == 0 && lane == 0) {
-        const long long t0 = clock64();
-        while (!mbar_try_wait(&sy.loaded, 0) && (unsigned long long)(clock64() - t0) < kWaitLimitCycles) {}
+        if (lane == 0) tma_store_wait_read();
     }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(sy.tmem_base, tmem_cols);
+        tmem_dealloc(tmem_base, tmem_cols);
     }
 }
 
