@@ -363,8 +363,9 @@ size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_
  * R [m_e, s] the KV assignment matrix onto s memory anchors (non-negative, every column with a
  * positive sum), Rbar = R with every column divided by its sum, d = head_dim.  Heads split the
  * feature dimension into n_heads contiguous blocks of head_dim; the softmax runs over the s
- * anchors.  bf16 tensor-core products with fp32 accumulation; K_c, V_c and the softmax weights
- * are rounded to bf16 on the way.
+ * anchors.  bf16 tensor-core products with fp32 accumulation; K_c and V_c are rounded to bf16
+ * on the way, the unnormalised softmax weights are cut to bf16 and divided by the sum of the
+ * cut values.
  *
  * q, k, v        dev  bf16 [n_img, m_e, n_heads * head_dim], 16-byte aligned
  * r              dev  fp32 [m_e, s], shared by the images

@@ -697,18 +697,27 @@ struct CompressOp {
     }
     static __device__ __forceinline__ uint64_t a_desc(uint32_t a0, int kk) { return umma_desc(a0 + kk * 2048, kAggBK * 128, 1024); }
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
-    static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, const Tile&) {}
-    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, const CUtensorMap*, uint32_t tmem, int ewarp,
+    // Before the accumulator is waited for: the divisor of this thread's row (memory anchor),
+    // the panels' column sums added in a fixed order so that every tile gets the same value.
+    // It waits in the thread's own shared-memory slot (the statistics array is unused here).
+    static __device__ __forceinline__ void prefetch(const Params& p, Smem& sm, int ewarp, int lane, const Tile& tl)
+    {
+        const int row = tl.m_tile * kAggBM + (ewarp & 3) * 32 + lane;
+        float sum = 0.f;
+        if (row < p.s) {
+#pragma unroll 8
+            for (int q = 0; q < p.n_parts; ++q) sum += __ldg(p.colsum_parts + (size_t)q * p.s + row);
+        }
+        reinterpret_cast<float*>(sm.stats[0])[ewarp * 32 + lane] = sum > 0.f ? 1.f / sum : 0.f;
+    }
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap*, uint32_t tmem, int ewarp,
                                                     int lane, int m0, const Tile& tl)
     {
         const int half_cols = tl.n >> 1;
         const int quarter = ewarp & 3, half = ewarp >> 2;
         const int row = m0 + quarter * 32 + lane;  // memory anchor
         const bool row_ok = row < p.s;
-        float sum = 0.f;  // fixed order of additions: every tile gets the same divisor
-        if (row_ok)
-            for (int q = 0; q < p.n_parts; ++q) sum += p.colsum_parts[(size_t)q * p.s + row];
-        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        const float inv = reinterpret_cast<const float*>(sm.stats[0])[ewarp * 32 + lane];
         const int nh = tl.n0 + half * half_cols;
         const bool second = tl.img >= p.n_img;
         __nv_bfloat16* out = (second ? p.out_v : p.out) +

@@ -12,8 +12,8 @@
 //   TMA      K_c[:, head] [s, d] (K-major) and V_c[:, head] [s, d] (MN-major) once; Q tiles
 //            [128, d] into a ring of two
 //   MMA 1    S = Q K_c^T -> TMEM columns [0, s)
-//   softmax  thread per query row: maximum, exp2, row sum; P as packed bf16 straight back into
-//            TMEM, columns [0, s / 2), behind the thread's own reads of S
+//   softmax  thread per query row: maximum, exp2, row sum; P cut to bf16 and packed straight back
+//            into TMEM, columns [0, s / 2), behind the thread's own reads of S
 //   MMA 2    O = P V_c with the A operand read from TMEM -> TMEM columns [s / 2, s / 2 + d).
 //            (With P in shared memory this chain was bound by shared-memory reads: 4 KB of P
 //            for every 2 KB of V_c and only 64 or 128 output columns to amortise them.)
@@ -37,8 +37,9 @@ __global__ void assign_convert_kernel(const float* __restrict__ r, int m_e, int 
     const int m_begin = blockIdx.x * kAssignRows, m_end = min(m_begin + kAssignRows, m_e);
     for (int c = threadIdx.x; c < s; c += blockDim.x) {
         float sum = 0.f;
-#pragma unroll 4
-        for (int m = m_begin; m < m_end; ++m) {
+#pragma unroll
+        for (int m = m_begin; m < m_begin + kAssignRows; ++m) {
+            if (m >= m_end) break;
             const __nv_bfloat16 v = __float2bfloat16_rn(r[(size_t)m * s + c]);
             r16[(size_t)m * s + c] = v;
             sum += __bfloat162float(v);
@@ -152,7 +153,9 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
         int abort;
     };
     Sync& sy = *reinterpret_cast<Sync*>(o_sm + 4 * d_blocks * 4096);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the warp index through a shuffle: the compiler then knows it is the same in all lanes and
+    // keeps what depends only on it (the MMA warp's addresses and descriptors) in uniform registers
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int head = blockIdx.y, img = blockIdx.z;
     const int tiles_total = (p.m_e + kAggBM - 1) / kAggBM;
     const int first = blockIdx.x * p.tiles_per_block;
@@ -210,41 +213,53 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
             const long long t0 = clock64();
             while ((unsigned long long)(clock64() - t0) < (1ull << 22)) {}
         }
-    } else if (warp == 1 && lane == 0 && !stop) {
-        // ---- MMA issue.  One descriptor per shared-memory operand, built once; a tile or K step
-        // further on only moves the start-address field (16-byte units in the low bits; shared
-        // memory addresses never carry out of it).
+    } else if (warp == 1 && !stop) {
+        // ---- MMA issue.  The whole warp walks the loop and the waits in step, one elected lane
+        // issues: a lone lane would hold every operand in its own registers and pay for moving
+        // them to the uniform registers the instruction reads, which made the 16 MMAs of the
+        // second chain take longer to issue than to run.  One descriptor per shared-memory
+        // operand, built once; a tile or K step further on only moves the start-address field
+        // (16-byte units in the low bits; shared memory addresses never carry out of it).
         const uint32_t idesc1 = umma_idesc(s, 0), idesc2 = umma_idesc(d, 1);
         const uint64_t desc_q = umma_desc(smem_u32(q_sm), 16, 1024), desc_k = umma_desc(smem_u32(k_sm), 16, 1024);
         const uint64_t desc_v = umma_desc(smem_u32(v_sm), 8192, 1024);
-        bool ok = mbar_wait(&sy.k_loaded, 0, abort, p.error, kAggTimeoutFull);
+        auto wait = [&](uint64_t* bar, uint32_t parity, int code) {
+            return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort, p.error, code)) != 0;
+        };
+        bool ok = wait(&sy.k_loaded, 0, kAggTimeoutFull);
         for (int t = 0; ok && t < n_tiles; ++t) {
             const int st = t & 1;
             // S[128, s] = Q(t) K_c^T, K = d; the previous tile's O has been read out of these columns
-            if (!(ok = mbar_wait(&sy.q_full[st], (t >> 1) & 1, abort, p.error, kAggTimeoutFull))) break;
-            if (!(ok = mbar_wait(&sy.s_free, (t & 1) ^ 1, abort, p.error, kAggTimeoutAcc))) break;
+            if (!(ok = wait(&sy.q_full[st], (t >> 1) & 1, kAggTimeoutFull))) break;
+            if (!(ok = wait(&sy.s_free, (t & 1) ^ 1, kAggTimeoutAcc))) break;
             tc_fence_after_sync();
             for (int db = 0; db < d_blocks; ++db) {
                 const uint64_t a = desc_q + (uint64_t)(((st * d_blocks + db) * 16384) >> 4);
                 const uint64_t b = desc_k + (uint64_t)((db * s * 128) >> 4);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base, a + 2 * kk, b + 2 * kk, idesc1, (db | kk) != 0);
+                for (int kk = 0; kk < 4; ++kk)
+                    if (elect_one()) umma_bf16(tmem_base, a + 2 * kk, b + 2 * kk, idesc1, (db | kk) != 0);
             }
-            umma_commit(&sy.q_empty[st]);
-            umma_commit(&sy.s_full);
-            if (t == 0 && !(ok = mbar_wait(&sy.v_loaded, 0, abort, p.error, kAggTimeoutFull))) break;
+            if (elect_one()) {
+                umma_commit(&sy.q_empty[st]);
+                umma_commit(&sy.s_full);
+            }
+            __syncwarp();
+            if (t == 0 && !(ok = wait(&sy.v_loaded, 0, kAggTimeoutFull))) break;
             // O[128, d] = P V_c, K = s: A from TMEM (8 columns per K step of 16), B blocks of 64
             // anchors are d_blocks x 8 KB apart, K steps inside a block 2 KB
-            if (!(ok = mbar_wait(&sy.p_ready, t & 1, abort, p.error, kAggTimeoutAcc))) break;
+            if (!(ok = wait(&sy.p_ready, t & 1, kAggTimeoutAcc))) break;
             tc_fence_after_sync();
             for (int sb = 0; sb < s_blocks; ++sb) {
                 const uint64_t b = desc_v + (uint64_t)((sb * d_blocks * 8192) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
-                    umma_bf16_a_tmem(tmem_base + o_col, tmem_base + (uint32_t)(sb * 32 + kk * 8), b + 128 * kk, idesc2,
-                                     (sb | kk) != 0);
+                    if (elect_one())
+                        umma_bf16_a_tmem(tmem_base + o_col, tmem_base + (uint32_t)(sb * 32 + kk * 8), b + 128 * kk, idesc2,
+                                         (sb | kk) != 0);
             }
-            umma_commit(&sy.o_done);
+            if (elect_one()) umma_commit(&sy.o_done);
+            __syncwarp();
         }
     } else if (warp >= 2 && !stop) {
         // ---- softmax and output: thread = query row (TMEM lane) 32 * (warp % 4) + lane
@@ -267,11 +282,14 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float x0 = exp2_fast(fmaf(__uint_as_float(acc[2 * e]), p.scale_log2e, -shift));
-                    const float x1 = exp2_fast(fmaf(__uint_as_float(acc[2 * e + 1]), p.scale_log2e, -shift));
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);  // x0 in the low half
-                    row_sum += __low2float(h) + __high2float(h);
-                    w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                    // The weights are cut to bf16 (upper halves of the fp32 words), not rounded: a
+                    // rounding conversion shares its pipe with exp2, which already bounds this
+                    // pass.  The row sum adds the cut values, so the common part of the error
+                    // cancels in O / row sum.
+                    const uint32_t x0 = __float_as_uint(exp2_fast(fmaf(__uint_as_float(acc[2 * e]), p.scale_log2e, -shift)));
+                    const uint32_t x1 = __float_as_uint(exp2_fast(fmaf(__uint_as_float(acc[2 * e + 1]), p.scale_log2e, -shift)));
+                    row_sum += __uint_as_float(x0 & 0xFFFF0000u) + __uint_as_float(x1 & 0xFFFF0000u);
+                    w[e] = __byte_perm(x0, x1, 0x7632);  // x0's upper half below x1's
                 }
                 tmem_store8(tm + (uint32_t)(c0 >> 1), w);
             });
@@ -285,6 +303,11 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
             if (lane == 0) tma_store_wait_read();  // the previous tile's store has read the staging rows
             __syncwarp();
             for_each_chunk(tm + o_col, d, [&](const uint32_t (&acc)[32], int c0) {
+                if (c0 + 32 >= d) {  // the last of O is in registers: the next tile's S may overwrite it
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sy.s_free);
+                }
                 uint8_t* blk = o_stage + (c0 >> 6) * 4096 + lane * 128;  // this row in the 64-column block
                 const int j0 = (c0 & 32) >> 3;                           // first 16-byte piece of the chunk
 #pragma unroll
@@ -299,15 +322,13 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
                     *reinterpret_cast<uint4*>(blk + (((j0 + q4) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             });
-            fence_async_smem();      // the bulk store reads the staging rows through the async proxy
-            tc_fence_before_sync();  // and O has been read out of TMEM
+            fence_async_smem();  // the bulk store reads the staging rows through the async proxy
             __syncwarp();
             if (lane == 0) {
                 const int m_first = (first + t) * kAggBM + quarter * 32;
                 if (m_first < p.m_e)  // rows past m_e are clipped by the store
                     for (int db = 0; db < d_blocks; ++db)
                         tma_store_3d(&map_o, o_stage + db * 4096, head * d + db * 64, m_first, img);
-                mbar_arrive(&sy.s_free);
             }
         }
         if (lane == 0) tma_store_wait_read();

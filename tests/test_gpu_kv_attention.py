@@ -4,8 +4,10 @@ Tolerance, from the arithmetic of the CUDA path (bf16 inputs, the same for both 
   * K_c and V_c are weighted averages taken with bf16-rounded weights (relative 2^-9), accumulated in
     fp32 and rounded to bf16 (2^-9): each is off by at most 2^-8 of the same average of absolute values;
   * a logit q . k_c / sqrt(d) is therefore off by at most lam = 2^-8 * max (|q| . |K_c|) / sqrt(d), a
-    softmax weight by the factor exp(2 lam), plus 2^-8 for its bf16 rounding and that of the row sum:
-        eps_w = exp(2 lam) - 1 + 2^-8;
+    softmax weight by the factor exp(2 lam); the weights are cut (not rounded) to bf16, each losing a
+    fraction in [0, 2^-8], and normalised by the sum of the cut weights, which loses a fraction in the
+    same range: a normalised weight moves by at most the factor 1 / (1 - 2^-8):
+        eps_w = exp(2 lam) - 1 + 2^-8 (1 + 2^-7);
   * out = W V_c inherits eps_w from the weights and 2^-8 from V_c, relative to W |V_c|, plus 2^-9 |out|
     for the bf16 result:   |out_gpu - out_oracle| <= (eps_w + 2^-8) (W |V_c|) + 2^-9 |out|.
 """
@@ -62,7 +64,7 @@ def check(q, k, v, r, heads):
         for h in range(heads):
             c = slice(h * d, (h + 1) * d)
             lam = 2.0 ** -8 * np.max(np.abs(q64[:, c]) @ abs_kc[:, c].T) / np.sqrt(d)
-            eps_w = np.expm1(2 * lam) + 2.0 ** -8
+            eps_w = np.expm1(2 * lam) + 2.0 ** -8 * (1 + 2.0 ** -7)
             logits = q64[:, c] @ k_c[:, c].T / np.sqrt(d)
             w = np.exp(logits - logits.max(axis=1, keepdims=True))
             w /= w.sum(axis=1, keepdims=True)
