@@ -99,8 +99,11 @@ civic_status_t civic_select_seq(const float* scores, int32_t n_seq, const civic_
  *
  * Paper: as civic_select; the paper's stated next step is long-form video (Section 5), where
  * one segment has far more tokens than a thread block can hold.  Same definition and the same
- * output as civic_select for any n up to 2^31 - 1, computed by many thread blocks per segment
- * in five consecutive launches that communicate through `workspace`.
+ * output as civic_select for any n up to 2^31 - 1, computed by many thread blocks per segment:
+ * in five consecutive launches that communicate through `workspace`, or, with the library's own
+ * chunking (chunk_tokens = 0) and where that is the faster of the two (segments up to 16 384
+ * tokens, batches of segments up to 65 536), in ONE launch of a cluster of four thread blocks
+ * per segment that communicate through distributed shared memory and leave `workspace` alone.
  *
  * workspace        dev, caller-owned scratch of at least civic_select_workspace_bytes(...)
  *                  bytes, 256-byte aligned; contents on entry are irrelevant, contents on return

@@ -55,7 +55,7 @@ __device__ __forceinline__ int region_row_start(const LargeParams& p, int g)
 __device__ __forceinline__ void chunk_range(const LargeParams& p, int chunk, int& g0, int& g1, int& tok0,
                                             int& tok1)
 {
-    g0 = chunk * p.rows_per_chunk;
+    g0 = min(chunk * p.rows_per_chunk, p.t * p.n_rh);  // a block past the last region row gets nothing
     g1 = min(g0 + p.rows_per_chunk, p.t * p.n_rh);
     tok0 = region_row_start(p, g0);
     tok1 = region_row_start(p, g1);
@@ -64,13 +64,11 @@ __device__ __forceinline__ void chunk_range(const LargeParams& p, int chunk, int
 // Block-wide search of a finished histogram: the bin (counted from the top) that holds the
 // rank-th candidate, and the rank inside that bin.  Every thread returns the same pair.
 // `tmp` is 34 words of shared memory.
-__device__ __forceinline__ void find_digit(const uint32_t* __restrict__ ghist, int bins, uint32_t rank,
-                                           uint32_t* tmp, uint32_t& digit, uint32_t& rank_in_bin)
+// Thread `tid` brings the counts of bins 2*tid and 2*tid+1 (0 beyond the histogram).
+__device__ __forceinline__ void find_digit_counts(uint32_t c_lo, uint32_t c_hi, uint32_t rank, uint32_t* tmp,
+                                                  uint32_t& digit, uint32_t& rank_in_bin)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // thread `tid` owns bins 2*tid and 2*tid+1 (none beyond `bins`)
-    const uint32_t c_lo = 2 * tid < bins ? ghist[2 * tid] : 0u;
-    const uint32_t c_hi = 2 * tid + 1 < bins ? ghist[2 * tid + 1] : 0u;
     const uint32_t local = c_lo + c_hi;
     uint32_t incl = local;  // sum over the threads >= mine of my warp
 #pragma unroll
@@ -92,6 +90,14 @@ __device__ __forceinline__ void find_digit(const uint32_t* __restrict__ ghist, i
     __syncthreads();
 }
 
+__device__ __forceinline__ void find_digit(const uint32_t* __restrict__ ghist, int bins, uint32_t rank,
+                                           uint32_t* tmp, uint32_t& digit, uint32_t& rank_in_bin)
+{
+    const int tid = threadIdx.x;
+    find_digit_counts(2 * tid < bins ? ghist[2 * tid] : 0u, 2 * tid + 1 < bins ? ghist[2 * tid + 1] : 0u, rank, tmp,
+                      digit, rank_in_bin);
+}
+
 // Adds a block's shared-memory histogram to the segment's global one.
 __device__ __forceinline__ void flush_hist(uint32_t* shist, uint32_t* ghist, int bins)
 {
@@ -101,26 +107,12 @@ __device__ __forceinline__ void flush_hist(uint32_t* shist, uint32_t* ghist, int
     }
 }
 
-// K1: floor + histogram of key bits 31..21.
-__global__ void __launch_bounds__(kLargeThreads) large_floor_kernel(const __grid_constant__ LargeParams p)
+// The retention floor inside one chunk: bit i of `resv` (zeroed by the caller) is set for the
+// reserved tokens; `keys` holds the chunk's keys.  Whole tiles only, by the choice of the chunks.
+__device__ __forceinline__ void chunk_floor(const LargeParams& p, const uint32_t* keys, uint32_t* resv, int g0, int g1,
+                                            int tok0, int cn, int cn_pad)
 {
-    extern __shared__ __align__(16) uint32_t smem[];
-    uint32_t* shist = smem;                       // [kLargeBins]
-    uint32_t* resv = shist + kLargeBins;          // [kLargeMaxChunk / 32] bit per chunk-local token
-    uint32_t* keys = resv + kLargeMaxChunk / 32;  // [chunk tokens]
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
-    const int seg = blockIdx.x / p.n_chunks, chunk = blockIdx.x - seg * p.n_chunks;
-    int g0, g1, tok0, tok1;
-    chunk_range(p, chunk, g0, g1, tok0, tok1);
-    const int cn = tok1 - tok0, cn_pad = (cn + 31) & ~31;
-    const float* scores = p.scores + (size_t)seg * p.n + tok0;
-    wait_for_prior_kernels();
-
-    for (int i = tid; i < cn_pad; i += nt) keys[i] = i < cn ? score_key(__ldg(scores + i)) : 0u;
-    for (int b = tid; b < kLargeBins; b += nt) shist[b] = 0u;
-    for (int i = tid; i < kLargeMaxChunk / 32; i += nt) resv[i] = 0u;
-    __syncthreads();
-
     const int n_rw = (p.w + p.region_w - 1) / p.region_w;
     if (p.m == 1) {
         // one thread per tile walks it in index order and keeps the first maximum
@@ -167,6 +159,29 @@ __global__ void __launch_bounds__(kLargeThreads) large_floor_kernel(const __grid
             if (lane == 0) resv[i >> 5] = word;
         }
     }
+}
+
+// K1: floor + histogram of key bits 31..21.
+__global__ void __launch_bounds__(kLargeThreads) large_floor_kernel(const __grid_constant__ LargeParams p)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* shist = smem;                       // [kLargeBins]
+    uint32_t* resv = shist + kLargeBins;          // [kLargeMaxChunk / 32] bit per chunk-local token
+    uint32_t* keys = resv + kLargeMaxChunk / 32;  // [chunk tokens]
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int seg = blockIdx.x / p.n_chunks, chunk = blockIdx.x - seg * p.n_chunks;
+    int g0, g1, tok0, tok1;
+    chunk_range(p, chunk, g0, g1, tok0, tok1);
+    const int cn = tok1 - tok0, cn_pad = (cn + 31) & ~31;
+    const float* scores = p.scores + (size_t)seg * p.n + tok0;
+    wait_for_prior_kernels();
+
+    for (int i = tid; i < cn_pad; i += nt) keys[i] = i < cn ? score_key(__ldg(scores + i)) : 0u;
+    for (int b = tid; b < kLargeBins; b += nt) shist[b] = 0u;
+    for (int i = tid; i < kLargeMaxChunk / 32; i += nt) resv[i] = 0u;
+    __syncthreads();
+
+    chunk_floor(p, keys, resv, g0, g1, tok0, cn, cn_pad);
     __syncthreads();
 
     uint8_t* flags = p.flags + (size_t)seg * p.n + tok0;

@@ -117,6 +117,56 @@ def test_long_videos(t, h, w, rh, rw, m, frac, kind):
     assert_parity(s.astype(np.float32), t, h, w, rh, rw, m, n // frac)
 
 
+def test_default_chunking_takes_one_launch_of_block_clusters():
+    """Segments up to 16 K tokens (and batches of larger ones) with the library's own chunking: one launch, a
+    cluster of four blocks per segment."""
+    rng = np.random.default_rng(77)
+    specials = np.array([0x80000000, 0x00000000, 0x7F800000, 0xFF800000, 0x00000001, 0x80000001, 0x7FC00000,
+                         0xFFC00000, 0x3F800000, 0xBF800000], dtype=np.uint32).view(np.float32)
+    done = 0
+    for trial in range(200):
+        t = int(rng.integers(1, 7))
+        h = int(rng.integers(4, 90))
+        w = int(rng.integers(4, 90))
+        rh = int(rng.integers(1, 12))
+        rw = int(rng.integers(1, 12))
+        m = int(rng.integers(0, 4))
+        n = t * h * w
+        if n > 16384 or done == 48:
+            continue
+        done += 1
+        n_res = O.reserved_count(t, h, w, rh, rw, m)
+        k = [n_res, n, int(rng.integers(n_res, n + 1))][done % 3] if done % 5 == 0 else int(rng.integers(n_res, n + 1))
+        n_seg = int(rng.integers(1, 4))
+        kind = done % 4
+        if kind == 0:
+            s = rng.random((n_seg, n))
+        elif kind == 1:
+            s = rng.integers(0, 5, (n_seg, n))  # heavy ties: the threshold class spans the blocks
+        elif kind == 2:
+            s = rng.choice(specials, size=(n_seg, n))
+        else:
+            s = np.exp(rng.standard_normal((n_seg, n)) * 8)  # wide exponent range
+        before = civic.launch_count()
+        assert_parity(np.asarray(s, dtype=np.float32), t, h, w, rh, rw, m, k)
+        assert civic.launch_count() - before == (1 if k > 0 else 0), (t, h, w, rh, rw, m, k)
+    assert done == 48
+    # two region rows for a cluster of four blocks: the last two blocks hold nothing
+    s = rng.random((2, 64 * 128)).astype(np.float32)
+    before = civic.launch_count()
+    assert_parity(s, 1, 64, 128, 32, 16, 1, 3000)
+    assert civic.launch_count() - before == 1
+    # all scores equal: every kept token beyond the floor is a tie split by index across the blocks
+    ones = np.ones((2, 3 * 60 * 70), dtype=np.float32)
+    for m, k in [(0, 1), (1, 5000), (2, 12600)]:
+        assert_parity(ones, 3, 60, 70, 6, 7, m, k)
+    # a batch of mid-sized segments (more tokens than one wave of small blocks): still one launch
+    s = np.floor(rng.random((8, 16 * 56 * 56)) * 256).astype(np.float32)
+    before = civic.launch_count()
+    assert_parity(s, 16, 56, 56, 4, 4, 1, 16 * 56 * 56 // 3)
+    assert civic.launch_count() - before == 1
+
+
 def test_agrees_with_the_one_block_kernel_at_its_largest_segment():
     n_max = civic.select_max_tokens()
     h = 64
