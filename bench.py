@@ -736,6 +736,102 @@ def run_kv_attention(args):
     print(json.dumps(line), flush=True)
 
 
+def run_long_select(args):
+    """`--workload longsel_*`: one step = one civic_select_large call on segments beyond one thread
+    block; timed with the library's own chunking (which may take the one-launch cluster path) and
+    with an explicit chunk of the same size (always the five launches), as a plain loop and as
+    replays of a CUDA graph of one call."""
+    import numpy as np
+    import torch
+
+    from paper_2605_28115_b200 import build as civic_build
+    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import workloads as W
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1 or args.gpus != 1:
+        raise SystemExit("this workload is benchmarked on one GPU")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    dev = "cuda:0"
+    civic_build.build()
+    civic.load()
+    wl = W.LONG_BY_NAME[args.workload]
+    scores_host = W.scores(wl)
+    scores = torch.from_numpy(scores_host).to(dev)
+    desc = civic.SelectDesc(wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+    out = torch.empty((wl.n_seg, wl.k), dtype=torch.int32, device=dev)
+    row = min(wl.region_h, wl.h) * wl.w
+    explicit = max(2048, min(16384, (wl.n_seg * wl.n + 147) // 148))
+    explicit = max(row, explicit // row * row)  # the default's size, rounded to whole region rows
+    warm = max(args.warmup, 3)
+
+    def timed(chunk):
+        ws = torch.empty(civic.select_workspace_bytes(desc, wl.n_seg, chunk), dtype=torch.uint8, device=dev)
+        call = lambda: civic.civic_select_large(scores, desc, keep_idx=out, workspace=ws, chunk_tokens=chunk)
+        before = civic.launch_count()
+        call()
+        per_call = civic.launch_count() - before
+        for _ in range(warm):
+            call()
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for _ in range(args.steps):
+            call()
+        end.record()
+        torch.cuda.synchronize()
+        plain_us = start.elapsed_time(end) / args.steps * 1e3
+        graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                call()
+        for _ in range(warm):
+            graph.replay()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(args.steps):
+            graph.replay()
+        end.record()
+        torch.cuda.synchronize()
+        return {"launches_per_call": per_call, "plain_loop_us": plain_us,
+                "graph_replay_us": start.elapsed_time(end) / args.steps * 1e3}
+
+    sampler = ClockSampler(0)
+    launches0 = civic.launch_count()
+    sampler.start()
+    own, five = timed(0), timed(explicit)
+    clocks = sampler.stop()
+    launches = civic.launch_count() - launches0
+    cpu = None
+    if not args.no_cpu_baseline:  # the oracle as it stands, timed on the host cores; its result is compared too
+        import oracle
+
+        threads = oracle.default.set_threads(0)
+        times = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            want = oracle.default.select(scores_host, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+            times.append(time.perf_counter() - t0)
+        med = statistics.median(times)
+        cpu = {"value": wl.n_seg * wl.n / med / 1e6, "unit": "Mtokens/s", "cores": threads, "kind": "oracle",
+               "sample": f"the whole batch, median of 3 runs, {med * 1e3:.1f} ms",
+               "gpu_result_equals_oracle": bool(np.array_equal(out.cpu().numpy(), want))}
+    us = own["graph_replay_us"]
+    line = {"metric": "long_segment_selection_Mtokens_per_s", "value": wl.n_seg * wl.n / us, "unit": "Mtokens/s",
+            "n_gpus": 1, "steps": args.steps, "warmup": warm, "ms_per_step": us * 1e-3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {"workload": wl.name, "n_seg": wl.n_seg, "grid_thw": [wl.t, wl.h, wl.w],
+                       "region_hw": [wl.region_h, wl.region_w], "floor_per_region": wl.floor_m, "k": wl.k,
+                       "scores": wl.score_kind, "l2": "scores fit in L2 and are not flushed: a latency figure",
+                       "parallelism": "single"},
+            "own_chunking": own, "five_launches": dict(five, chunk_tokens=explicit),
+            "gpu_launches": launches, "clocks": clocks,
+            "roofline": {"bound": "latency", "kernel": "civic_select_large", "achieved": us, "peak": None, "unit": "us",
+                         "frac": None, "traffic": None},
+            "e2e": None, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+
+
 def run_aggregate_reference(args):
     """The fp64 numpy oracle of Eq. 8 on this machine's host cores; each step is ONE image of the
     workload (a bounded sample), at most 10 steps."""
@@ -828,7 +924,11 @@ def run_reference(args):
 
 if __name__ == "__main__":
     a = parse_args()
-    if a.workload.startswith("kvattn_"):
+    if a.workload.startswith("longsel_"):
+        if a.impl == "reference":
+            raise SystemExit("the reference arm covers the select + compact + KV and the aggregation workloads")
+        run_long_select(a)
+    elif a.workload.startswith("kvattn_"):
         if a.impl == "reference":
             raise SystemExit("the reference arm covers the select + compact + KV and the aggregation workloads")
         run_kv_attention(a)

@@ -144,6 +144,14 @@ C5_QUARTER = C5_HALF.replace(name="c5_hires_keep_1_4", k=784)
 ALL = (C1, C2, C3, C4, C5_HALF, C5_THIRD, C5_QUARTER)
 BY_NAME = {wl.name: wl for wl in ALL}
 
+# Selection alone on segments beyond one thread block (long videos, Section 5 of the paper):
+# no payload, K = n / 3.  A 128-frame clip at 56 x 56 tokens per two frames, a batch of eight
+# 32-frame clips, and a batch of four 8-frame clips.
+LONG_VIDEO = Workload("longsel_video_128f", 6, 1, 64, 56, 56, 4, 4, 1, 64 * 56 * 56 // 3, "quant256")
+LONG_BATCH8 = Workload("longsel_batch8_32f", 7, 8, 16, 56, 56, 4, 4, 1, 16 * 56 * 56 // 3, "lognormal")
+LONG_BATCH4 = Workload("longsel_batch4_8f", 8, 4, 4, 56, 56, 4, 4, 1, 4 * 56 * 56 // 3, "uniform")
+LONG_BY_NAME = {wl.name: wl for wl in (LONG_VIDEO, LONG_BATCH8, LONG_BATCH4)}
+
 
 def scores(wl: Workload, seg: Optional[int] = None) -> np.ndarray:
     """Importance scores, fp32.  [n_seg, n], or [n] for one segment."""
