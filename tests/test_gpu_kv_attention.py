@@ -84,7 +84,9 @@ def check(q, k, v, r, heads):
     (1, 1024, 16, 64, 256),  # Qwen3-VL-2B-shaped vision layer: 1024 compact tokens, 16 heads of 64, 256 anchors
     (10, 700, 16, 64, 64),   # more (head, image) pairs than SMs: blocks walk three query tiles, the last ragged
     (5, 1100, 32, 64, 128),  # nine query tiles in three blocks per pair
-    (20, 520, 8, 128, 128),  # five tiles per block with 128-wide heads: both TMEM buffers and Q slots reused twice
+    (20, 520, 8, 128, 128),  # five tiles per block with 128-wide heads: both Q slots reused twice
+    (3, 300, 50, 128, 256),  # the largest shared-memory footprint (one block per SM), three tiles per block
+    (2, 150, 80, 64, 192),   # 192 anchors (P and O share 256 TMEM columns with S), two tiles per block
 ])
 def test_against_oracle(n_img, m_e, heads, d, s):
     q, k, v, r = inputs(n_img, m_e, heads, d, s, seed=m_e + s)
