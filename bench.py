@@ -364,9 +364,9 @@ class HostState:
         return all(torch.equal(d.cpu(), h) for d, h in pairs)
 
 
-def cpu_baseline(st: DeviceState, budget_s: float = 20.0):
+def cpu_baseline(st: DeviceState, limit_s: float = 20.0):
     """The oracle as it stands, timed on this machine's host cores on the same inputs (copied
-    from the device): a few whole passes, bounded by `budget_s`."""
+    from the device): a few whole passes, bounded by `limit_s`."""
     import numpy as np
     import torch
 
@@ -385,7 +385,7 @@ def cpu_baseline(st: DeviceState, budget_s: float = 20.0):
     nbytes = step_bytes(sample)["total"]
     times = []
     t_begin = time.perf_counter()
-    while len(times) < 3 or (time.perf_counter() - t_begin < budget_s / 2 and len(times) < 15):
+    while len(times) < 3 or (time.perf_counter() - t_begin < limit_s / 2 and len(times) < 15):
         t0 = time.perf_counter()
         keep = o.select(st.scores_host, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
         o.compact(hidden, st.pos_host, keep)
