@@ -107,6 +107,29 @@ def test_select_all_equal_and_degenerate_regions():
     assert_select_parity(np.zeros((3, 1), np.float32), 1, 1, 1, 1, 1, 1, 1)
 
 
+def test_select_threshold_decided_by_the_leading_digits():
+    """Keys built so that the radix search can stop after its first, second or third digit (the threshold bin
+    is wanted whole), with several different keys inside the bins that are taken whole."""
+    rng = np.random.default_rng(31)
+    n = 24 * 24
+    for low_bits in (24, 16, 8, 0):  # key bits below the digit that decides
+        # a few well separated groups in the leading bits, arbitrary bits below
+        lead = rng.integers(1, 40, size=(2, n)).astype(np.uint32)
+        low = rng.integers(0, 1 << low_bits, size=(2, n)).astype(np.uint32) if low_bits else np.zeros((2, n), np.uint32)
+        bits = (np.uint32(0x30000000) + (lead << np.uint32(low_bits)) + low).astype(np.uint32)
+        s = bits.view(np.float32)
+        assert np.all(np.isfinite(s))
+        counts = np.bincount(lead[0], minlength=40)
+        above = int(counts[20:].sum())  # exactly the tokens of the groups 20..39 of segment 0: whole bins
+        for m, k in [(0, max(above, 1)), (0, 7), (1, 36 + 50), (2, 300), (0, n - 1)]:
+            assert_select_parity(s, 1, 24, 24, 4, 4, m, k)
+    # powers of four: every token alone in its leading-digit bin, any K stops after the first digit
+    p4 = (4.0 ** -np.arange(60, dtype=np.float64)).astype(np.float32)[None, :]
+    for k in (1, 17, 59, 60):
+        assert_select_parity(np.ascontiguousarray(p4[:, ::-1]), 1, 6, 10, 2, 5, 0, k)
+        assert_select_parity(p4, 1, 6, 10, 2, 5, 1, max(k, 6))
+
+
 def test_select_special_values():
     specials = np.array([0x80000000, 0x00000000, 0x7F800000, 0xFF800000, 0x00000001, 0x80000001,
                          0x7FC00000, 0xFFC00000, 0x7F800001, 0xFF800001, 0x7FFFFFFF, 0xFFFFFFFF,
