@@ -17,8 +17,9 @@ __device__ __forceinline__ void wait_for_prior_kernels()
 }
 
 // Lets the next kernel of the stream begin its launch now (it still waits for this whole grid
-// to complete before it touches memory).  Only the small grids call it: early blocks of a
-// successor would take resident-block slots away from a bandwidth-bound grid.
+// to complete before it touches memory).  Only the small grids (selection, index kernels) call
+// it: early blocks of a successor would take resident-block slots away from a bandwidth-bound
+// grid, and measured slower next to the persistent tensor-core kernels too.
 __device__ __forceinline__ void release_next_kernel()
 {
     asm volatile("griddepcontrol.launch_dependents;");

@@ -61,6 +61,7 @@ __global__ void __launch_bounds__(kClusterThreads) select_cluster_kernel(const _
     chunk_range(p, chunk, g0, g1, tok0, tok1);
     const int cn = tok1 - tok0, cn_pad = (cn + 31) & ~31;
     const float* scores = p.scores + (size_t)seg * p.n + tok0;
+    release_next_kernel();
     wait_for_prior_kernels();
 
     for (int i = tid; i < cn_pad; i += nt) keys[i] = i < cn ? score_key(__ldg(scores + i)) : 0u;

@@ -174,6 +174,7 @@ __global__ void __launch_bounds__(kLargeThreads) large_floor_kernel(const __grid
     chunk_range(p, chunk, g0, g1, tok0, tok1);
     const int cn = tok1 - tok0, cn_pad = (cn + 31) & ~31;
     const float* scores = p.scores + (size_t)seg * p.n + tok0;
+    release_next_kernel();
     wait_for_prior_kernels();
 
     for (int i = tid; i < cn_pad; i += nt) keys[i] = i < cn ? score_key(__ldg(scores + i)) : 0u;
@@ -204,6 +205,7 @@ __global__ void __launch_bounds__(kLargeThreads) large_hist_kernel(const __grid_
     const int seg = blockIdx.x / p.n_chunks, chunk = blockIdx.x - seg * p.n_chunks;
     int g0, g1, tok0, tok1;
     chunk_range(p, chunk, g0, g1, tok0, tok1);
+    release_next_kernel();
     wait_for_prior_kernels();
     if (p.k_fill <= 0) return;
     uint32_t* sel = p.sel + (size_t)seg * kLargeSelWords;
@@ -244,6 +246,7 @@ __global__ void __launch_bounds__(kLargeThreads) large_count_kernel(const __grid
     const int seg = blockIdx.x / p.n_chunks, chunk = blockIdx.x - seg * p.n_chunks;
     int g0, g1, tok0, tok1;
     chunk_range(p, chunk, g0, g1, tok0, tok1);
+    release_next_kernel();
     wait_for_prior_kernels();
     uint32_t* sel = p.sel + (size_t)seg * kLargeSelWords;
     uint32_t T = 0xFFFFFFFFu, need_eq = 0;
@@ -280,6 +283,7 @@ __global__ void __launch_bounds__(kLargeThreads) large_place_kernel(const __grid
     const int seg = blockIdx.x / p.n_chunks, chunk = blockIdx.x - seg * p.n_chunks;
     int g0, g1, tok0, tok1;
     chunk_range(p, chunk, g0, g1, tok0, tok1);
+    release_next_kernel();
     wait_for_prior_kernels();
     const uint32_t* sel = p.sel + (size_t)seg * kLargeSelWords;
     const uint32_t T = sel[4], need_eq = sel[5];
