@@ -14,12 +14,15 @@
  *     overlap inputs (checked where both extents are known; overlap -> CIVIC_ERR_INVALID_ARG).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
  *     enqueued on it and the call returns without synchronising.  The library allocates no
- *     device memory and keeps no state between calls.
+ *     device memory.  What it keeps between calls is named at the entry concerned: a launch
+ *     counter, the programmatic-launch switch, and the contents of the scratch array built
+ *     in for civic_select_large_static.
  *   - Arguments are validated on the host BEFORE anything is launched; on any status other
  *     than CIVIC_OK nothing was enqueued.  CIVIC_ERR_CUDA wraps a failed launch or attribute
  *     call (the CUDA error string is available from civic_last_cuda_error()).
- *   - There are no data-dependent errors: whether the retention floor fits into the budget
- *     depends on shapes only.  The validity of index arrays passed to the compaction calls
+ *   - No returned status depends on the data: whether the retention floor fits into the
+ *     budget depends on shapes only.  (The two tensor-core calls also write a device status
+ *     word, to be read after synchronising: see there.)  The validity of index arrays passed to the compaction calls
  *     (in range, one row per output row) is the caller's contract, as they normally come
  *     straight from civic_select / civic_seq_indices.
  *   - A token grid is (t, h, w), token index i = (tt*h + hh)*w + ww (row-major), n = t*h*w.
