@@ -87,6 +87,9 @@ def check(q, k, v, r, heads):
     (20, 520, 8, 128, 128),  # five tiles per block with 128-wide heads: both Q slots reused twice
     (3, 300, 50, 128, 256),  # the largest shared-memory footprint (one block per SM), three tiles per block
     (2, 150, 80, 64, 192),   # 192 anchors (P and O share 256 TMEM columns with S), two tiles per block
+    (1, 5, 2, 64, 64),       # fewer queries than one warp's 32 rows: one partly filled store box, three skipped
+    (2, 33, 3, 128, 128),    # one row into the second warp's box
+    (1, 129, 1, 64, 256),    # one row into the second query tile
 ])
 def test_against_oracle(n_img, m_e, heads, d, s):
     q, k, v, r = inputs(n_img, m_e, heads, d, s, seed=m_e + s)
