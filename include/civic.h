@@ -15,16 +15,27 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
  *     enqueued on it and the call returns without synchronising.  The library allocates no
  *     device memory.  What it keeps between calls is named at the entry concerned: a launch
- *     counter, the programmatic-launch switch, and the contents of the scratch array built
- *     in for civic_select_large_static.
- *   - Arguments are validated on the host BEFORE anything is launched; on any status other
- *     than CIVIC_OK nothing was enqueued.  CIVIC_ERR_CUDA wraps a failed launch or attribute
- *     call (the CUDA error string is available from civic_last_cuda_error()).
+ *     counter, the programmatic-launch switch, the calling thread's index-check record
+ *     (civic_set_index_check), per-device caches of device properties, and the contents of
+ *     the scratch array built in for civic_select_large_static.
+ *   - Arguments are validated on the host BEFORE anything is launched: every status other
+ *     than CIVIC_OK and CIVIC_ERR_CUDA means that nothing was enqueued.  CIVIC_ERR_CUDA wraps
+ *     a failed CUDA runtime call (its text is available from civic_last_cuda_error()); some
+ *     entries enqueue several launches (civic_select_large, the two tensor-core calls, K/V
+ *     calls over more than 80 layers, ragged batches over more than 64 segments), so after
+ *     CIVIC_ERR_CUDA earlier launches of the same call may already be enqueued and its outputs
+ *     and scratch are undefined.
+ *   - Threads: every entry may be called from several host threads at once, on the same or
+ *     different devices and streams, as long as concurrent calls do not share output or
+ *     scratch buffers.  Process-wide switches (civic_set_programmatic_launch) are atomic;
+ *     civic_set_index_check and civic_last_cuda_error are per calling thread.
  *   - No returned status depends on the data: whether the retention floor fits into the
- *     budget depends on shapes only.  (The two tensor-core calls also write a device status
- *     word, to be read after synchronising: see there.)  The validity of index arrays passed to the compaction calls
- *     (in range, one row per output row) is the caller's contract, as they normally come
- *     straight from civic_select / civic_seq_indices.
+ *     budget depends on shapes only.  What the kernels find on the device is reported through
+ *     device words the caller reads after synchronising: the status word of the two
+ *     tensor-core calls, and the fault record of civic_set_index_check /
+ *     civic_validate_indices.  Without that check the validity of index arrays passed to the
+ *     compaction calls (in range, one row per output row) is the caller's contract, as they
+ *     normally come straight from civic_select / civic_seq_indices.
  *   - A token grid is (t, h, w), token index i = (tt*h + hh)*w + ww (row-major), n = t*h*w.
  */
 #ifndef CIVIC_H_
@@ -392,6 +403,67 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
 /* Scratch bytes civic_kv_compressed_attention needs; 0 if the shape is invalid or unsupported. */
 size_t civic_kv_compressed_attention_workspace_bytes(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
                                                      int32_t s);
+
+/*
+ * Device-side validation of index arrays.
+ *
+ * Paper: the compact rows are "indexed by compact visual segments" with inherited positions
+ * (Section 3.5); the paper has no counterpart to checking those indices, this is the library's
+ * own safety net.  The compaction calls (civic_compact, civic_compact_kv, _kv_heads, _kv_paged,
+ * civic_merge_embeddings, civic_compact_pos_planes) read `keep_idx` / `seq_idx` / `block_table`
+ * on the device, so a wrong value cannot be caught by the host-side validation.  With a fault
+ * record set, they run kernels that test every index they use: a row whose source index lies
+ * outside [0, seq_len) (outside [0, n_vis) for the merge), or whose page lies outside
+ * [0, n_pages), is NEITHER READ NOR WRITTEN, and the fault is recorded.  Nothing traps; all other
+ * rows are moved as usual.
+ *
+ * fault record  dev int32[4] = {code, row, position, value}: code is a civic_index_fault_t, row the
+ *               sequence / segment (index row) concerned, position the column of the index array
+ *               (the page slot of the block table for CIVIC_INDEX_BAD_PAGE), value the offending
+ *               entry.  The first kernel thread to meet a fault claims the record; later faults
+ *               leave it alone, so it names ONE offending entry (which one is unspecified when
+ *               there are several).  The library never clears it: zero it (cudaMemsetAsync)
+ *               before the calls to be checked and read it after synchronising.
+ *
+ * civic_set_index_check   sets (NULL: clears) the record used by the CALLING THREAD's later
+ *               compaction calls; returns CIVIC_ERR_ALIGNMENT for a pointer that is not 4-byte
+ *               aligned.  Off by default; when off the calls launch the unchecked kernels and pay
+ *               nothing.  The record must stay valid until those calls have completed.
+ * civic_validate_indices  checks an index array [n_rows, row_len] on its own: every value in
+ *               [0, limit) and, with require_ascending != 0, every row strictly ascending
+ *               (CIVIC_INDEX_NOT_ASCENDING names the first position that is not larger than its
+ *               predecessor).  One small launch; n_rows * row_len == 0 enqueues nothing.
+ */
+typedef enum {
+    CIVIC_INDEX_OK = 0,
+    CIVIC_INDEX_OUT_OF_RANGE = 1,
+    CIVIC_INDEX_NOT_ASCENDING = 2,
+    CIVIC_INDEX_BAD_PAGE = 3
+} civic_index_fault_t;
+
+civic_status_t civic_set_index_check(int32_t* fault_record);
+
+civic_status_t civic_validate_indices(const int32_t* idx, int32_t n_rows, int32_t row_len, int32_t limit,
+                                      int32_t require_ascending, int32_t* fault_record, void* stream);
+
+/*
+ * civic_selftest_bounded_wait -- shows that a wait inside the tensor-core kernels that never gets
+ * its signal ends with a status instead of a hang.
+ *
+ * Paper: no counterpart.  The kernels of civic_anchor_aggregate and
+ * civic_kv_compressed_attention wait on shared-memory barriers through one bounded wait routine
+ * (limit about one second of SM cycles); when the limit runs out the thread records a code in the
+ * call's device status word and raises a flag that makes the block's other waits return.  This
+ * entry runs that same routine in a one-block kernel on a barrier that nothing ever signals, with
+ * no copy and no tensor-core operation in flight: one thread waits with `limit_cycles` and times
+ * out, a second thread waits with the ordinary limit and must leave through the flag.
+ *
+ * limit_cycles  1 .. 2^24 SM cycles (a few milliseconds at most)
+ * record        dev int32[2], cleared and then written: [0] = 1 (the code a starved operand wait
+ *               reports), [1] = 1 if the second waiter left because of the flag
+ * One 8-byte memset and one launch; the context stays usable.
+ */
+civic_status_t civic_selftest_bounded_wait(uint64_t limit_cycles, int32_t* record, void* stream);
 
 /* Static, human-readable name of a status. */
 const char* civic_status_string(civic_status_t status);

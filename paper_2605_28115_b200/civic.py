@@ -31,7 +31,10 @@ EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "c
            "civic_select_ragged", "civic_floor_from_ratio",
            "civic_select_large_static", "civic_select_static_scratch_bytes",
            "civic_anchor_aggregate", "civic_anchor_aggregate_workspace_bytes",
-           "civic_kv_compressed_attention", "civic_kv_compressed_attention_workspace_bytes")
+           "civic_kv_compressed_attention", "civic_kv_compressed_attention_workspace_bytes",
+           "civic_set_index_check", "civic_validate_indices", "civic_selftest_bounded_wait")
+
+INDEX_FAULTS = ("CIVIC_INDEX_OK", "CIVIC_INDEX_OUT_OF_RANGE", "CIVIC_INDEX_NOT_ASCENDING", "CIVIC_INDEX_BAD_PAGE")
 
 
 class CivicError(RuntimeError):
@@ -114,6 +117,12 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_kv_compressed_attention.restype = ctypes.c_int
     lib.civic_kv_compressed_attention_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.civic_kv_compressed_attention_workspace_bytes.restype = sz
+    lib.civic_set_index_check.argtypes = [vp]
+    lib.civic_set_index_check.restype = ctypes.c_int
+    lib.civic_validate_indices.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+    lib.civic_validate_indices.restype = ctypes.c_int
+    lib.civic_selftest_bounded_wait.argtypes = [ctypes.c_uint64, vp, vp]
+    lib.civic_selftest_bounded_wait.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -651,3 +660,46 @@ def civic_kv_compressed_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Ten
     with _on_device(dev):
         _check(load().civic_kv_compressed_attention(*args, _stream_ptr(stream)), "civic_kv_compressed_attention")
     return out, device_status
+
+
+class index_check:
+    """Context manager: inside it this thread's compaction calls validate their index arrays on the
+    device and record the first fault in `record` (int32 [4] on the device: code, row, position,
+    value; see INDEX_FAULTS).  The record is not cleared here."""
+
+    def __init__(self, record: torch.Tensor):
+        if record.numel() < 4:
+            raise ValueError("the fault record must hold 4 int32")
+        self.ptr = _dev_ptr(record, "record", torch.int32)
+        self.keepalive = record
+
+    def __enter__(self):
+        _check(load().civic_set_index_check(self.ptr), "civic_set_index_check")
+        return self
+
+    def __exit__(self, *exc):
+        load().civic_set_index_check(None)
+
+
+def civic_validate_indices(idx: torch.Tensor, limit: int, record: torch.Tensor, require_ascending: bool = True,
+                           stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """idx int32 [n_rows, row_len]: every value in [0, limit), rows strictly ascending if asked;
+    the first fault found goes to `record` (int32 [4], sticky)."""
+    if idx.dim() != 2 or record.numel() < 4:
+        raise ValueError("idx must be [n_rows, row_len] and the record hold 4 int32")
+    args = (_dev_ptr(idx, "idx", torch.int32), idx.shape[0], idx.shape[1], limit, 1 if require_ascending else 0,
+            _dev_ptr(record, "record", torch.int32))
+    with _on_device(_device_of(idx, record)):
+        _check(load().civic_validate_indices(*args, _stream_ptr(stream)), "civic_validate_indices")
+    return record
+
+
+def civic_selftest_bounded_wait(limit_cycles: int, record: torch.Tensor,
+                                stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Runs the kernels' bounded wait on a barrier nobody signals; record int32 [2] -> (time-out code, 1)."""
+    if record.numel() < 2:
+        raise ValueError("the record must hold 2 int32")
+    with _on_device(_device_of(record)):
+        _check(load().civic_selftest_bounded_wait(limit_cycles, _dev_ptr(record, "record", torch.int32),
+                                                  _stream_ptr(stream)), "civic_selftest_bounded_wait")
+    return record

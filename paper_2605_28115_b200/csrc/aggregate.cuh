@@ -71,15 +71,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false when the block has been told to stop (*abort != 0) or the limit
-// ran out, in which case it also raises *abort and records `code` in the kernel's error word.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* error, int code)
+// (SM cycles) ran out, in which case it also raises *abort and records `code` in the kernel's
+// error word.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int* error, int code,
+                                          unsigned long long limit = kWaitLimitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
-        if ((unsigned long long)(clock64() - t0) > kWaitLimitCycles) {
+        if ((unsigned long long)(clock64() - t0) > limit) {
             *abort = 1;
             atomicCAS(error, 0, code);
             return false;
@@ -873,6 +875,31 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
         tc_fence_after_sync();
         if (kPair) tmem_dealloc_pair(tmem_base, 512);
         else tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// Self-test of the bounded wait: one block, one mbarrier that nobody ever arrives on, no copy and
+// no MMA in flight.  Thread 0 waits with the caller's (short) limit, runs into it and raises the
+// block's stop flag; thread 32 waits on the same barrier with the library's ordinary limit and must
+// leave through the stop flag.  record[0] = the time-out code, record[1] = 1 if the second waiter
+// left because of the flag.
+__global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned long long limit, int* record)
+{
+    __shared__ uint64_t bar;
+    __shared__ int stop;
+    wait_for_prior_kernels();
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        stop = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    volatile int* abort = &stop;
+    if (threadIdx.x == 0) {
+        mbar_wait(&bar, 0, abort, record, kAggTimeoutFull, limit);
+    } else if (threadIdx.x == 32) {
+        const bool ok = mbar_wait(&bar, 0, abort, record, kAggTimeoutAcc);
+        if (!ok && *abort) record[1] = 1;
     }
 }
 

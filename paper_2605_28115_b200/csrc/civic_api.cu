@@ -24,9 +24,14 @@ std::atomic<int> g_programmatic{1};
 bool programmatic() { return g_programmatic.load(std::memory_order_relaxed) != 0; }
 thread_local char g_cuda_error[256] = "";
 
+// Fault record the calling thread's compaction calls validate their index arrays into (device
+// int32[4]); NULL = the unchecked kernels.
+thread_local int32_t* g_index_check = nullptr;
+
 civic_status_t cuda_fail(cudaError_t e, const char* what)
 {
     snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    (void)cudaGetLastError();  // the runtime's own "last error" is not left behind for the caller's next call
     return CIVIC_ERR_CUDA;
 }
 
@@ -74,9 +79,41 @@ int sm_count()
     return v;
 }
 
+// Index of the current device in the per-device caches below, or -1 (then nothing is cached).
+int device_slot()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    return dev;
+}
+
+// The largest dynamic shared memory a kernel may ask for is a per-device function attribute.
+// It is raised ONCE per device to the most the kernel can ever need, not per call to that
+// call's size: two host threads launching different shapes would otherwise undo each other's
+// setting between cudaFuncSetAttribute and the launch.
+template <class Kernel>
+civic_status_t allow_dynamic_smem(Kernel kernel, size_t max_bytes, std::atomic<int>* done /*[64]*/)
+{
+    const int dev = device_slot();
+    if (dev >= 0 && done[dev].load(std::memory_order_acquire)) return CIVIC_OK;
+    CIVIC_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_bytes));
+    if (dev >= 0) done[dev].store(1, std::memory_order_release);
+    return CIVIC_OK;
+}
+
 // Launch the row gather for up to kMaxGatherTensors tensors sharing one index array.
+template <int MODE, bool CHECK>
+civic_status_t launch_gather_checked(civic::GatherParams& p, cudaStream_t stream);
+
 template <int MODE>
 civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
+{
+    p.check = g_index_check;
+    return p.check ? launch_gather_checked<MODE, true>(p, stream) : launch_gather_checked<MODE, false>(p, stream);
+}
+
+template <int MODE, bool CHECK>
+civic_status_t launch_gather_checked(civic::GatherParams& p, cudaStream_t stream)
 {
     const long long total_rows = (long long)p.n_tensors * p.n_planes * p.s_out;
     const bool has_pos = p.pos_src != nullptr;
@@ -102,11 +139,11 @@ civic_status_t launch_gather(civic::GatherParams& p, cudaStream_t stream)
     const bool pdl = programmatic();
     cudaError_t e;
     if (vec16)
-        e = small ? civic::launch(pdl, civic::gather_rows_kernel<uint4, 4, MODE, true>, grid, threads, 0, stream, p)
-                  : civic::launch(pdl, civic::gather_rows_kernel<uint4, 4, MODE, false>, grid, threads, 0, stream, p);
+        e = small ? civic::launch(pdl, civic::gather_rows_kernel<uint4, 4, MODE, true, CHECK>, grid, threads, 0, stream, p)
+                  : civic::launch(pdl, civic::gather_rows_kernel<uint4, 4, MODE, false, CHECK>, grid, threads, 0, stream, p);
     else
-        e = small ? civic::launch(pdl, civic::gather_rows_kernel<uint32_t, 8, MODE, true>, grid, threads, 0, stream, p)
-                  : civic::launch(pdl, civic::gather_rows_kernel<uint32_t, 8, MODE, false>, grid, threads, 0, stream, p);
+        e = small ? civic::launch(pdl, civic::gather_rows_kernel<uint32_t, 8, MODE, true, CHECK>, grid, threads, 0, stream, p)
+                  : civic::launch(pdl, civic::gather_rows_kernel<uint32_t, 8, MODE, false, CHECK>, grid, threads, 0, stream, p);
     CIVIC_CUDA_TRY(e);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CIVIC_OK;
@@ -232,8 +269,10 @@ civic_status_t launch_cluster_select(const float* scores, int32_t n_seg, const c
     p.m = d.floor_per_region; p.k = d.k; p.k_fill = k_fill;
     p.n_rh = pl.n_rh; p.rows_per_chunk = (int32_t)rows_per_chunk; p.n_chunks = blocks;
     const size_t smem = civic::select_cluster_smem_bytes((int)chunk_tokens);
-    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)smem));
+    static std::atomic<int> smem_allowed[64];
+    const civic_status_t as = allow_dynamic_smem(civic::select_cluster_kernel,
+                                                 civic::select_cluster_smem_bytes(civic::kClusterMaxChunk), smem_allowed);
+    if (as != CIVIC_OK) return as;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(n_seg * blocks));
     cfg.blockDim = dim3(civic::kClusterThreads);
@@ -252,9 +291,21 @@ civic_status_t launch_cluster_select(const float* scores, int32_t n_seg, const c
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    int resident = 0;  // clusters of this shape the device can hold at once
-    CIVIC_CUDA_TRY(cudaOccupancyMaxActiveClusters(&resident, civic::select_cluster_kernel, &cfg));
-    if (resident < 1) return CIVIC_ERR_UNSUPPORTED;
+    // Can the device hold a cluster of this kernel at all?  Asked once per device, for the largest
+    // block the kernel is ever launched with (a smaller one then fits too): 1 = yes, 2 = no.
+    static std::atomic<int> placeable[64];
+    const int dev = device_slot();
+    int fits = dev >= 0 ? placeable[dev].load(std::memory_order_relaxed) : 0;
+    if (fits == 0) {
+        cudaLaunchConfig_t probe = cfg;
+        probe.gridDim = dim3((unsigned)blocks);
+        probe.dynamicSmemBytes = civic::select_cluster_smem_bytes(civic::kClusterMaxChunk);
+        int resident = 0;
+        CIVIC_CUDA_TRY(cudaOccupancyMaxActiveClusters(&resident, civic::select_cluster_kernel, &probe));
+        fits = resident >= 1 ? 1 : 2;
+        if (dev >= 0) placeable[dev].store(fits, std::memory_order_relaxed);
+    }
+    if (fits != 1) return CIVIC_ERR_UNSUPPORTED;
     CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::select_cluster_kernel, p));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CIVIC_OK;
@@ -285,9 +336,12 @@ civic_status_t launch_large(const float* scores, int32_t n_seg, const civic_sele
     CIVIC_CUDA_TRY(cudaMemsetAsync(ws + pl.hist_off, 0,
                                    (size_t)n_seg * (3 * civic::kLargeBins + civic::kLargeSelWords) * 4, stream));
     const size_t smem = (size_t)(civic::kLargeBins + civic::kLargeMaxChunk / 32 + ((pl.chunk_tokens + 31) & ~31)) * 4;
-    if (smem > 48 * 1024)
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::large_floor_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        static std::atomic<int> smem_allowed[64];
+        const size_t most = (size_t)(civic::kLargeBins + civic::kLargeMaxChunk / 32 + civic::kLargeMaxChunk) * 4;
+        const civic_status_t as = allow_dynamic_smem(civic::large_floor_kernel, most, smem_allowed);
+        if (as != CIVIC_OK) return as;
+    }
     const unsigned grid = (unsigned)(n_seg * pl.n_chunks), threads = civic::kLargeThreads;
     const bool pdl = programmatic();
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::large_floor_kernel, grid, threads, smem, stream, p));
@@ -333,9 +387,12 @@ civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_selec
     p.vis_start = vis_start;
 
     const size_t smem = civic::select_smem_bytes(p.shape.n);
-    if (smem > 48 * 1024)
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        static std::atomic<int> smem_allowed[64];
+        const civic_status_t as = allow_dynamic_smem(civic::select_kernel,
+                                                     civic::select_smem_bytes(civic_select_max_tokens()), smem_allowed);
+        if (as != CIVIC_OK) return as;
+    }
     const int threads = select_threads(p.shape.n);
     CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::select_kernel, (unsigned)n_seg, (unsigned)threads,
                                  smem, (cudaStream_t)stream, p));
@@ -444,8 +501,11 @@ civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, c
                            const typename Op::Params& params, int32_t total_tiles, cudaStream_t stream)
 {
     const size_t smem = sizeof(typename Op::Smem) + 1024;
-    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::aggregate_gemm_kernel<Op>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        static std::atomic<int> smem_allowed[64];
+        const civic_status_t as = allow_dynamic_smem(civic::aggregate_gemm_kernel<Op>, smem, smem_allowed);
+        if (as != CIVIC_OK) return as;
+    }
     // persistent: one block per SM, or one pair of blocks (a cluster of two) per two SMs
     const int workers_max = sm_count() / Op::kCtas;
     const int workers = total_tiles < workers_max ? total_tiles : workers_max;
@@ -804,6 +864,50 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
         if ((ms = make_map(enc, &map_vc, vc, 3, dims, str, 64)) != CIVIC_OK) return ms;
     }
 
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
+    const int32_t q_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
+    CUtensorMap map_o;  // boxes of 32 rows x 64 features: one softmax warp's share of a tile
+    {
+        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
+        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32)) != CIVIC_OK) return ms;
+    }
+    civic::AttnParams ap;
+    ap.error = device_status; ap.m_e = m_e; ap.d = head_dim; ap.s = s;
+    ap.scale_log2e = scale_log2e;
+    // Once per device: the kernel may use all of an SM's memory as shared memory (so that two blocks
+    // of 113 KB can be resident), and the figures that decide how many blocks fit on an SM
+    // together.  (The runtime's occupancy query answers 1 for this kernel whatever its shared
+    // memory, while two blocks were measured running side by side on the SMs.)
+    struct AttnDevice { std::atomic<int> ready; int smem_per_sm, reserved, regs_per_sm, regs_per_thread; };
+    static AttnDevice attn_dev[64];
+    AttnDevice local_info = {};
+    const int dev = device_slot();
+    AttnDevice& info = dev >= 0 ? attn_dev[dev] : local_info;
+    if (!info.ready.load(std::memory_order_acquire)) {
+        int device = 0;
+        CIVIC_CUDA_TRY(cudaGetDevice(&device));
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kMaxDynamicSmem));
+        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                            (int)cudaSharedmemCarveoutMaxShared));
+        CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&info.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, device));
+        CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&info.reserved, cudaDevAttrReservedSharedMemoryPerBlock, device));
+        CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&info.regs_per_sm, cudaDevAttrMaxRegistersPerMultiprocessor, device));
+        cudaFuncAttributes fattr;
+        CIVIC_CUDA_TRY(cudaFuncGetAttributes(&fattr, civic::kv_attention_kernel));
+        info.regs_per_thread = fattr.numRegs;
+        info.ready.store(1, std::memory_order_release);
+    }
+    const int smem_per_sm = info.smem_per_sm, reserved = info.reserved, regs_per_sm = info.regs_per_sm;
+    const int regs_per_block = ((info.regs_per_thread + 7) / 8 * 8) * civic::kAttnThreads;
+    int blocks_per_sm = (int)((size_t)smem_per_sm / (pl.attn_smem + (size_t)reserved));
+    blocks_per_sm = std::min(blocks_per_sm, regs_per_sm / std::max(regs_per_block, 1));
+    blocks_per_sm = std::min(blocks_per_sm, 2048 / civic::kAttnThreads);
+    blocks_per_sm = std::min(blocks_per_sm, (int)(512 / civic::attn_tmem_cols(head_dim, s)));
+    ap.tiles_per_block = attention_tiles_per_block(q_tiles, (int64_t)n_heads * n_img, blocks_per_sm);
+
+    // everything that can fail on the host has happened: from here on work is enqueued
     const bool pdl = programmatic();
     CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
     float* partial = (float*)(ws + pl.partial_off);
@@ -825,38 +929,6 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
         if (gs != CIVIC_OK) return gs;
     }
 
-    const float scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
-    const int32_t q_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
-    CUtensorMap map_o;  // boxes of 32 rows x 64 features: one softmax warp's share of a tile
-    {
-        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
-        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
-        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32)) != CIVIC_OK) return ms;
-    }
-    civic::AttnParams ap;
-    ap.error = device_status; ap.m_e = m_e; ap.d = head_dim; ap.s = s;
-    ap.scale_log2e = scale_log2e;
-    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)pl.attn_smem));
-    // all of the SM's memory as shared memory, so that two blocks of 113 KB can be resident
-    CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                        (int)cudaSharedmemCarveoutMaxShared));
-    // Blocks that fit on an SM together, by shared memory, registers, threads and tensor memory
-    // columns.  (The runtime's occupancy query answers 1 for this kernel whatever its shared
-    // memory, while two blocks were measured running side by side on the SMs.)
-    int dev = 0, smem_per_sm = 0, reserved = 0, regs_per_sm = 0;
-    CIVIC_CUDA_TRY(cudaGetDevice(&dev));
-    CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev));
-    CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&reserved, cudaDevAttrReservedSharedMemoryPerBlock, dev));
-    CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&regs_per_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev));
-    cudaFuncAttributes fattr;
-    CIVIC_CUDA_TRY(cudaFuncGetAttributes(&fattr, civic::kv_attention_kernel));
-    const int regs_per_block = ((fattr.numRegs + 7) / 8 * 8) * civic::kAttnThreads;
-    int blocks_per_sm = (int)((size_t)smem_per_sm / (pl.attn_smem + (size_t)reserved));
-    blocks_per_sm = std::min(blocks_per_sm, regs_per_sm / std::max(regs_per_block, 1));
-    blocks_per_sm = std::min(blocks_per_sm, 2048 / civic::kAttnThreads);
-    blocks_per_sm = std::min(blocks_per_sm, (int)(512 / civic::attn_tmem_cols(head_dim, s)));
-    ap.tiles_per_block = attention_tiles_per_block(q_tiles, (int64_t)n_heads * n_img, blocks_per_sm);
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel,
                                  dim3((unsigned)((q_tiles + ap.tiles_per_block - 1) / ap.tiles_per_block),
                                       (unsigned)n_heads, (unsigned)n_img),
@@ -912,9 +984,12 @@ civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civ
             n_max = n > n_max ? n : n_max;
         }
         const size_t smem = civic::select_smem_bytes(n_max);
-        if (smem > 48 * 1024)
-            CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::select_ragged_kernel,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        {
+            static std::atomic<int> smem_allowed[64];
+            const civic_status_t as = allow_dynamic_smem(
+                civic::select_ragged_kernel, civic::select_smem_bytes(civic_select_max_tokens()), smem_allowed);
+            if (as != CIVIC_OK) return as;
+        }
         CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::select_ragged_kernel, (unsigned)ns,
                                      (unsigned)select_threads(n_max), smem, (cudaStream_t)stream, p));
         g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -1109,6 +1184,7 @@ civic_status_t civic_compact_kv_paged(const void* const* k_src, const void* cons
     p.block_table = block_table;
     p.max_pages = max_pages_per_seq;
     p.page_size = page_size;
+    p.n_pages = n_pages;
     return launch_kv<civic::kPaged>(p, k_src, v_src, k_cache, v_cache, n_layers, (cudaStream_t)stream);
 }
 
@@ -1164,7 +1240,43 @@ civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, in
     if (blocks > 8LL * sm_count()) blocks = 8LL * sm_count();
     CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::gather_pos_planes_kernel, (unsigned)blocks, threads, 0,
                                  (cudaStream_t)stream, pos, seq_idx, pos_out, n_planes, n_seq, seq_len,
-                                 s_out));
+                                 s_out, g_index_check));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+civic_status_t civic_set_index_check(int32_t* fault_record)
+{
+    if (!aligned(fault_record, 4)) return CIVIC_ERR_ALIGNMENT;
+    g_index_check = fault_record;
+    return CIVIC_OK;
+}
+
+civic_status_t civic_validate_indices(const int32_t* idx, int32_t n_rows, int32_t row_len, int32_t limit,
+                                      int32_t require_ascending, int32_t* fault_record, void* stream)
+{
+    if (n_rows < 0 || row_len < 0 || limit < 0) return CIVIC_ERR_INVALID_ARG;
+    const long long total = (long long)n_rows * row_len;
+    if (total == 0) return CIVIC_OK;
+    if (!idx || !fault_record) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(idx, 4) || !aligned(fault_record, 4)) return CIVIC_ERR_ALIGNMENT;
+    if (overlaps(idx, (size_t)total * 4, fault_record, 16)) return CIVIC_ERR_INVALID_ARG;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    if (blocks > 8LL * sm_count()) blocks = 8LL * sm_count();
+    CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::validate_indices_kernel, (unsigned)blocks, threads, 0,
+                                 (cudaStream_t)stream, idx, n_rows, row_len, limit, require_ascending, fault_record));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+civic_status_t civic_selftest_bounded_wait(uint64_t limit_cycles, int32_t* record, void* stream)
+{
+    if (!record || limit_cycles == 0 || limit_cycles > ((uint64_t)1 << 24)) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(record, 4)) return CIVIC_ERR_ALIGNMENT;
+    CIVIC_CUDA_TRY(cudaMemsetAsync(record, 0, 8, (cudaStream_t)stream));
+    CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::bounded_wait_selftest_kernel, 1u, 64u, 0, (cudaStream_t)stream,
+                                 (unsigned long long)limit_cycles, (int*)record));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CIVIC_OK;
 }

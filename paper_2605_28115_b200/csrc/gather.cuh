@@ -42,7 +42,24 @@ struct GatherParams {
     // kMerge: src[0] is the text [n_planes, seq_len, row], visual the dense visual rows
     const char* visual;  // [n_planes, n_vis, row]
     int32_t vis_start, n_vis, k_vis;
+    // index validation (kernels instantiated with CHECK only): int32[4] fault record, see
+    // report_bad_index; n_pages bounds the block table's entries
+    int32_t* check;
+    int32_t n_pages;
 };
+
+// Fault record of the checked kernels: {code, plane, position, offending value}.  The first
+// thread to find a fault claims word 0 (0 -> code) and fills in the rest; later faults leave the
+// record alone, so it names ONE offending entry.  The record is sticky: only the caller clears it.
+enum IndexFault { kIndexOk = 0, kIndexOutOfRange = 1, kIndexNotAscending = 2, kIndexBadPage = 3 };
+__device__ __forceinline__ void report_bad_index(int32_t* record, int code, int plane, int pos, int value)
+{
+    if (atomicCAS(record, 0, code) == 0) {
+        record[1] = plane;
+        record[2] = pos;
+        record[3] = value;
+    }
+}
 
 template <typename VecT>
 __device__ __forceinline__ VecT load_stream(const VecT* p);
@@ -64,6 +81,7 @@ __device__ __forceinline__ uint32_t load_stream<uint32_t>(const uint32_t* p)
 __device__ __forceinline__ void store_stream(uint4* p, uint4 v) { __stcs(p, v); }
 __device__ __forceinline__ void store_stream(uint32_t* p, uint32_t v) { __stcs(p, v); }
 
+template <bool CHECK>
 __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int n_blocks)
 {
     const long long total = (long long)p.n_planes * p.s_out * 3;
@@ -73,36 +91,59 @@ __device__ __forceinline__ void gather_pos(const GatherParams& p, int block, int
         const int c = (int)(e - row * 3);
         const int s = (int)(row / p.s_out);
         const int32_t i = p.idx[row];
+        if (CHECK && (uint32_t)i >= (uint32_t)p.seq_len) {  // neither read nor written
+            report_bad_index(p.check, kIndexOutOfRange, s, (int)(row - (long long)s * p.s_out), i);
+            continue;
+        }
         p.pos_dst[e] = p.pos_src[((size_t)s * p.seq_len + i) * 3 + c];
     }
 }
 
 // Source row of output row j of plane q; idx_row is the plane's row of the index array.
-template <int MODE>
-__device__ __forceinline__ const char* source_row(const GatherParams& p, int tensor, int q, int idx_row, int j)
+// With CHECK an index outside its range is recorded and the function returns false: the caller
+// then neither reads nor writes that row.
+template <int MODE, bool CHECK>
+__device__ __forceinline__ bool source_row(const GatherParams& p, int tensor, int q, int idx_row, int j,
+                                           const char*& src)
 {
     if constexpr (MODE == kMerge) {
-        if (j < p.vis_start) return p.src[0] + ((size_t)q * p.seq_len + j) * p.row_bytes;
-        if (j < p.vis_start + p.k_vis) {
+        if (j < p.vis_start) {
+            src = p.src[0] + ((size_t)q * p.seq_len + j) * p.row_bytes;
+        } else if (j < p.vis_start + p.k_vis) {
             const int32_t i = __ldg(p.idx + (size_t)q * p.k_vis + (j - p.vis_start));
-            return p.visual + ((size_t)q * p.n_vis + i) * p.row_bytes;
+            if (CHECK && (uint32_t)i >= (uint32_t)p.n_vis) {
+                report_bad_index(p.check, kIndexOutOfRange, q, j - p.vis_start, i);
+                return false;
+            }
+            src = p.visual + ((size_t)q * p.n_vis + i) * p.row_bytes;
+        } else {
+            src = p.src[0] + ((size_t)q * p.seq_len + (j - p.k_vis + p.n_vis)) * p.row_bytes;
         }
-        return p.src[0] + ((size_t)q * p.seq_len + (j - p.k_vis + p.n_vis)) * p.row_bytes;
     } else {
         const int32_t i = __ldg(p.idx + (size_t)idx_row * p.s_out + j);
-        return p.src[tensor] + ((size_t)q * p.seq_len + i) * p.row_bytes;
+        if (CHECK && (uint32_t)i >= (uint32_t)p.seq_len) {
+            report_bad_index(p.check, kIndexOutOfRange, idx_row, j, i);
+            return false;
+        }
+        src = p.src[tensor] + ((size_t)q * p.seq_len + i) * p.row_bytes;
     }
+    return true;
 }
 
-template <int MODE>
-__device__ __forceinline__ char* destination_row(const GatherParams& p, int tensor, int q, int j)
+template <int MODE, bool CHECK>
+__device__ __forceinline__ bool destination_row(const GatherParams& p, int tensor, int q, int j, char*& dst)
 {
     if constexpr (MODE == kPaged) {
         const int32_t page = __ldg(p.block_table + (size_t)q * p.max_pages + j / p.page_size);
-        return p.dst[tensor] + ((size_t)page * p.page_size + j % p.page_size) * p.row_bytes;
+        if (CHECK && (uint32_t)page >= (uint32_t)p.n_pages) {
+            report_bad_index(p.check, kIndexBadPage, q, j / p.page_size, page);
+            return false;
+        }
+        dst = p.dst[tensor] + ((size_t)page * p.page_size + j % p.page_size) * p.row_bytes;
     } else {
-        return p.dst[tensor] + ((size_t)q * p.s_out + j) * p.row_bytes;
+        dst = p.dst[tensor] + ((size_t)q * p.s_out + j) * p.row_bytes;
     }
+    return true;
 }
 
 // One warp per tile of 32 * UNROLL vectors (2 KB for 16-byte vectors), no grid-stride loop.
@@ -110,12 +151,12 @@ __device__ __forceinline__ char* destination_row(const GatherParams& p, int tens
 // source and destination in address order, which measured faster on B200 than a persistent
 // grid-stride loop.  Every lane has its UNROLL loads in flight before its first store.
 // LARGE: a row is ceil(vecs / tile) tiles.  SMALL: a tile is floor(tile / vecs) whole rows.
-template <typename VecT, int UNROLL, int MODE, bool SMALL>
+template <typename VecT, int UNROLL, int MODE, bool SMALL, bool CHECK>
 __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __grid_constant__ GatherParams p)
 {
     wait_for_prior_kernels();
     if (blockIdx.x >= p.main_blocks) {
-        gather_pos(p, blockIdx.x - p.main_blocks, gridDim.x - p.main_blocks);
+        gather_pos<CHECK>(p, blockIdx.x - p.main_blocks, gridDim.x - p.main_blocks);
         return;
     }
     constexpr int kTileVecs = 32 * UNROLL;
@@ -135,8 +176,13 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __gri
         const int q = (int)(rem / p.s_out);
         const int j = (int)(rem - (long long)q * p.s_out);
         const int idx_row = MODE == kHeads ? q / p.idx_div : q;
-        const VecT* src = reinterpret_cast<const VecT*>(source_row<MODE>(p, tensor, q, idx_row, j));
-        VecT* dst = reinterpret_cast<VecT*>(destination_row<MODE>(p, tensor, q, j));
+        const char* src_row = nullptr;
+        char* dst_row = nullptr;
+        const bool ok = source_row<MODE, CHECK>(p, tensor, q, idx_row, j, src_row) &&
+                        destination_row<MODE, CHECK>(p, tensor, q, j, dst_row);
+        if (CHECK && !ok) return;  // the whole warp: a tile lies inside one row
+        const VecT* src = reinterpret_cast<const VecT*>(src_row);
+        VecT* dst = reinterpret_cast<VecT*>(dst_row);
         const int v0 = tile * kTileVecs + lane;
         VecT buf[UNROLL];
 #pragma unroll
@@ -174,9 +220,14 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __gri
                 if (q == n_planes) { q = 0; idx_row = 0; ++tensor; }
             }
             if (r < rows_per_tile && tensor < (uint32_t)p.n_tensors) {
-                buf[u] = load_stream(reinterpret_cast<const VecT*>(
-                                         source_row<MODE>(p, (int)tensor, (int)q, (int)idx_row, (int)j)) + c);
-                dst[u] = reinterpret_cast<VecT*>(destination_row<MODE>(p, (int)tensor, (int)q, (int)j)) + c;
+                const char* src_row = nullptr;
+                char* dst_row = nullptr;
+                const bool ok = source_row<MODE, CHECK>(p, (int)tensor, (int)q, (int)idx_row, (int)j, src_row) &&
+                                destination_row<MODE, CHECK>(p, (int)tensor, (int)q, (int)j, dst_row);
+                if (!CHECK || ok) {
+                    buf[u] = load_stream(reinterpret_cast<const VecT*>(src_row) + c);
+                    dst[u] = reinterpret_cast<VecT*>(dst_row) + c;
+                }
             }
             r += step_r;
             c += step_c;
@@ -188,10 +239,11 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const __gri
     }
 }
 
-// out[c, s, j] = pos[c, s, idx[s, j]] for plane-major position ids.
+// out[c, s, j] = pos[c, s, idx[s, j]] for plane-major position ids.  `check` (a fault record as
+// in report_bad_index, or NULL) switches the range test of the indices on.
 __global__ void gather_pos_planes_kernel(const int32_t* __restrict__ pos, const int32_t* __restrict__ idx,
                                          int32_t* __restrict__ out, int n_planes, int n_seq, int seq_len,
-                                         int s_out)
+                                         int s_out, int32_t* check)
 {
     release_next_kernel();
     wait_for_prior_kernels();
@@ -201,7 +253,28 @@ __global__ void gather_pos_planes_kernel(const int32_t* __restrict__ pos, const 
         const int c = (int)(e / per_plane);
         const long long rem = e - (long long)c * per_plane;  // s * s_out + j
         const int s = (int)(rem / s_out);
-        out[e] = pos[((size_t)c * n_seq + s) * seq_len + idx[rem]];
+        const int32_t i = idx[rem];
+        if (check && (uint32_t)i >= (uint32_t)seq_len) {
+            report_bad_index(check, kIndexOutOfRange, s, (int)(rem - (long long)s * s_out), i);
+            continue;
+        }
+        out[e] = pos[((size_t)c * n_seq + s) * seq_len + i];
+    }
+}
+
+// Stand-alone validation of an index array [n_rows, row_len]: every value in [0, limit) and, if
+// asked, every row strictly ascending.  Thread per entry; faults go to the record.
+__global__ void validate_indices_kernel(const int32_t* __restrict__ idx, int n_rows, int row_len, int limit,
+                                        int ascending, int32_t* record)
+{
+    wait_for_prior_kernels();
+    const long long total = (long long)n_rows * row_len;
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const int row = (int)(e / row_len), j = (int)(e - (long long)row * row_len);
+        const int32_t i = idx[e];
+        if ((uint32_t)i >= (uint32_t)limit) report_bad_index(record, kIndexOutOfRange, row, j, i);
+        else if (ascending && j > 0 && idx[e - 1] >= i) report_bad_index(record, kIndexNotAscending, row, j, i);
     }
 }
 

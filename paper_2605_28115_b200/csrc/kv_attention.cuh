@@ -138,10 +138,9 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
 {
     extern __shared__ __align__(1024) uint8_t attn_smem[];
     uint8_t* base = attn_smem;
-    if (smem_u32(base) & 1023u) {  // the swizzled tiles would be misplaced: refuse, before anything is set up
-        if (threadIdx.x == 0) atomicCAS(p.error, 0, kAggMisaligned);
-        return;
-    }
+    // the swizzled tiles would be misplaced: the block then does no work (reported below, after
+    // the wait for the previous kernels like every other access to global memory)
+    const bool misplaced = (smem_u32(base) & 1023u) != 0;
     const int d = p.d, s = p.s, d_blocks = d >> 6, s_blocks = s >> 6;
     uint8_t* k_sm = base;
     uint8_t* v_sm = k_sm + d_blocks * s * 128;
@@ -180,11 +179,12 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
     }
     if (warp == 1) tmem_alloc(&sy.tmem_base, tmem_cols);
     wait_for_prior_kernels();
+    if (misplaced && threadIdx.x == 0) atomicCAS(p.error, 0, kAggMisaligned);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sy.tmem_base;
-    const bool stop = *p.error != 0 || n_tiles <= 0;
+    const bool stop = misplaced || *p.error != 0 || n_tiles <= 0;
 
     // A wait on a "free / empty" barrier uses the opposite parity, so the first pass over a
     // fresh barrier falls through.

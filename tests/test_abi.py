@@ -271,3 +271,22 @@ def test_binding_refuses_cpu_tensors():
 def test_missing_library_fails_loudly(tmp_path):
     with pytest.raises(RuntimeError, match="no fallback"):
         civic.load(str(tmp_path / "libcivic.so"))
+
+
+def test_index_check_entries_validate_on_host(lib):
+    before = lib.civic_launch_count()
+    assert lib.civic_set_index_check(0x1002) == 4
+    assert lib.civic_set_index_check(0x1000) == 0
+    assert lib.civic_set_index_check(None) == 0
+    f = lib.civic_validate_indices
+    assert f(0x1000, -1, 4, 10, 1, 0x9000, None) == 1
+    assert f(0x1000, 2, 4, -1, 1, 0x9000, None) == 1
+    assert f(None, 2, 4, 10, 1, 0x9000, None) == 1
+    assert f(0x1000, 2, 4, 10, 1, None, None) == 1
+    assert f(0x1002, 2, 4, 10, 1, 0x9000, None) == 4
+    assert f(0x1000, 2, 4, 10, 1, 0x1010, None) == 1  # the record inside the index array
+    assert f(0x1000, 0, 4, 10, 1, None, None) == 0    # nothing to check
+    g = lib.civic_selftest_bounded_wait
+    assert g(0, 0x1000, None) == 1 and g(1 << 25, 0x1000, None) == 1 and g(100, None, None) == 1
+    assert g(100, 0x1002, None) == 4
+    assert lib.civic_launch_count() == before

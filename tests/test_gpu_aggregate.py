@@ -24,6 +24,7 @@ from paper_2605_28115_b200 import build, civic
 pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
+BOUND_SHARE = 0.5  # regression bar: the largest error as a share of the derived bound
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -65,11 +66,18 @@ def check(x, a, tau):
     z_o, mass_o = OA.anchor_aggregate_batch(x64, a64, tau)
     e = eps_w(tau, d_v)
     z_g = z.float().cpu().numpy().astype(np.float64)
+    worst = 0.0
     for i in range(n_img):
         w = OA.aggregation_weights(x64[i], a64, tau)
         bound = e * (w @ np.abs(x64[i])) + 2.0 ** -9 * np.abs(z_o[i])
-        assert np.all(np.abs(z_g[i] - z_o[i]) <= bound), (i, float(np.max(np.abs(z_g[i] - z_o[i]) / bound)))
-    assert np.all(np.abs(mass.cpu().numpy() - mass_o) <= e * mass_o + 1e-30)
+        share = np.abs(z_g[i] - z_o[i]) / np.maximum(bound, 1e-300)
+        assert np.all(share <= 1.0), (i, float(share.max()))
+        worst = max(worst, float(share.max()))
+    mass_share = np.abs(mass.cpu().numpy() - mass_o) / (e * mass_o + 1e-30)
+    assert np.all(mass_share <= 1.0)
+    worst = max(worst, float(mass_share.max()))
+    # the bound is a worst case; an accuracy regression that stays inside it is still seen here
+    assert worst <= BOUND_SHARE, f"largest error is {worst:.2f} of the bound (bar {BOUND_SHARE})"
     return z, mass
 
 
@@ -124,3 +132,26 @@ def test_token_mass_feeds_the_selection():
     assert int(status.item()) == 0
     want = oracle.default.select(mass.cpu().numpy(), 1, 32, 32, 4, 4, 1, 341)
     assert np.array_equal(keep.cpu().numpy(), want)
+
+
+def test_a_wait_that_never_gets_its_signal_ends_with_a_status():
+    """The kernels' bounded wait, run on a barrier nobody signals (no copy, no tensor-core work in
+    flight): it comes back within a millisecond with the time-out code in the device word, the
+    block's second waiter leaves through the stop flag, and the next ordinary call on the same
+    stream is still right."""
+    rec = torch.full((2,), -1, dtype=torch.int32, device=DEV)
+    civic.civic_selftest_bounded_wait(1 << 16, rec)  # first call: module load, not timed
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rec.fill_(-1)
+    start.record()
+    civic.civic_selftest_bounded_wait(1 << 16, rec)
+    end.record()
+    x, a = inputs(1, 200, 130, 128, seed=330)
+    check(x, a, 0.1)  # enqueued behind the self-test on the same stream
+    assert rec.cpu().tolist() == [1, 1]  # kAggTimeoutFull; the flag released the second waiter
+    assert start.elapsed_time(end) < 1.0, "the wait did not stop at its limit (2^16 cycles = 33 us)"
+    lib = civic.load()
+    assert lib.civic_selftest_bounded_wait(0, rec.data_ptr(), None) == 1
+    assert lib.civic_selftest_bounded_wait(1 << 25, rec.data_ptr(), None) == 1
+    assert lib.civic_selftest_bounded_wait(100, None, None) == 1

@@ -21,6 +21,7 @@ from paper_2605_28115_b200 import build, civic
 pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
+BOUND_SHARE = 0.5
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -72,6 +73,9 @@ def check(q, k, v, r, heads):
             err = np.abs(got[i][:, c] - want[:, c])
             assert np.all(err <= bound), (i, h, float(np.max(err / bound)))
             worst = max(worst, float(np.max(err / bound)))
+    # The bound is a worst case; measured, the kernels use about a fifth of it.  Half of it is the
+    # regression bar: a change that loses accuracy inside the bound is still seen.
+    assert worst <= BOUND_SHARE, f"largest error is {worst:.2f} of the bound (bar {BOUND_SHARE})"
     return out, worst
 
 

@@ -188,7 +188,7 @@ def padded(shape, dtype, fill):
     return view, check
 
 
-@pytest.mark.parametrize("wl", [W.C1, W.C2, W.C4, W.C5_THIRD], ids=lambda wl: wl.name)
+@pytest.mark.parametrize("wl", [W.C1, W.C2, W.C3, W.C4, W.C5_HALF, W.C5_THIRD, W.C5_QUARTER], ids=lambda wl: wl.name)
 def test_compact_workloads(wl):
     s = W.scores(wl)
     keep = O.select(s, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)

@@ -1,6 +1,10 @@
-"""The N > 1 path on CPU: two gloo ranks split the segments, run their shards independently
-(here with the CPU oracle standing in for the device path) and reproduce the unsharded result
-with no payload exchange; timing is reduced with MAX."""
+"""The host-side plumbing of the N > 1 path on CPU: the partition helper (shard_range), the
+throughput bookkeeping and the MAX reduction of the timing over two gloo ranks.
+
+What this file does NOT show: anything about the CUDA path.  In the two-rank test both the
+sharded and the unsharded results come from the CPU oracle; it checks only that the partition
+covers every segment exactly once and that no payload has to be exchanged.  The device path on
+several GPUs is `bench.py --gpus N`."""
 import os
 import socket
 
