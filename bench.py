@@ -34,13 +34,24 @@ UNIT = "GB/s"
 KV_EVENT_STRIDE = 10
 FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used when MEASURED_PEAKS.json is absent
 
-# DRAM bytes (read + write) of ONE civic_compact_kv launch, from the ncu capture summarised in
-# profiles/; keyed by workload name.  None = not captured for that workload.
+# DRAM bytes (read + write) of ONE civic_compact_kv launch, keyed by workload name: NOT measured by
+# the run that prints them, but taken from the ncu captures summarised in profiles/ (an 8-layer case
+# of the same kernel, dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled by 36 / 8: the
+# traffic grows in proportion to the layers).  Absent = not captured for that workload.
 NCU_DRAM_TRAFFIC_PER_LAUNCH = {
-    # profiles/gather_rows_kernel_c3_kv.md: 8-layer capture, reads x4.5, writes = algorithmic minus
-    # the 52.0 MB that were still dirty in L2 when the kernel ended
-    "c3_kv_qwen3vl8b": 1_859_200_000,
+    # reads x4.5, writes = algorithmic minus the 52.0 MB that were still dirty in L2 at kernel end
+    "c3_kv_qwen3vl8b": (1_859_200_000, "profiles/gather_rows_kernel_c3_kv.md"),
 }
+TRAFFIC_SOURCE = ("ncu capture of an 8-layer case of the same kernel, scaled to {layers} layers; "
+                  "not measured by this run ({file})")
+
+
+def ncu_traffic(wl_name, layers):
+    """(bytes per launch, where the figure comes from) or (None, None)."""
+    hit = NCU_DRAM_TRAFFIC_PER_LAUNCH.get(wl_name)
+    if not hit:
+        return None, None
+    return hit[0], TRAFFIC_SOURCE.format(layers=layers, file=hit[1])
 
 
 def parse_args():
@@ -62,6 +73,8 @@ def parse_args():
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time its replays: the GPU-side latency of the "
                          "step without the Python binding's per-call host time (for the small workloads)")
+    ap.add_argument("--no-others", action="store_true",
+                    help="skip the other workloads that the default run times after the main one")
     ap.add_argument("--layers", type=int, default=0,
                     help="shrink the workload to this many K/V layers (profiling a small case); "
                          "the JSON line then names the reduced workload")
@@ -92,6 +105,10 @@ def pick_workload(args):
     if args.layers and wl.n_layers:
         wl = wl.replace(name=f"{wl.name}_reduced_to_{args.layers}_layers", n_layers=args.layers)
     return wl
+
+
+def parallelism_of(world):
+    return f"dp{world}" if world > 1 else "single"
 
 
 def config_of(wl, extra=None):
@@ -400,6 +417,312 @@ def cpu_baseline(st: DeviceState, limit_s: float = 20.0):
             "ms_per_sample": med * 1e3}
 
 
+def path_equals_oracle(st: DeviceState) -> bool:
+    """Every result of the last device-resident step of `st` against the CPU oracle, bit for bit:
+    keep indices, hidden rows, position ids, sequence indices, all layers' K and V rows."""
+    import numpy as np
+    import torch
+
+    import oracle
+
+    wl, o = st.wl, oracle.default
+    o.set_threads(0)
+    bits = lambda x: x.contiguous().view(torch.int16).cpu().numpy()
+    keep = o.select(st.scores_host, wl.t, wl.h, wl.w, wl.region_h, wl.region_w, wl.floor_m, wl.k)
+    ok = np.array_equal(st.keep.cpu().numpy(), keep)
+    h_o, p_o = o.compact(bits(st.hidden) if st.hidden is not None else None, st.pos_host, keep)
+    if st.hidden is not None:
+        ok = ok and np.array_equal(bits(st.hidden_out), h_o)
+    ok = ok and np.array_equal(st.pos_out.cpu().numpy(), p_o)
+    if wl.n_layers and st.kv_layout == "token_major":
+        idx = o.seq_indices(keep, wl.seq_len, wl.text_before, wl.n)
+        ok = ok and np.array_equal(st.seq_idx.cpu().numpy(), idx)
+        row = wl.kv_heads * wl.head_dim
+        flat = lambda x: bits(x).reshape(wl.n_seg, -1, row)
+        for l0 in range(0, wl.n_layers, 6):  # six layers at a time bounds the host copies
+            ls = range(l0, min(l0 + 6, wl.n_layers))
+            k_o, v_o = o.compact_kv([flat(st.k_src[l]) for l in ls], [flat(st.v_src[l]) for l in ls], idx)
+            for j, l in enumerate(ls):
+                ok = ok and np.array_equal(flat(st.k_dst[l]), k_o[j]) and np.array_equal(flat(st.v_dst[l]), v_o[j])
+    return bool(ok)
+
+
+def contiguous_copy_rate(st: DeviceState, launches=10):
+    """GB/s of civic_compact_kv when it keeps EVERY row (identity indices): the same kernel as a plain
+    contiguous copy of the whole K/V set, i.e. the most this gather could reach on this GPU today."""
+    import torch
+
+    from paper_2605_28115_b200 import civic
+
+    wl = st.wl
+    idx = torch.arange(wl.seq_len, dtype=torch.int32, device=st.dev).repeat(wl.n_seg, 1).contiguous()
+    k_all = [torch.empty_like(x) for x in st.k_src]
+    v_all = [torch.empty_like(x) for x in st.v_src]
+    tables = civic.kv_tables(st.k_src, st.v_src, k_all, v_all)
+    for _ in range(2):
+        civic.civic_compact_kv(tables, idx)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(launches):
+        civic.civic_compact_kv(tables, idx)
+    end.record()
+    torch.cuda.synchronize()
+    nbytes = 2 * sum(x.numel() * x.element_size() for x in st.k_src + st.v_src)
+    return nbytes / (start.elapsed_time(end) / launches * 1e-3) / 1e9
+
+
+def kv_roofline(wl, kv_bytes, kv_ms, kv_layout="token_major", default_variant=True):
+    """The roofline object of the K/V gather from event-bracketed launches (ms each)."""
+    kv_avg = sum(kv_ms) / len(kv_ms)
+    peak, which = measured_peak()
+    achieved = kv_bytes / (kv_avg * 1e-3) / 1e9
+    kernel = {"token_major": "civic_compact_kv", "head_major": "civic_compact_kv_heads",
+              "paged": "civic_compact_kv_paged"}[kv_layout]
+    traffic, source = ncu_traffic(wl.name, wl.n_layers) if default_variant else (None, None)
+    return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_source": which, "traffic": traffic, "traffic_source": source,
+            "algorithmic_bytes_per_launch": kv_bytes, "us_per_launch": kv_avg * 1e3,
+            "us_per_launch_min": min(kv_ms) * 1e3, "launches_timed": len(kv_ms),
+            "frac_of_8TBps_nominal": achieved / 8000.0}
+
+
+def time_other_path_workload(wl, dev, steps, with_oracle):
+    """One of the other select + compact (+ K/V) configurations on one GPU: device-resident steps as a
+    plain loop; the K/V configurations bracket every tenth K/V launch with events, the small ones are
+    also timed as replays of a CUDA graph of one step."""
+    import torch
+
+    from paper_2605_28115_b200 import civic
+
+    st = DeviceState(wl, dev, 0)
+    nbytes = step_bytes(wl)
+    for _ in range(5):
+        st.step()
+    torch.cuda.synchronize()
+    kv_ev = {i: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for i in range(0, steps, 10)} if wl.n_layers else {}
+    sampler = ClockSampler(torch.device(dev).index or 0)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = civic.launch_count()
+    sampler.start()
+    torch.cuda.synchronize()
+    start.record()
+    for i in range(steps):
+        st.step(kv_ev.get(i))
+    end.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(end) / steps
+    out = {"workload": wl.name, "steps": steps, "us_per_step": ms * 1e3,
+           "value": nbytes["total"] / (ms * 1e-3) / 1e9, "unit": UNIT, "bytes_per_step": nbytes["total"],
+           "gpu_launches": civic.launch_count() - launches0,
+           "l2": config_of(wl)["l2"]}
+    if kv_ev:
+        out["roofline"] = kv_roofline(wl, nbytes["kv"], [a.elapsed_time(b) for a, b in kv_ev.values()])
+    else:  # launch-bound: also as a graph of one step, without the binding's host time per call
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            st.step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                st.step()
+        for _ in range(5):
+            graph.replay()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(steps):
+            graph.replay()
+        end.record()
+        torch.cuda.synchronize()
+        out["graph_replay_us_per_step"] = start.elapsed_time(end) / steps * 1e3
+        peak, _ = measured_peak()
+        out["hbm_time_us_at_measured_peak"] = nbytes["total"] / peak / 1e3
+        st.step()
+        torch.cuda.synchronize()
+    out["clocks"] = sampler.stop()
+    if with_oracle:
+        out["equals_oracle"] = path_equals_oracle(st)
+    return out
+
+
+def aggregate_within_bound(x0, anchors, tau, z0, mass):
+    """Image 0 of a civic_anchor_aggregate result against the fp64 oracle: the largest error as a
+    share of the element-wise bound derived from the arithmetic (bf16 anchors, fp32 accumulation,
+    bf16 weights and result), and the oracle's time."""
+    import numpy as np
+
+    from oracle import aggregate as OA
+
+    d_v = x0.shape[2]
+    x64, a64 = x0[0].double().cpu().numpy(), anchors.double().cpu().numpy()
+    t0 = time.perf_counter()
+    z_o, w_o = OA.anchor_aggregate(x64, a64, tau)
+    seconds = time.perf_counter() - t0
+    d_cos = 2.0 ** -9 + d_v * 2.0 ** -24
+    eps_w = np.expm1(2 * d_cos / tau) + 2.0 ** -8
+    w = OA.aggregation_weights(x64, a64, tau)
+    bound = eps_w * (w @ np.abs(x64)) + 2.0 ** -9 * np.abs(z_o)
+    err = np.abs(z0[0].float().cpu().numpy().astype(np.float64) - z_o)
+    share = float(np.max(err / np.maximum(bound, 1e-300)))
+    mass_o = w.sum(axis=0)
+    share = max(share, float(np.max(np.abs(mass[0].cpu().numpy() - mass_o) / (eps_w * mass_o + 1e-30))))
+    return share, float(err.max()), seconds
+
+
+def time_aggregate(w, dev, steps, warm):
+    """civic_anchor_aggregate (Eq. 8) on workload `w`: (result dict, tensors for further checks)."""
+    import torch
+
+    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import workloads as W
+
+    x0, anchors = W.agg_inputs(w, dev)
+    z0 = torch.empty((w.n_img, w.m_e, w.d_v), dtype=torch.bfloat16, device=dev)
+    mass = torch.empty((w.n_img, w.t_e), dtype=torch.float32, device=dev)
+    ws = torch.empty(civic.anchor_aggregate_workspace_bytes(w.n_img, w.t_e, w.m_e, w.d_v), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        civic.civic_anchor_aggregate(x0, anchors, w.tau, z0=z0, token_mass=mass, workspace=ws, device_status=status)
+
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.device(dev).index or 0)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = civic.launch_count()
+    sampler.start()
+    start.record()
+    for _ in range(steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = civic.launch_count() - launches0
+    ms = start.elapsed_time(end) / steps
+    if int(status.item()) != 0:
+        raise SystemExit(f"a wait inside the aggregation kernels timed out (status {int(status.item())})")
+    value = w.flops / (ms * 1e-3) / 1e12
+    burst, sustained, which = measured_tensor_peak()
+    timed_s = ms * 1e-3 * steps
+    peak = sustained if timed_s > 0.5 else burst  # a long loop runs under the power cap
+    roofline = {"bound": "tensor", "kernel": "civic_anchor_aggregate: five launches, of which the two tcgen05 "
+                "contractions carry all the flops (the other three are HBM-bound helpers and are inside the time)",
+                "achieved": value, "peak": peak, "unit": "TFLOP/s", "frac": value / peak, "peak_source": which,
+                "peak_kind": "sustained" if timed_s > 0.5 else "burst", "frac_of_burst_peak": value / burst,
+                "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
+    res = {"workload": w.name, "steps": steps, "us_per_step": ms * 1e3, "value": value, "unit": "TFLOP/s",
+           "gpu_launches": launches, "clocks": clocks, "roofline": roofline}
+    return res, (x0, anchors, z0, mass, step)
+
+
+def kv_attention_within_bound(q, k, v, r, n_heads, out):
+    """Image 0 of a civic_kv_compressed_attention result against the fp64 oracle: the largest error as
+    a share of the element-wise bound derived from the arithmetic, and the oracle's time."""
+    import numpy as np
+
+    from oracle import aggregate as OA
+
+    q64, k64, v64 = (a[0].double().cpu().numpy() for a in (q, k, v))
+    r64 = r.double().cpu().numpy()
+    d = q64.shape[1] // n_heads
+    t0 = time.perf_counter()
+    want, k_c, v_c = OA.kv_compressed_attention(q64, k64, v64, r64, n_heads)
+    seconds = time.perf_counter() - t0
+    rbar = OA.column_normalize(r64)
+    abs_kc, abs_vc = rbar.T @ np.abs(k64), rbar.T @ np.abs(v64)
+    got = out[0].float().cpu().numpy().astype(np.float64)
+    share = 0.0
+    for h in range(n_heads):
+        c = slice(h * d, (h + 1) * d)
+        lam = 2.0 ** -8 * np.max(np.abs(q64[:, c]) @ abs_kc[:, c].T) / np.sqrt(d)
+        eps_w = np.expm1(2 * lam) + 2.0 ** -8 * (1 + 2.0 ** -7)
+        logits = q64[:, c] @ k_c[:, c].T / np.sqrt(d)
+        wgt = np.exp(logits - logits.max(axis=1, keepdims=True))
+        wgt /= wgt.sum(axis=1, keepdims=True)
+        bound = (eps_w + 2.0 ** -8) * (wgt @ abs_vc[:, c]) + 2.0 ** -9 * np.abs(want[:, c])
+        share = max(share, float(np.max(np.abs(got[:, c] - want[:, c]) / np.maximum(bound, 1e-300))))
+    return share, float(np.max(np.abs(got - want))), seconds
+
+
+def time_kv_attention(w, dev, steps, warm):
+    """civic_kv_compressed_attention (Eq. 9) on workload `w`: (result dict, tensors for further checks)."""
+    import torch
+
+    from paper_2605_28115_b200 import civic
+    from paper_2605_28115_b200 import workloads as W
+
+    q, k, v, r = W.kvattn_inputs(w, dev)
+    out = torch.empty_like(q)
+    ws = torch.empty(civic.kv_compressed_attention_workspace_bytes(w.n_img, w.m_e, w.n_heads, w.head_dim, w.s),
+                     dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        civic.civic_kv_compressed_attention(q, k, v, r, w.n_heads, out=out, workspace=ws, device_status=status)
+
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.device(dev).index or 0)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = civic.launch_count()
+    sampler.start()
+    start.record()
+    for _ in range(steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = civic.launch_count() - launches0
+    ms = start.elapsed_time(end) / steps
+    if int(status.item()) != 0:
+        raise SystemExit(f"a wait inside the kernels timed out (status {int(status.item())})")
+    value = w.flops / (ms * 1e-3) / 1e12
+    burst, _, which = measured_tensor_peak()
+    roofline = {"bound": "tensor", "kernel": "civic_kv_compressed_attention (latency-bound at this size)",
+                "achieved": value, "peak": burst, "unit": "TFLOP/s", "frac": value / burst, "peak_source": which,
+                "peak_kind": "burst", "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
+    res = {"workload": w.name, "steps": steps, "us_per_step": ms * 1e3, "value": value, "unit": "TFLOP/s",
+           "gpu_launches": launches, "clocks": clocks, "roofline": roofline}
+    return res, (q, k, v, r, out)
+
+
+def other_workloads(dev, with_oracle):
+    """What the default run measures after its main workload, each with its own clocks and its own
+    comparison against the CPU oracle: the other K/V configurations (roofline fraction of the K/V
+    launch), the small configurations (latency, plain and as a graph), Eq. 8 and Eq. 9."""
+    import gc
+
+    import torch
+
+    from paper_2605_28115_b200 import workloads as W
+
+    out = {}
+    for wl, steps in ((W.C5_HALF, 200), (W.C5_THIRD, 200), (W.C5_QUARTER, 200),
+                      (W.C1, 2000), (W.C2, 2000), (W.C4, 2000)):
+        out[wl.name] = time_other_path_workload(wl, dev, steps, with_oracle)
+        gc.collect()
+        torch.cuda.empty_cache()
+    w = W.AGG_896
+    res, (x0, anchors, z0, mass, _) = time_aggregate(w, dev, 3000, 20)
+    if with_oracle:
+        share, err, _ = aggregate_within_bound(x0, anchors, w.tau, z0, mass)
+        res.update(equals_oracle=share <= 1.0, largest_error_as_share_of_bound=share, largest_abs_error=err,
+                   oracle_sample="image 0 of the batch, element-wise bound derived from the bf16 arithmetic")
+    out[w.name] = res
+    del x0, anchors, z0, mass
+    w = W.KVATTN_896
+    res, (q, k, v, r, o) = time_kv_attention(w, dev, 3000, 20)
+    if with_oracle:
+        share, err, _ = kv_attention_within_bound(q, k, v, r, w.n_heads, o)
+        res.update(equals_oracle=share <= 1.0, largest_error_as_share_of_bound=share, largest_abs_error=err,
+                   oracle_sample="image 0 of the batch, element-wise bound derived from the bf16 arithmetic")
+    out[w.name] = res
+    return out
+
+
 def run_civic(args):
     import torch
     import torch.distributed as dist
@@ -428,7 +751,8 @@ def run_civic(args):
     wl = pick_workload(args)
     st = DeviceState(wl, dev, rank, args.kv_layout, args.merge)
     nbytes = step_bytes(wl, st.merge)
-    default_variant = args.kv_layout == "token_major" and not st.merge
+    merge_on = st.merge
+    default_variant = args.kv_layout == "token_major" and not merge_on
 
     def barrier():
         if world > 1:
@@ -480,17 +804,12 @@ def run_civic(args):
 
     roofline = None
     if kv_ev:
-        kv_ms = [a.elapsed_time(b) for a, b in kv_ev.values()]
-        kv_avg = sum(kv_ms) / len(kv_ms)
-        peak, which = measured_peak()
-        achieved = nbytes["kv"] / (kv_avg * 1e-3) / 1e9
-        kernel = {"token_major": "civic_compact_kv", "head_major": "civic_compact_kv_heads",
-                  "paged": "civic_compact_kv_paged"}[args.kv_layout]
-        roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
-                    "unit": "GB/s", "frac": achieved / peak, "peak_source": which,
-                    "traffic": NCU_DRAM_TRAFFIC_PER_LAUNCH.get(wl.name) if default_variant else None,
-                    "algorithmic_bytes_per_launch": nbytes["kv"], "us_per_launch": kv_avg * 1e3,
-                    "us_per_launch_min": min(kv_ms) * 1e3, "launches_timed": len(kv_ms), "frac_of_8TBps_nominal": achieved / 8000.0}
+        roofline = kv_roofline(wl, nbytes["kv"], [a.elapsed_time(b) for a, b in kv_ev.values()], args.kv_layout,
+                               default_variant)
+        if default_variant:
+            own = contiguous_copy_rate(st)
+            roofline["same_kernel_keeping_every_row_gbs"] = own
+            roofline["frac_of_same_kernel_keeping_every_row"] = roofline["achieved"] / own
 
     # end to end: pinned host inputs -> path -> pinned host results, every step
     e2e = None
@@ -529,21 +848,34 @@ def run_civic(args):
                "results_match_device_path": modes[best]["results_match_device_path"]}
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and default_variant:
+    with_oracle = rank == 0 and world == 1 and not args.no_cpu_baseline and default_variant
+    if with_oracle:
         cpu = cpu_baseline(st)
+        st.step()
+        torch.cuda.synchronize()
+        cpu["gpu_result_equals_oracle"] = path_equals_oracle(st)
+
+    # the other configurations, Eq. 8 and Eq. 9: only beside the default single-GPU measurement
+    others = None
+    if (rank == 0 and world == 1 and default_variant and not args.no_others and graph is None
+            and args.workload == "c3_kv_qwen3vl8b" and not args.layers):
+        import gc
+
+        del st
+        gc.collect()
+        torch.cuda.empty_cache()
+        others = other_workloads(dev, with_oracle)
 
     if rank == 0:
+        variant = {} if default_variant else {"workload": wl.name + (
+            "" if args.kv_layout == "token_major" else "+" + args.kv_layout) + ("+merge" if merge_on else "")}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-                "config": config_of(wl, {"parallelism": f"dp{world}" if world > 1 else "single",
-                                         "cuda_graph": graph is not None,
-                                         "kv_layout": args.kv_layout, "merge": st.merge,
-                                         **({} if default_variant else {"workload": wl.name + (
-                                             "" if args.kv_layout == "token_major" else "+" + args.kv_layout)
-                                             + ("+merge" if st.merge else "")})}),
+                "config": config_of(wl, {"parallelism": parallelism_of(world), **variant}),
+                "variant": {"cuda_graph": graph is not None, "kv_layout": args.kv_layout, "merge": merge_on},
                 "bytes_per_step": nbytes, "gpu_launches": launches, "clocks": clocks,
-                "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+                "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "other_workloads": others}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
@@ -555,7 +887,6 @@ def run_civic(args):
 def run_aggregate(args):
     """`--workload agg_*`: one step = one civic_anchor_aggregate call (anchor preparation, token
     statistics, the two tensor-core contractions, token mass) on a batch of images."""
-    import numpy as np
     import torch
 
     from paper_2605_28115_b200 import build as civic_build
@@ -570,42 +901,9 @@ def run_aggregate(args):
     civic_build.build()
     civic.load()
     w = W.AGG_BY_NAME[args.workload]
-    x0, anchors = W.agg_inputs(w, dev)
-    z0 = torch.empty((w.n_img, w.m_e, w.d_v), dtype=torch.bfloat16, device=dev)
-    mass = torch.empty((w.n_img, w.t_e), dtype=torch.float32, device=dev)
-    ws = torch.empty(civic.anchor_aggregate_workspace_bytes(w.n_img, w.t_e, w.m_e, w.d_v), dtype=torch.uint8, device=dev)
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-
-    def step():
-        civic.civic_anchor_aggregate(x0, anchors, w.tau, z0=z0, token_mass=mass, workspace=ws, device_status=status)
-
     warm = max(args.warmup, 3)
-    for _ in range(warm):
-        step()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(0)
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = civic.launch_count()
-    sampler.start()
-    start.record()
-    for _ in range(args.steps):
-        step()
-    end.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    launches = civic.launch_count() - launches0
-    ms = start.elapsed_time(end) / args.steps
-    if int(status.item()) != 0:
-        raise SystemExit(f"a wait inside the aggregation kernels timed out (status {int(status.item())})")
-    value = w.flops / (ms * 1e-3) / 1e12
-    burst, sustained, which = measured_tensor_peak()
-    timed_s = ms * 1e-3 * args.steps
-    peak = sustained if timed_s > 0.5 else burst  # a long loop runs under the power cap
-    roofline = {"bound": "tensor", "kernel": "civic_anchor_aggregate: five launches, of which the two tcgen05 "
-                "contractions carry all the flops (the other three are HBM-bound helpers and are inside the time)",
-                "achieved": value, "peak": peak, "unit": "TFLOP/s", "frac": value / peak, "peak_source": which,
-                "peak_kind": "sustained" if timed_s > 0.5 else "burst", "frac_of_burst_peak": value / burst,
-                "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
+    res, (x0, anchors, z0, mass, step) = time_aggregate(w, dev, args.steps, warm)
+    ms = res["us_per_step"] * 1e-3
 
     # end to end: pinned host tokens in, compact rows and token mass back out
     e2e = None
@@ -636,35 +934,25 @@ def run_aggregate(args):
 
     cpu = None
     if not args.no_cpu_baseline:
-        from oracle import aggregate as OA
+        share, err, seconds = aggregate_within_bound(x0, anchors, w.tau, z0, mass)
+        cpu = {"value": w.flops / w.n_img / seconds / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": f"the fp64 numpy oracle on ONE of the {w.n_img} images, one run, {seconds * 1e3:.0f} ms per image",
+               "max_abs_difference_to_gpu_result": err, "largest_error_as_share_of_bound": share,
+               "gpu_result_equals_oracle": share <= 1.0}
 
-        x64 = x0[0].double().cpu().numpy()
-        a64 = anchors.double().cpu().numpy()
-        times = []
-        t_begin = time.perf_counter()
-        while len(times) < 2 or (time.perf_counter() - t_begin < 10 and len(times) < 8):
-            t0 = time.perf_counter()
-            z_o, w_o = OA.anchor_aggregate(x64, a64, w.tau)
-            times.append(time.perf_counter() - t0)
-        med = statistics.median(times)
-        err = float(np.max(np.abs(z0[0].float().cpu().numpy() - z_o)))
-        cpu = {"value": w.flops / w.n_img / med / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
-               "sample": f"the fp64 numpy oracle on ONE of the {w.n_img} images, median of {len(times)} runs, "
-                         f"{med * 1e3:.0f} ms per image", "max_abs_difference_to_gpu_result": err}
-
-    line = {"metric": "aggregation_TFLOPs_eq8", "value": value, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
+    line = {"metric": "aggregation_TFLOPs_eq8", "value": res["value"], "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "n_img": w.n_img, "t_e": w.t_e, "m_e": w.m_e, "d_v": w.d_v, "tau": w.tau,
                        "l2": "the tokens (75 MB) and the weights W_A (67 MB) together exceed L2; no flush",
                        "parallelism": "single"},
-            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu}
+            "gpu_launches": res["gpu_launches"], "clocks": res["clocks"], "roofline": res["roofline"], "e2e": e2e,
+            "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
 
 
 def run_kv_attention(args):
     """`--workload kvattn_*`: one step = one civic_kv_compressed_attention call (Eq. 9)."""
-    import numpy as np
     import torch
 
     from paper_2605_28115_b200 import build as civic_build
@@ -679,60 +967,23 @@ def run_kv_attention(args):
     civic_build.build()
     civic.load()
     w = W.KVATTN_BY_NAME[args.workload]
-    q, k, v, r = W.kvattn_inputs(w, dev)
-    out = torch.empty_like(q)
-    ws = torch.empty(civic.kv_compressed_attention_workspace_bytes(w.n_img, w.m_e, w.n_heads, w.head_dim, w.s),
-                     dtype=torch.uint8, device=dev)
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-
-    def step():
-        civic.civic_kv_compressed_attention(q, k, v, r, w.n_heads, out=out, workspace=ws, device_status=status)
-
     warm = max(args.warmup, 3)
-    for _ in range(warm):
-        step()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(0)
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = civic.launch_count()
-    sampler.start()
-    start.record()
-    for _ in range(args.steps):
-        step()
-    end.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    launches = civic.launch_count() - launches0
-    ms = start.elapsed_time(end) / args.steps
-    if int(status.item()) != 0:
-        raise SystemExit(f"a wait inside the kernels timed out (status {int(status.item())})")
-    value = w.flops / (ms * 1e-3) / 1e12
-    burst, sustained, which = measured_tensor_peak()
-    roofline = {"bound": "tensor", "kernel": "civic_kv_compressed_attention (three launches; latency-bound at this size)",
-                "achieved": value, "peak": burst, "unit": "TFLOP/s", "frac": value / burst, "peak_source": which,
-                "peak_kind": "burst", "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}
+    res, (q, k, v, r, out) = time_kv_attention(w, dev, args.steps, warm)
     cpu = None
     if not args.no_cpu_baseline:
-        from oracle import aggregate as OA
-
-        q64, k64, v64 = (a[0].double().cpu().numpy() for a in (q, k, v))
-        r64 = r.double().cpu().numpy()
-        times = []
-        for _ in range(3):
-            t0 = time.perf_counter()
-            want, _, _ = OA.kv_compressed_attention(q64, k64, v64, r64, w.n_heads)
-            times.append(time.perf_counter() - t0)
-        med = statistics.median(times)
-        cpu = {"value": w.flops / w.n_img / med / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
-               "sample": f"the fp64 numpy oracle on ONE of the {w.n_img} images, median of 3 runs, {med * 1e3:.0f} ms",
-               "max_abs_difference_to_gpu_result": float(np.max(np.abs(out[0].float().cpu().numpy() - want)))}
-    line = {"metric": "kv_compressed_attention_TFLOPs_eq9", "value": value, "unit": "TFLOP/s", "n_gpus": 1,
-            "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        share, err, seconds = kv_attention_within_bound(q, k, v, r, w.n_heads, out)
+        cpu = {"value": w.flops / w.n_img / seconds / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": f"the fp64 numpy oracle on ONE of the {w.n_img} images, one run, {seconds * 1e3:.0f} ms",
+               "max_abs_difference_to_gpu_result": err, "largest_error_as_share_of_bound": share,
+               "gpu_result_equals_oracle": share <= 1.0}
+    line = {"metric": "kv_compressed_attention_TFLOPs_eq9", "value": res["value"], "unit": "TFLOP/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": warm, "ms_per_step": res["us_per_step"] * 1e-3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "n_img": w.n_img, "m_e": w.m_e, "n_heads": w.n_heads, "head_dim": w.head_dim,
                        "s": w.s, "l2": "working set (50 MB) smaller than L2 and not flushed: a latency figure",
                        "parallelism": "single"},
-            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "e2e": None, "cpu_baseline": cpu}
+            "gpu_launches": res["gpu_launches"], "clocks": res["clocks"], "roofline": res["roofline"], "e2e": None,
+            "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
 
 
@@ -914,7 +1165,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-            "config": config_of(wl, {"sample": sample_txt}),
+            "config": config_of(wl, {"parallelism": parallelism_of(args.gpus)}),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": sample_txt},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
