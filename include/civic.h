@@ -360,7 +360,7 @@ civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, in
  *                its time limit (the kernels then stop cleanly and the outputs are invalid).
  *                Read it after synchronising the stream.
  * d_v must be a multiple of 64 (CIVIC_ERR_UNSUPPORTED otherwise); t_e and m_e are arbitrary.
- * Inputs must be finite.  Three launches and one 4-byte memset (five launches with token_mass).
+ * Inputs must be finite.  Three launches (five with token_mass); the first one clears the status word.
  */
 civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
                                       int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
@@ -392,8 +392,13 @@ size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_
  * device_status  dev  int32, written: 0, or non-zero if a wait inside a kernel hit its time limit
  *                or a kernel found its shared memory misplaced (the kernels then stop cleanly and
  *                `out` is invalid).  Read it after synchronising the stream.
- * head_dim must be 64 or 128 and s a multiple of 64 up to 256: CIVIC_ERR_UNSUPPORTED otherwise.
- * Three launches and a 4-byte memset.
+ * head_dim: a multiple of 8 up to 128 (64 and 128 are the fast cases; a width such as 72 -- 1152-wide
+ * vision towers with 16 heads -- is handled by storing every head of K_c and V_c with zero
+ * columns up to the next multiple of 16).  s: a multiple of 64 up to 512 (Table 2's "Anchors"
+ * ablation uses 128 and 512).  CIVIC_ERR_UNSUPPORTED otherwise.  Up to 256 anchors a head's K_c
+ * and V_c stay in shared memory while a block walks its query tiles; beyond that one block per SM
+ * holds K_c and, for heads wider than 64, streams V_c from L2 for every query tile.
+ * Three launches; the first one clears the status word.
  */
 civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const void* v, const float* r,
                                              int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
@@ -403,6 +408,39 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
 /* Scratch bytes civic_kv_compressed_attention needs; 0 if the shape is invalid or unsupported. */
 size_t civic_kv_compressed_attention_workspace_bytes(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
                                                      int32_t s);
+
+/*
+ * Constants prepared once.
+ *
+ * Paper: the anchors A of Eq. 8 and the assignment R of Eq. 9 are learned parameters (Section 3.3,
+ * 3.4): at inference they do not change from call to call.  What the two tensor-core calls derive
+ * from them alone -- Q_A = Norm(LN(A)) in bf16 with its row sums; R in bf16 with its column sums --
+ * can therefore be computed once and handed to the `_prepared` variants, which skip that work
+ * (the conversion of R for Eq. 9; the anchor half of the preparation launch for Eq. 8) and give
+ * bit-identical results to the plain calls.
+ *
+ * prepared        dev, caller-owned, 256-byte aligned, at least civic_anchor_prepared_bytes(m_e, d_v)
+ *                 / civic_kv_attention_prepared_bytes(m_e, s) bytes (0 = unsupported shape); written
+ *                 by the `_prepare` call, only read by the `_prepared` calls, opaque to the caller.
+ *                 CIVIC_ERR_WORKSPACE if too small.
+ * The `_prepared` calls take the same arguments as civic_anchor_aggregate /
+ * civic_kv_compressed_attention with `prepared` in the place of `anchors` / `r`; their workspace is
+ * sized by the same *_workspace_bytes functions.  One launch (two for R).
+ */
+size_t civic_anchor_prepared_bytes(int32_t m_e, int32_t d_v);
+civic_status_t civic_anchor_prepare(const float* anchors, int32_t m_e, int32_t d_v, void* prepared,
+                                    size_t prepared_bytes, void* stream);
+civic_status_t civic_anchor_aggregate_prepared(const void* x0, const void* prepared, int32_t n_img, int32_t t_e,
+                                               int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
+                                               void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                               void* stream);
+size_t civic_kv_attention_prepared_bytes(int32_t m_e, int32_t s);
+civic_status_t civic_kv_attention_prepare(const float* r, int32_t m_e, int32_t s, void* prepared, size_t prepared_bytes,
+                                          void* stream);
+civic_status_t civic_kv_compressed_attention_prepared(const void* q, const void* k, const void* v, const void* prepared,
+                                                      int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                                      int32_t s, void* out, void* workspace, size_t workspace_bytes,
+                                                      int32_t* device_status, void* stream);
 
 /*
  * Device-side validation of index arrays.

@@ -32,7 +32,9 @@ EXPORTS = ("civic_select", "civic_select_max_tokens", "civic_reserved_count", "c
            "civic_select_large_static", "civic_select_static_scratch_bytes",
            "civic_anchor_aggregate", "civic_anchor_aggregate_workspace_bytes",
            "civic_kv_compressed_attention", "civic_kv_compressed_attention_workspace_bytes",
-           "civic_set_index_check", "civic_validate_indices", "civic_selftest_bounded_wait")
+           "civic_set_index_check", "civic_validate_indices", "civic_selftest_bounded_wait",
+           "civic_anchor_prepared_bytes", "civic_anchor_prepare", "civic_anchor_aggregate_prepared",
+           "civic_kv_attention_prepared_bytes", "civic_kv_attention_prepare", "civic_kv_compressed_attention_prepared")
 
 INDEX_FAULTS = ("CIVIC_INDEX_OK", "CIVIC_INDEX_OUT_OF_RANGE", "CIVIC_INDEX_NOT_ASCENDING", "CIVIC_INDEX_BAD_PAGE")
 
@@ -117,6 +119,18 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.civic_kv_compressed_attention.restype = ctypes.c_int
     lib.civic_kv_compressed_attention_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.civic_kv_compressed_attention_workspace_bytes.restype = sz
+    lib.civic_anchor_prepared_bytes.argtypes = [i32, i32]
+    lib.civic_anchor_prepared_bytes.restype = sz
+    lib.civic_anchor_prepare.argtypes = [vp, i32, i32, vp, sz, vp]
+    lib.civic_anchor_prepare.restype = ctypes.c_int
+    lib.civic_anchor_aggregate_prepared.argtypes = [vp, vp, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, sz, vp, vp]
+    lib.civic_anchor_aggregate_prepared.restype = ctypes.c_int
+    lib.civic_kv_attention_prepared_bytes.argtypes = [i32, i32]
+    lib.civic_kv_attention_prepared_bytes.restype = sz
+    lib.civic_kv_attention_prepare.argtypes = [vp, i32, i32, vp, sz, vp]
+    lib.civic_kv_attention_prepare.restype = ctypes.c_int
+    lib.civic_kv_compressed_attention_prepared.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    lib.civic_kv_compressed_attention_prepared.restype = ctypes.c_int
     lib.civic_set_index_check.argtypes = [vp]
     lib.civic_set_index_check.restype = ctypes.c_int
     lib.civic_validate_indices.argtypes = [vp, i32, i32, i32, i32, vp, vp]
@@ -593,17 +607,46 @@ def anchor_aggregate_workspace_bytes(n_img: int, t_e: int, m_e: int, d_v: int) -
     return int(load().civic_anchor_aggregate_workspace_bytes(n_img, t_e, m_e, d_v))
 
 
-def civic_anchor_aggregate(x0: torch.Tensor, anchors: torch.Tensor, tau: float,
+@dataclasses.dataclass
+class PreparedAnchors:
+    """Q_A = Norm(LN(A)) in bf16 and its row sums, written once by civic_anchor_prepare."""
+    buffer: torch.Tensor
+    m_e: int
+    d_v: int
+
+
+def civic_anchor_prepare(anchors: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> PreparedAnchors:
+    """anchors fp32 [m_e, d_v] -> the per-model constants of Eq. 8, for civic_anchor_aggregate(x0, prepared, ...)."""
+    if anchors.dim() != 2:
+        raise ValueError("anchors must be [m_e, d_v]")
+    m_e, d_v = anchors.shape
+    need = int(load().civic_anchor_prepared_bytes(m_e, d_v))
+    if need == 0:
+        raise CivicError(5, "civic_anchor_prepared_bytes")
+    buf = torch.empty(need, dtype=torch.uint8, device=_device_of(anchors))
+    with _on_device(_device_of(anchors)):
+        _check(load().civic_anchor_prepare(_dev_ptr(anchors, "anchors", torch.float32), m_e, d_v,
+                                           _dev_ptr(buf, "prepared"), need, _stream_ptr(stream)), "civic_anchor_prepare")
+    return PreparedAnchors(buf, m_e, d_v)
+
+
+def civic_anchor_aggregate(x0: torch.Tensor, anchors, tau: float,
                            z0: Optional[torch.Tensor] = None, token_mass: Optional[torch.Tensor] = None,
                            want_mass: bool = True, workspace: Optional[torch.Tensor] = None,
                            device_status: Optional[torch.Tensor] = None,
                            stream: Optional[torch.cuda.Stream] = None):
-    """Eq. 8: x0 bf16 [n_img, t_e, d_v], anchors fp32 [m_e, d_v] -> (z0 bf16 [n_img, m_e, d_v],
-    token mass fp32 [n_img, t_e] or None, device_status int32 [1]: 0 after a clean run)."""
-    if x0.dim() != 3 or anchors.dim() != 2 or anchors.shape[1] != x0.shape[2]:
-        raise ValueError("x0 must be [n_img, t_e, d_v] and anchors [m_e, d_v]")
+    """Eq. 8: x0 bf16 [n_img, t_e, d_v], anchors fp32 [m_e, d_v] (or PreparedAnchors) ->
+    (z0 bf16 [n_img, m_e, d_v], token mass fp32 [n_img, t_e] or None, device_status int32 [1]: 0 after a clean run)."""
+    prepared = anchors if isinstance(anchors, PreparedAnchors) else None
+    if prepared is not None:
+        if x0.dim() != 3 or prepared.d_v != x0.shape[2]:
+            raise ValueError("x0 must be [n_img, t_e, d_v] with the prepared anchors' d_v")
+        m_e = prepared.m_e
+    else:
+        if x0.dim() != 3 or anchors.dim() != 2 or anchors.shape[1] != x0.shape[2]:
+            raise ValueError("x0 must be [n_img, t_e, d_v] and anchors [m_e, d_v]")
+        m_e = anchors.shape[0]
     n_img, t_e, d_v = x0.shape
-    m_e = anchors.shape[0]
     dev = _device_of(x0)
     if z0 is None:
         z0 = torch.empty((n_img, m_e, d_v), dtype=torch.bfloat16, device=dev)
@@ -618,12 +661,14 @@ def civic_anchor_aggregate(x0: torch.Tensor, anchors: torch.Tensor, tau: float,
                                 dtype=torch.uint8, device=dev)
     if device_status is None:
         device_status = torch.empty((1,), dtype=torch.int32, device=dev)
-    args = (_dev_ptr(x0, "x0", torch.bfloat16), _dev_ptr(anchors, "anchors", torch.float32), n_img, t_e, m_e, d_v,
+    a_ptr = _dev_ptr(prepared.buffer, "prepared") if prepared is not None else _dev_ptr(anchors, "anchors", torch.float32)
+    args = (_dev_ptr(x0, "x0", torch.bfloat16), a_ptr, n_img, t_e, m_e, d_v,
             ctypes.c_float(tau), _dev_ptr(z0, "z0", torch.bfloat16), _dev_ptr(token_mass, "token_mass", torch.float32),
             _dev_ptr(workspace, "workspace", torch.uint8), workspace.numel(),
             _dev_ptr(device_status, "device_status", torch.int32))
+    fn = load().civic_anchor_aggregate_prepared if prepared is not None else load().civic_anchor_aggregate
     with _on_device(dev):
-        _check(load().civic_anchor_aggregate(*args, _stream_ptr(stream)), "civic_anchor_aggregate")
+        _check(fn(*args, _stream_ptr(stream)), "civic_anchor_aggregate")
     return z0, token_mass, device_status
 
 
@@ -631,18 +676,43 @@ def kv_compressed_attention_workspace_bytes(n_img: int, m_e: int, n_heads: int, 
     return int(load().civic_kv_compressed_attention_workspace_bytes(n_img, m_e, n_heads, head_dim, s))
 
 
-def civic_kv_compressed_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, r: torch.Tensor, n_heads: int,
+@dataclasses.dataclass
+class PreparedAssignment:
+    """R in bf16 and its column sums, written once by civic_kv_attention_prepare."""
+    buffer: torch.Tensor
+    m_e: int
+    s: int
+
+
+def civic_kv_attention_prepare(r: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> PreparedAssignment:
+    """r fp32 [m_e, s] -> the per-model constants of Eq. 9, for civic_kv_compressed_attention(q, k, v, prepared, ...)."""
+    if r.dim() != 2:
+        raise ValueError("r must be [m_e, s]")
+    m_e, s = r.shape
+    need = int(load().civic_kv_attention_prepared_bytes(m_e, s))
+    if need == 0:
+        raise CivicError(5, "civic_kv_attention_prepared_bytes")
+    buf = torch.empty(need, dtype=torch.uint8, device=_device_of(r))
+    with _on_device(_device_of(r)):
+        _check(load().civic_kv_attention_prepare(_dev_ptr(r, "r", torch.float32), m_e, s, _dev_ptr(buf, "prepared"), need,
+                                                 _stream_ptr(stream)), "civic_kv_attention_prepare")
+    return PreparedAssignment(buf, m_e, s)
+
+
+def civic_kv_compressed_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, r, n_heads: int,
                                   out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
                                   device_status: Optional[torch.Tensor] = None,
                                   stream: Optional[torch.cuda.Stream] = None):
-    """Eq. 9 for projected q, k, v bf16 [n_img, m_e, n_heads * d] and the assignment r fp32 [m_e, s] ->
-    (attention output bf16 [n_img, m_e, n_heads * d], device_status int32 [1]: 0 after a clean run)."""
-    if q.dim() != 3 or q.shape != k.shape or q.shape != v.shape or r.dim() != 2 or r.shape[0] != q.shape[1]:
+    """Eq. 9 for projected q, k, v bf16 [n_img, m_e, n_heads * d] and the assignment r fp32 [m_e, s] (or a
+    PreparedAssignment) -> (attention output bf16 [n_img, m_e, n_heads * d], device_status int32 [1]: 0 after a clean run)."""
+    prepared = r if isinstance(r, PreparedAssignment) else None
+    r_rows, r_cols = (prepared.m_e, prepared.s) if prepared is not None else (tuple(r.shape) if r.dim() == 2 else (-1, -1))
+    if q.dim() != 3 or q.shape != k.shape or q.shape != v.shape or r_rows != q.shape[1]:
         raise ValueError("q, k, v must be [n_img, m_e, D] and r [m_e, s]")
     n_img, m_e, dim = q.shape
     if dim % n_heads:
         raise ValueError("the feature dimension must be a multiple of n_heads")
-    head_dim, s = dim // n_heads, r.shape[1]
+    head_dim, s = dim // n_heads, r_cols
     dev = _device_of(q)
     if out is None:
         out = torch.empty_like(q)
@@ -653,12 +723,14 @@ def civic_kv_compressed_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Ten
                                 dtype=torch.uint8, device=dev)
     if device_status is None:
         device_status = torch.empty((1,), dtype=torch.int32, device=dev)
+    r_ptr = _dev_ptr(prepared.buffer, "prepared") if prepared is not None else _dev_ptr(r, "r", torch.float32)
     args = (_dev_ptr(q, "q", torch.bfloat16), _dev_ptr(k, "k", torch.bfloat16), _dev_ptr(v, "v", torch.bfloat16),
-            _dev_ptr(r, "r", torch.float32), n_img, m_e, n_heads, head_dim, s, _dev_ptr(out, "out", torch.bfloat16),
+            r_ptr, n_img, m_e, n_heads, head_dim, s, _dev_ptr(out, "out", torch.bfloat16),
             _dev_ptr(workspace, "workspace", torch.uint8), workspace.numel(),
             _dev_ptr(device_status, "device_status", torch.int32))
+    fn = load().civic_kv_compressed_attention_prepared if prepared is not None else load().civic_kv_compressed_attention
     with _on_device(dev):
-        _check(load().civic_kv_compressed_attention(*args, _stream_ptr(stream)), "civic_kv_compressed_attention")
+        _check(fn(*args, _stream_ptr(stream)), "civic_kv_compressed_attention")
     return out, device_status
 
 

@@ -272,13 +272,18 @@ __device__ __forceinline__ float normalise_scale(float ss, int d_v, float ln_eps
     return ss > 0.f ? inv_std / fmaxf(norm, norm_eps) : 0.f;
 }
 
+// Token rows per warp and loads in flight per row: one row and four 16-byte loads per lane measured
+// fastest on B200 (18.3 us for 75 MB; two or four rows per warp 20 .. 29 us, deeper unrolling 22 us).
+constexpr int kPrepRows = 1;
+constexpr int kPrepUnroll = 4;
 __global__ void __launch_bounds__(256) aggregate_prep_kernel(const float* __restrict__ anchors, int m_e,
                                                              const __nv_bfloat16* __restrict__ x, long long n_tokens,
                                                              int d_v, float ln_eps, float norm_eps,
                                                              __nv_bfloat16* __restrict__ q, float* __restrict__ qsum,
-                                                             float2* __restrict__ stats)
+                                                             float2* __restrict__ stats, int* __restrict__ status)
 {
     wait_for_prior_kernels();
+    if (status && blockIdx.x == 0 && threadIdx.x == 0) *status = 0;  // the call's status word starts clean
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp < m_e) {
@@ -300,32 +305,47 @@ __global__ void __launch_bounds__(256) aggregate_prep_kernel(const float* __rest
         if (lane == 0) qsum[warp] = rounded_sum;
         return;
     }
-    const long long tok = warp - m_e;
-    if (tok >= n_tokens) return;
-    // ---- token row (bf16, d_v a multiple of 8): one pass of 16-byte loads; sums are taken
-    // relative to the row's first element so that the variance keeps its accuracy
-    const uint4* row = reinterpret_cast<const uint4*>(x + tok * d_v);
+    // ---- token rows (bf16, d_v a multiple of 8): a warp takes kPrepRows consecutive rows, their
+    // 16-byte loads interleaved; sums are taken relative to the row's first element so that the
+    // variance keeps its accuracy
+    const long long tok0 = (warp - m_e) * kPrepRows;
+    if (tok0 >= n_tokens) return;
     const int vecs = d_v >> 3;
-    const float shift = __bfloat162float(x[tok * d_v]);
-    float s = 0.f, s2 = 0.f;
-#pragma unroll 4
-    for (int v = lane; v < vecs; v += 32) {
-        const uint4 u = __ldg(row + v);
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+    const uint4* row[kPrepRows];
+    float shift[kPrepRows], s[kPrepRows], s2[kPrepRows];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(h[e]);
-            const float a = f.x - shift, b = f.y - shift;
-            s += a + b;
-            s2 += a * a + b * b;
+    for (int r = 0; r < kPrepRows; ++r) {
+        const long long tok = tok0 + r < n_tokens ? tok0 + r : tok0;  // past the end: the first row again, not stored
+        row[r] = reinterpret_cast<const uint4*>(x + tok * d_v);
+        shift[r] = __bfloat162float(x[tok * d_v]);
+        s[r] = 0.f;
+        s2[r] = 0.f;
+    }
+#pragma unroll kPrepUnroll
+    for (int v = lane; v < vecs; v += 32) {
+        uint4 u[kPrepRows];
+#pragma unroll
+        for (int r = 0; r < kPrepRows; ++r) u[r] = __ldg(row[r] + v);
+#pragma unroll
+        for (int r = 0; r < kPrepRows; ++r) {
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[r]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __bfloat1622float2(h[e]);
+                const float a = f.x - shift[r], b = f.y - shift[r];
+                s[r] += a + b;
+                s2[r] += a * a + b * b;
+            }
         }
     }
-    s = warp_sum(s);
-    s2 = warp_sum(s2);
-    if (lane == 0) {
-        const float mean_shifted = s / d_v;
-        const float ss = fmaxf(s2 - s * mean_shifted, 0.f);  // sum (x - mu)^2
-        stats[tok] = make_float2(mean_shifted + shift, normalise_scale(ss, d_v, ln_eps, norm_eps));
+#pragma unroll
+    for (int r = 0; r < kPrepRows; ++r) {
+        const float sum = warp_sum(s[r]), sum2 = warp_sum(s2[r]);
+        if (lane == 0 && tok0 + r < n_tokens) {
+            const float mean_shifted = sum / d_v;
+            const float ss = fmaxf(sum2 - sum * mean_shifted, 0.f);  // sum (x - mu)^2
+            stats[tok0 + r] = make_float2(mean_shifted + shift[r], normalise_scale(ss, d_v, ln_eps, norm_eps));
+        }
     }
 }
 
@@ -664,11 +684,15 @@ struct ValuesOp {
 struct CompressParams {
     const float* colsum_parts;  // [n_parts, s] column sums of the bf16-rounded assignment matrix, by row panel
     int32_t n_parts;
-    __nv_bfloat16* out;    // [n_img, s, d_v]  K_c
-    __nv_bfloat16* out_v;  // [n_img, s, d_v]  V_c
+    __nv_bfloat16* out;    // [n_img, s, out_ld]  K_c
+    __nv_bfloat16* out_v;  // [n_img, s, out_ld]  V_c
     int* error;
     TileGrid grid;         // over 2 n_img "images": K of every image, then V
     int32_t s, m_e, d_v, n_img;
+    // Output layout: the d_v features are heads of head_dim columns; every head is written as
+    // head_ld >= head_dim columns, the extra ones zero (out_ld = d_v / head_dim * head_ld).  The
+    // attention kernel reads whole 16-column K steps, so a 72-wide head is stored 80 wide.
+    int32_t head_dim, head_ld, out_ld;
 };
 
 template <int BN_>
@@ -723,13 +747,15 @@ struct CompressOp {
         const int nh = tl.n0 + half * half_cols;
         const bool second = tl.img >= p.n_img;
         __nv_bfloat16* out = (second ? p.out_v : p.out) +
-                             ((size_t)(second ? tl.img - p.n_img : tl.img) * p.s + (row_ok ? row : 0)) * p.d_v + nh;
+                             ((size_t)(second ? tl.img - p.n_img : tl.img) * p.s + (row_ok ? row : 0)) * p.out_ld;
+        const int pad = p.head_ld - p.head_dim;  // 0 or 8 columns (head_dim is a multiple of 8)
         for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * half_cols, half_cols,
                        [&](const uint32_t (&acc)[32], int c0) {
             if (row_ok) {
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                    if (nh + c0 + q4 * 8 < p.d_v) {
+                    const int f = nh + c0 + q4 * 8;  // first of 8 features: a group never straddles two heads
+                    if (f < p.d_v) {
                         uint32_t w[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
@@ -737,7 +763,11 @@ struct CompressOp {
                                                                            __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv);
                             w[e] = *reinterpret_cast<const uint32_t*>(&h);
                         }
-                        *reinterpret_cast<uint4*>(out + c0 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                        const int head = pad ? f / p.head_dim : 0;
+                        __nv_bfloat16* at = out + f + head * pad;
+                        *reinterpret_cast<uint4*>(at) = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (pad && f - head * p.head_dim == p.head_dim - 8)  // the head's last group: zeros behind it
+                            *reinterpret_cast<uint4*>(at + 8) = make_uint4(0u, 0u, 0u, 0u);
                     }
                 }
             }
@@ -904,27 +934,34 @@ __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned long
 }
 
 // Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m], in two deterministic steps.
-//   token_mass_partial_kernel  a block reads a panel of kMassPanel whole rows of P (contiguous
-//                              in memory, so DRAM pages are used in full) and writes the panel's
-//                              weighted column sums;
+//   token_mass_partial_kernel  a block takes a panel of kMassPanel rows of P over a slab of 256 token
+//                              columns (512 contiguous bytes per row); its eight warps take every
+//                              eighth row, and their sums are added in warp order through shared
+//                              memory;
 //   token_mass_reduce_kernel   adds the panels' sums in a fixed order.
-// (One block per column slab reading all rows at an 8 KB stride measured 2.7 TB/s.)
-constexpr int kMassPanel = 16;
-__global__ void __launch_bounds__(256) token_mass_partial_kernel(const __nv_bfloat16* __restrict__ p,
-                                                                 const float* __restrict__ inv_l, int m_e, int t_e,
-                                                                 int t_ld, int n_panels, float* __restrict__ partial)
+// Measured on 8 x 1024 x 4096 weights (us, partial + reduce): panels of 16 rows over all columns,
+// thread per 8 columns: 14.8 + 4.6; the same over slabs of 1024 columns: 12.1 + 9.5 (the reduction
+// pays for 64 panels); panels of 64 rows: 21.0 + 3.6 (too few, too long threads).
+constexpr int kMassPanel = 128;
+constexpr int kMassWarps = 8;
+__global__ void __launch_bounds__(kMassWarps * 32) token_mass_partial_kernel(const __nv_bfloat16* __restrict__ p,
+                                                                             const float* __restrict__ inv_l, int m_e,
+                                                                             int t_e, int t_ld, int n_panels,
+                                                                             float* __restrict__ partial)
 {
+    __shared__ float4 sums[kMassWarps][32][2];
     wait_for_prior_kernels();
-    const int panel = blockIdx.x, img = blockIdx.y;
+    const int panel = blockIdx.x, img = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m_begin = panel * kMassPanel, m_end = min(m_begin + kMassPanel, m_e);
     const float* il = inv_l + (size_t)img * m_e;
-    float* out = partial + ((size_t)img * n_panels + panel) * t_ld;
-    // thread = 8 consecutive token columns (one 16-byte load per row); t_ld is a multiple of 8
-    for (int c = threadIdx.x * 8; c < t_ld; c += blockDim.x * 8) {
-        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        const __nv_bfloat16* col = p + ((size_t)img * m_e + m_begin) * t_ld + c;
+    // lane = 8 consecutive token columns (one 16-byte load per row); t_ld is a multiple of 8
+    const int c = blockIdx.y * 256 + lane * 8;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (c < t_ld) {
+        const __nv_bfloat16* col = p + ((size_t)img * m_e + m_begin + warp) * t_ld + c;
 #pragma unroll 8
-        for (int m = m_begin; m < m_end; ++m, col += t_ld) {
+        for (int m = m_begin + warp; m < m_end; m += kMassWarps, col += (size_t)kMassWarps * t_ld) {
             const uint4 u = __ldg(reinterpret_cast<const uint4*>(col));
             const float w = __ldg(il + m);
             const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
@@ -935,8 +972,20 @@ __global__ void __launch_bounds__(256) token_mass_partial_kernel(const __nv_bflo
                 acc[2 * e + 1] += f.y * w;
             }
         }
-        *reinterpret_cast<float4*>(out + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        *reinterpret_cast<float4*>(out + c + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    }
+    sums[warp][lane][0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    sums[warp][lane][1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    __syncthreads();
+    if (threadIdx.x < 64) {  // thread = 4 of the slab's 256 columns: the warps' sums in warp order
+        const int l = threadIdx.x >> 1, half = threadIdx.x & 1;
+        float4 t = sums[0][l][half];
+#pragma unroll
+        for (int w = 1; w < kMassWarps; ++w) {
+            const float4 v = sums[w][l][half];
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        const int col = blockIdx.y * 256 + l * 8 + half * 4;
+        if (col < t_ld) *reinterpret_cast<float4*>(partial + ((size_t)img * n_panels + panel) * t_ld + col) = t;
     }
 }
 

@@ -22,7 +22,7 @@ std::atomic<uint64_t> g_launches{0};
 std::atomic<int> g_programmatic{1};
 
 bool programmatic() { return g_programmatic.load(std::memory_order_relaxed) != 0; }
-thread_local char g_cuda_error[256] = "";
+thread_local char g_cuda_error[512] = "";
 
 // Fault record the calling thread's compaction calls validate their index arrays into (device
 // int32[4]); NULL = the unchecked kernels.
@@ -449,15 +449,18 @@ civic_status_t tensor_map_encoder(EncodeTiledFn* out)
 }
 
 // bf16 tensor of rank 2 or 3, innermost dimension first; boxes of 64 elements (128 B, swizzled).
+// box_cols = 64 gives the swizzled 128-byte rows the MMA descriptors expect; any other width (a
+// multiple of 8 columns below 64) gives a plain, unswizzled box (used to store a head's last columns).
 civic_status_t make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                        const uint64_t* strides_bytes, uint32_t box_rows)
+                        const uint64_t* strides_bytes, uint32_t box_rows, uint32_t box_cols = 64)
 {
     cuuint64_t gdim[3] = {dims[0], dims[1], rank == 3 ? dims[2] : 1};
     cuuint64_t gstr[2] = {strides_bytes[0], rank == 3 ? strides_bytes[1] : 0};
-    cuuint32_t box[3] = {64, box_rows, 1};
+    cuuint32_t box[3] = {box_cols, box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
-                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_error, sizeof g_cuda_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -470,6 +473,7 @@ struct AggPlan {
     int32_t t_ld, n_tiles_t, values_bn;
     int32_t n_panels;
     size_t q_off, qsum_off, stats_off, p_off, lpart_off, invl_off, mass_off, total;
+    size_t prepared_total;  // Q_A in bf16 | its row sums: what civic_anchor_prepare writes
 };
 
 civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d_v, AggPlan& pl)
@@ -486,6 +490,7 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
     auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
     pl.q_off = take((size_t)m_e * d_v * 2);
     pl.qsum_off = take((size_t)m_e * 4);
+    pl.prepared_total = off;
     pl.stats_off = take((size_t)n_img * t_e * 8);
     pl.p_off = take((size_t)n_img * m_e * pl.t_ld * 2);
     pl.lpart_off = take((size_t)n_img * m_e * 2 * pl.n_tiles_t * 4);  // two column halves per token tile
@@ -657,26 +662,54 @@ size_t civic_anchor_aggregate_workspace_bytes(int32_t n_img, int32_t t_e, int32_
     return plan_aggregate(n_img, t_e, m_e, d_v, pl) == CIVIC_OK ? pl.total : 0;
 }
 
-civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
-                                      int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
-                                      void* workspace, size_t workspace_bytes, int32_t* device_status,
-                                      void* stream_)
+size_t civic_anchor_prepared_bytes(int32_t m_e, int32_t d_v)
+{
+    AggPlan pl;
+    return plan_aggregate(1, 1, m_e, d_v, pl) == CIVIC_OK ? pl.prepared_total : 0;
+}
+
+civic_status_t civic_anchor_prepare(const float* anchors, int32_t m_e, int32_t d_v, void* prepared,
+                                    size_t prepared_bytes, void* stream)
+{
+    AggPlan pl;
+    const civic_status_t st = plan_aggregate(1, 1, m_e, d_v, pl);
+    if (st != CIVIC_OK) return st;
+    if (!anchors || !prepared) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(anchors, 4) || !aligned(prepared, 256)) return CIVIC_ERR_ALIGNMENT;
+    if (prepared_bytes < pl.prepared_total) return CIVIC_ERR_WORKSPACE;
+    if (overlaps(anchors, (size_t)m_e * d_v * 4, prepared, pl.prepared_total)) return CIVIC_ERR_INVALID_ARG;
+    char* prep = (char*)prepared;
+    CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::aggregate_prep_kernel, (unsigned)((m_e + 7) / 8), 256u, 0,
+                                 (cudaStream_t)stream, anchors, m_e, (const __nv_bfloat16*)nullptr, 0LL, d_v, 1e-5f,
+                                 1e-12f, (__nv_bfloat16*)(prep + pl.q_off), (float*)(prep + pl.qsum_off),
+                                 (float2*)nullptr, (int*)nullptr));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CIVIC_OK;
+}
+
+// Eq. 8 with the anchors either raw (`anchors`, normalised here on every call) or prepared once
+// (`prepared`, written by civic_anchor_prepare).
+static civic_status_t aggregate_impl(const void* x0, const float* anchors, const void* prepared, int32_t n_img,
+                                     int32_t t_e, int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
+                                     void* workspace, size_t workspace_bytes, int32_t* device_status, void* stream_)
 {
     AggPlan pl;
     const civic_status_t st = plan_aggregate(n_img, t_e, m_e, d_v, pl);
     if (st != CIVIC_OK) return st;
     if (!(tau >= 0.025f) || !(tau <= 1e30f)) return CIVIC_ERR_UNSUPPORTED;  // also rejects NaN
     if (n_img == 0) return CIVIC_OK;
-    if (!x0 || !anchors || !z0 || !device_status) return CIVIC_ERR_INVALID_ARG;
-    if (!aligned(x0, 16) || !aligned(z0, 16) || !aligned(anchors, 4) || !aligned(token_mass, 4) ||
-        !aligned(device_status, 4))
+    if (!x0 || (!anchors && !prepared) || !z0 || !device_status) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(x0, 16) || !aligned(z0, 16) || !aligned(anchors, 4) || !aligned(prepared, 256) ||
+        !aligned(token_mass, 4) || !aligned(device_status, 4))
         return CIVIC_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < pl.total) return CIVIC_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return CIVIC_ERR_ALIGNMENT;
     const size_t x_bytes = (size_t)n_img * t_e * d_v * 2, z_bytes = (size_t)n_img * m_e * d_v * 2;
-    if (overlaps(z0, z_bytes, x0, x_bytes) || overlaps(z0, z_bytes, anchors, (size_t)m_e * d_v * 4) ||
+    const void* a_any = anchors ? (const void*)anchors : prepared;
+    const size_t a_bytes = anchors ? (size_t)m_e * d_v * 4 : pl.prepared_total;
+    if (overlaps(z0, z_bytes, x0, x_bytes) || overlaps(z0, z_bytes, a_any, a_bytes) ||
         overlaps(workspace, pl.total, x0, x_bytes) || overlaps(workspace, pl.total, z0, z_bytes) ||
-        overlaps(workspace, pl.total, anchors, (size_t)m_e * d_v * 4) ||
+        overlaps(workspace, pl.total, a_any, a_bytes) ||
         overlaps(token_mass, (size_t)n_img * t_e * 4, z0, z_bytes) ||
         overlaps(token_mass, (size_t)n_img * t_e * 4, workspace, pl.total) ||
         overlaps(device_status, 4, workspace, pl.total) || overlaps(device_status, 4, z0, z_bytes))
@@ -684,8 +717,9 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
 
     cudaStream_t stream = (cudaStream_t)stream_;
     char* ws = (char*)workspace;
-    __nv_bfloat16* q = (__nv_bfloat16*)(ws + pl.q_off);
-    float* qsum = (float*)(ws + pl.qsum_off);
+    char* prep = prepared ? (char*)const_cast<void*>(prepared) : ws;
+    __nv_bfloat16* q = (__nv_bfloat16*)(prep + pl.q_off);
+    float* qsum = (float*)(prep + pl.qsum_off);
     float2* stats = (float2*)(ws + pl.stats_off);
     __nv_bfloat16* p = (__nv_bfloat16*)(ws + pl.p_off);
     float* lpart = (float*)(ws + pl.lpart_off);
@@ -714,11 +748,12 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     }
 
     const bool pdl = programmatic();
-    CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
     const long long n_tokens = (long long)n_img * t_e;
-    CIVIC_CUDA_TRY(civic::launch(pdl, civic::aggregate_prep_kernel, (unsigned)((m_e + n_tokens + 7) / 8), 256u, 0,
-                                 stream, anchors, m_e, (const __nv_bfloat16*)x0, n_tokens, d_v, 1e-5f, 1e-12f, q, qsum,
-                                 stats));
+    const int32_t prep_anchors = prepared ? 0 : m_e;  // prepared anchors: the launch takes the tokens only
+    const long long prep_warps = prep_anchors + (n_tokens + civic::kPrepRows - 1) / civic::kPrepRows;
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::aggregate_prep_kernel, (unsigned)((prep_warps + 7) / 8), 256u, 0,
+                                 stream, anchors, prep_anchors, (const __nv_bfloat16*)x0, n_tokens, d_v, 1e-5f, 1e-12f, q,
+                                 qsum, stats, (int*)device_status));  // also clears the status word
 
     const int32_t m_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
     civic::ScoresParams sp;
@@ -747,9 +782,10 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     int n_launched = 3;
     if (token_mass) {
         float* partial = (float*)(ws + pl.mass_off);
-        CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_partial_kernel, dim3((unsigned)pl.n_panels, (unsigned)n_img),
-                                     256u, 0, stream, (const __nv_bfloat16*)p, (const float*)inv_l, m_e, t_e, pl.t_ld,
-                                     pl.n_panels, partial));
+        CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_partial_kernel,
+                                     dim3((unsigned)pl.n_panels, (unsigned)((pl.t_ld + 255) / 256), (unsigned)n_img),
+                                     (unsigned)(civic::kMassWarps * 32), 0, stream, (const __nv_bfloat16*)p,
+                                     (const float*)inv_l, m_e, t_e, pl.t_ld, pl.n_panels, partial));
         CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_reduce_kernel, dim3((unsigned)((t_e + 63) / 64), (unsigned)n_img),
                                      64u, 0, stream, (const float*)partial, t_e, pl.t_ld, pl.n_panels, token_mass));
         n_launched += 2;
@@ -758,12 +794,35 @@ civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int3
     return CIVIC_OK;
 }
 
+civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
+                                      int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
+                                      void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                      void* stream)
+{
+    if (!anchors && n_img > 0) return CIVIC_ERR_INVALID_ARG;
+    return aggregate_impl(x0, anchors, nullptr, n_img, t_e, m_e, d_v, tau, z0, token_mass, workspace, workspace_bytes,
+                          device_status, stream);
+}
+
+civic_status_t civic_anchor_aggregate_prepared(const void* x0, const void* prepared, int32_t n_img, int32_t t_e,
+                                               int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
+                                               void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                               void* stream)
+{
+    if (!prepared && n_img > 0) return CIVIC_ERR_INVALID_ARG;
+    return aggregate_impl(x0, nullptr, prepared, n_img, t_e, m_e, d_v, tau, z0, token_mass, workspace, workspace_bytes,
+                          device_status, stream);
+}
+
 // ---- KV-compressed visual attention (Eq. 9) -------------------------------------------------
 
 struct KvAttnPlan {
     int32_t dim, compress_bn;
+    int32_t d_pad, dim_ld;      // a head's columns in K_c / V_c (zero padded to a multiple of 16), all heads'
+    int32_t q_slots, v_stream;  // shared-memory plan of the attention kernel
     int32_t n_parts;
     size_t r16_off, colsum_off, partial_off, kc_off, vc_off, total, attn_smem;
+    size_t prepared_total;      // R in bf16 | column sums | panel sums: what civic_kv_attention_prepare writes
 };
 
 // Query tiles per block of the attention kernel: the split that needs the fewest rounds of
@@ -786,13 +845,27 @@ static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_he
                                         KvAttnPlan& pl)
 {
     if (n_img < 0 || m_e < 1 || n_heads < 1 || head_dim < 1 || s < 1) return CIVIC_ERR_INVALID_ARG;
-    if ((head_dim != 64 && head_dim != 128) || s % 64 || s > 256 || n_img > 65535 || n_heads > 65535)
+    if (head_dim % 8 || head_dim > 128 || s % 64 || s > 512 || n_img > 65535 || n_heads > 65535)
         return CIVIC_ERR_UNSUPPORTED;
     const int64_t dim = (int64_t)n_heads * head_dim;
     if (dim > (1 << 20)) return CIVIC_ERR_UNSUPPORTED;
     pl.dim = (int32_t)dim;
-    pl.attn_smem = civic::attn_smem_bytes(head_dim, s);
-    if (pl.attn_smem > kMaxDynamicSmem) return CIVIC_ERR_UNSUPPORTED;
+    pl.d_pad = (head_dim + 15) / 16 * 16;
+    pl.dim_ld = n_heads * pl.d_pad;
+    // shared memory: everything resident with two Q tiles in flight if that fits; else one Q tile;
+    // else V_c streamed through two slots of 64 anchors
+    const int tries[3][2] = {{2, 0}, {1, 0}, {1, 1}};
+    pl.attn_smem = 0;
+    for (const auto& t : tries) {
+        const size_t bytes = civic::attn_smem_bytes(pl.d_pad, s, t[0], t[1]);
+        if (bytes <= kMaxDynamicSmem) {
+            pl.q_slots = t[0];
+            pl.v_stream = t[1];
+            pl.attn_smem = bytes;
+            break;
+        }
+    }
+    if (pl.attn_smem == 0) return CIVIC_ERR_UNSUPPORTED;
     pl.compress_bn = dim % 256 == 0 ? 256 : (dim % 192 == 0 ? 192 : 128);
     size_t off = 0;
     auto take = [&off](size_t bytes) { const size_t at = off; off += round_up(bytes, 256); return at; };
@@ -800,81 +873,98 @@ static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_he
     pl.colsum_off = take((size_t)s * 4);
     pl.n_parts = (m_e + civic::kAssignRows - 1) / civic::kAssignRows;
     pl.partial_off = take((size_t)pl.n_parts * s * 4);
-    pl.kc_off = take((size_t)n_img * s * dim * 2);
-    pl.vc_off = take((size_t)n_img * s * dim * 2);
+    pl.prepared_total = off;
+    pl.kc_off = take((size_t)n_img * s * pl.dim_ld * 2);
+    pl.vc_off = take((size_t)n_img * s * pl.dim_ld * 2);
     pl.total = off;
     return CIVIC_OK;
 }
 
-size_t civic_kv_compressed_attention_workspace_bytes(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
-                                                     int32_t s)
+// R -> bf16 and its column sums into `prep` (laid out as the head of the plan's workspace).
+// `reduce`: also add the panels' sums up (one more small launch), for a result that is kept.
+static civic_status_t launch_assign_prepare(const float* r, int32_t m_e, int32_t s, const KvAttnPlan& pl, char* prep,
+                                            bool reduce, int32_t* status_to_clear, cudaStream_t stream)
 {
-    KvAttnPlan pl;
-    return plan_kv_attention(n_img, m_e, n_heads, head_dim, s, pl) == CIVIC_OK ? pl.total : 0;
+    const bool pdl = programmatic();
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::assign_convert_kernel, (unsigned)pl.n_parts, (unsigned)s, 0, stream, r, m_e,
+                                 s, (__nv_bfloat16*)(prep + pl.r16_off), (float*)(prep + pl.partial_off),
+                                 (int*)status_to_clear));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (reduce) {
+        CIVIC_CUDA_TRY(civic::launch(pdl, civic::assign_colsum_kernel, (unsigned)((s + 127) / 128), 128u, 0, stream,
+                                     (const float*)(prep + pl.partial_off), pl.n_parts, s, (float*)(prep + pl.colsum_off)));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    return CIVIC_OK;
 }
 
-civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const void* v, const float* r,
-                                             int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
-                                             int32_t s, void* out, void* workspace, size_t workspace_bytes,
-                                             int32_t* device_status, void* stream_)
+// The compression GEMM and the attention kernel; r16 / colsum come from the caller's prepared
+// buffer or were just written into the workspace (then colsum_parts holds n_parts panel sums).
+static civic_status_t kv_attention_impl(const void* q, const void* k, const void* v, const float* r, const void* prepared,
+                                        int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim, int32_t s,
+                                        void* out, void* workspace, size_t workspace_bytes, int32_t* device_status,
+                                        void* stream_)
 {
     KvAttnPlan pl;
     const civic_status_t st = plan_kv_attention(n_img, m_e, n_heads, head_dim, s, pl);
     if (st != CIVIC_OK) return st;
     if (n_img == 0) return CIVIC_OK;
-    if (!q || !k || !v || !r || !out || !device_status) return CIVIC_ERR_INVALID_ARG;
+    if (!q || !k || !v || (!r && !prepared) || !out || !device_status) return CIVIC_ERR_INVALID_ARG;
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16) || !aligned(r, 4) ||
-        !aligned(device_status, 4))
+        !aligned(prepared, 256) || !aligned(device_status, 4))
         return CIVIC_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < pl.total) return CIVIC_ERR_WORKSPACE;
     if (!aligned(workspace, 256)) return CIVIC_ERR_ALIGNMENT;
     const size_t x_bytes = (size_t)n_img * m_e * pl.dim * 2;
+    const size_t r_bytes = r ? (size_t)m_e * s * 4 : pl.prepared_total;
+    const void* r_any = r ? (const void*)r : prepared;
     if (overlaps(out, x_bytes, q, x_bytes) || overlaps(out, x_bytes, k, x_bytes) || overlaps(out, x_bytes, v, x_bytes) ||
-        overlaps(out, x_bytes, r, (size_t)m_e * s * 4) || overlaps(workspace, pl.total, out, x_bytes) ||
+        overlaps(out, x_bytes, r_any, r_bytes) || overlaps(workspace, pl.total, out, x_bytes) ||
         overlaps(workspace, pl.total, q, x_bytes) || overlaps(workspace, pl.total, k, x_bytes) ||
-        overlaps(workspace, pl.total, v, x_bytes) || overlaps(workspace, pl.total, r, (size_t)m_e * s * 4) ||
+        overlaps(workspace, pl.total, v, x_bytes) || overlaps(workspace, pl.total, r_any, r_bytes) ||
         overlaps(device_status, 4, workspace, pl.total) || overlaps(device_status, 4, out, x_bytes))
         return CIVIC_ERR_INVALID_ARG;
 
     cudaStream_t stream = (cudaStream_t)stream_;
     char* ws = (char*)workspace;
-    __nv_bfloat16* r16 = (__nv_bfloat16*)(ws + pl.r16_off);
+    const char* prep = prepared ? (const char*)prepared : ws;
+    const __nv_bfloat16* r16 = (const __nv_bfloat16*)(prep + pl.r16_off);
     __nv_bfloat16* kc = (__nv_bfloat16*)(ws + pl.kc_off);
     __nv_bfloat16* vc = (__nv_bfloat16*)(ws + pl.vc_off);
 
     EncodeTiledFn enc = nullptr;
     civic_status_t ms = tensor_map_encoder(&enc);
     if (ms != CIVIC_OK) return ms;
-    CUtensorMap map_r, map_k_in, map_v_in, map_q, map_kc, map_vc;
+    CUtensorMap map_r, map_k_in, map_v_in, map_q, map_kc, map_vc, map_o, map_o_tail;
     {
         const uint64_t dims[2] = {(uint64_t)s, (uint64_t)m_e}, str[1] = {(uint64_t)s * 2};
         if ((ms = make_map(enc, &map_r, r16, 2, dims, str, 64)) != CIVIC_OK) return ms;
     }
+    const int32_t tail = head_dim % 64;
     {
         const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
         const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
         if ((ms = make_map(enc, &map_k_in, k, 3, dims, str, 64)) != CIVIC_OK) return ms;
         if ((ms = make_map(enc, &map_v_in, v, 3, dims, str, 64)) != CIVIC_OK) return ms;
         if ((ms = make_map(enc, &map_q, q, 3, dims, str, civic::kAggBM)) != CIVIC_OK) return ms;
+        // output boxes of 32 rows (one softmax warp's share of a tile): 64 columns wide, and the
+        // head's last columns where its width is not a multiple of 64
+        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_o_tail, out, 3, dims, str, 32, tail ? (uint32_t)tail : 64u)) != CIVIC_OK) return ms;
     }
     {
-        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)s, (uint64_t)n_img};
-        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)s * pl.dim * 2};
+        const uint64_t dims[3] = {(uint64_t)pl.dim_ld, (uint64_t)s, (uint64_t)n_img};
+        const uint64_t str[2] = {(uint64_t)pl.dim_ld * 2, (uint64_t)s * pl.dim_ld * 2};
         if ((ms = make_map(enc, &map_kc, kc, 3, dims, str, 64)) != CIVIC_OK) return ms;
         if ((ms = make_map(enc, &map_vc, vc, 3, dims, str, 64)) != CIVIC_OK) return ms;
     }
 
-    const float scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
     const int32_t q_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
-    CUtensorMap map_o;  // boxes of 32 rows x 64 features: one softmax warp's share of a tile
-    {
-        const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
-        const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
-        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32)) != CIVIC_OK) return ms;
-    }
     civic::AttnParams ap;
-    ap.error = device_status; ap.m_e = m_e; ap.d = head_dim; ap.s = s;
-    ap.scale_log2e = scale_log2e;
+    ap.error = device_status; ap.m_e = m_e; ap.s = s;
+    ap.d = head_dim; ap.d_pad = pl.d_pad; ap.d_ld = pl.d_pad;
+    ap.q_slots = pl.q_slots; ap.v_stream = pl.v_stream;
+    ap.scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
     // Once per device: the kernel may use all of an SM's memory as shared memory (so that two blocks
     // of 113 KB can be resident), and the figures that decide how many blocks fit on an SM
     // together.  (The runtime's occupancy query answers 1 for this kernel whatever its shared
@@ -899,23 +989,29 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
         info.regs_per_thread = fattr.numRegs;
         info.ready.store(1, std::memory_order_release);
     }
-    const int smem_per_sm = info.smem_per_sm, reserved = info.reserved, regs_per_sm = info.regs_per_sm;
     const int regs_per_block = ((info.regs_per_thread + 7) / 8 * 8) * civic::kAttnThreads;
-    int blocks_per_sm = (int)((size_t)smem_per_sm / (pl.attn_smem + (size_t)reserved));
-    blocks_per_sm = std::min(blocks_per_sm, regs_per_sm / std::max(regs_per_block, 1));
+    int blocks_per_sm = (int)((size_t)info.smem_per_sm / (pl.attn_smem + (size_t)info.reserved));
+    blocks_per_sm = std::min(blocks_per_sm, info.regs_per_sm / std::max(regs_per_block, 1));
     blocks_per_sm = std::min(blocks_per_sm, 2048 / civic::kAttnThreads);
-    blocks_per_sm = std::min(blocks_per_sm, (int)(512 / civic::attn_tmem_cols(head_dim, s)));
+    blocks_per_sm = std::min(blocks_per_sm, (int)(512 / civic::attn_tmem_cols(pl.d_pad, s)));
     ap.tiles_per_block = attention_tiles_per_block(q_tiles, (int64_t)n_heads * n_img, blocks_per_sm);
 
     // everything that can fail on the host has happened: from here on work is enqueued
     const bool pdl = programmatic();
-    CIVIC_CUDA_TRY(cudaMemsetAsync(device_status, 0, 4, stream));
-    float* partial = (float*)(ws + pl.partial_off);
-    CIVIC_CUDA_TRY(civic::launch(pdl, civic::assign_convert_kernel, (unsigned)pl.n_parts, (unsigned)s, 0, stream, r, m_e,
-                                 s, r16, partial));
-
     civic::CompressParams cp;
-    cp.colsum_parts = partial; cp.n_parts = pl.n_parts; cp.error = device_status; cp.s = s; cp.m_e = m_e; cp.d_v = pl.dim;
+    if (prepared) {  // no small kernel in front: a one-thread kernel clears the status word
+        CIVIC_CUDA_TRY(civic::launch(pdl, civic::clear_status_kernel, 1u, 32u, 0, stream, (int*)device_status));
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        cp.colsum_parts = (const float*)(prep + pl.colsum_off);
+        cp.n_parts = 1;
+    } else {
+        const civic_status_t as = launch_assign_prepare(r, m_e, s, pl, ws, false, device_status, stream);
+        if (as != CIVIC_OK) return as;
+        cp.colsum_parts = (const float*)(ws + pl.partial_off);
+        cp.n_parts = pl.n_parts;
+    }
+    cp.error = device_status; cp.s = s; cp.m_e = m_e; cp.d_v = pl.dim;
+    cp.head_dim = head_dim; cp.head_ld = pl.d_pad; cp.out_ld = pl.dim_ld;
     const int32_t s_tiles = (s + civic::kAggBM - 1) / civic::kAggBM;
     const int32_t f_tiles = (pl.dim + pl.compress_bn - 1) / pl.compress_bn;
     // K and V in one launch: the tile grid runs over 2 n_img "images"
@@ -928,13 +1024,59 @@ civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const
         else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
         if (gs != CIVIC_OK) return gs;
     }
-
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel,
                                  dim3((unsigned)((q_tiles + ap.tiles_per_block - 1) / ap.tiles_per_block),
                                       (unsigned)n_heads, (unsigned)n_img),
-                                 (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, map_o, ap));
-    g_launches.fetch_add(3, std::memory_order_relaxed);
+                                 (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, map_o,
+                                 map_o_tail, ap));
+    g_launches.fetch_add(2, std::memory_order_relaxed);
     return CIVIC_OK;
+}
+
+size_t civic_kv_compressed_attention_workspace_bytes(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                                     int32_t s)
+{
+    KvAttnPlan pl;
+    return plan_kv_attention(n_img, m_e, n_heads, head_dim, s, pl) == CIVIC_OK ? pl.total : 0;
+}
+
+civic_status_t civic_kv_compressed_attention(const void* q, const void* k, const void* v, const float* r,
+                                             int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                             int32_t s, void* out, void* workspace, size_t workspace_bytes,
+                                             int32_t* device_status, void* stream)
+{
+    if (!r && n_img > 0) return CIVIC_ERR_INVALID_ARG;
+    return kv_attention_impl(q, k, v, r, nullptr, n_img, m_e, n_heads, head_dim, s, out, workspace, workspace_bytes,
+                             device_status, stream);
+}
+
+size_t civic_kv_attention_prepared_bytes(int32_t m_e, int32_t s)
+{
+    KvAttnPlan pl;
+    return plan_kv_attention(1, m_e, 1, 64, s, pl) == CIVIC_OK ? pl.prepared_total : 0;
+}
+
+civic_status_t civic_kv_attention_prepare(const float* r, int32_t m_e, int32_t s, void* prepared, size_t prepared_bytes,
+                                          void* stream)
+{
+    KvAttnPlan pl;
+    const civic_status_t st = plan_kv_attention(1, m_e, 1, 64, s, pl);
+    if (st != CIVIC_OK) return st;
+    if (!r || !prepared) return CIVIC_ERR_INVALID_ARG;
+    if (!aligned(r, 4) || !aligned(prepared, 256)) return CIVIC_ERR_ALIGNMENT;
+    if (prepared_bytes < pl.prepared_total) return CIVIC_ERR_WORKSPACE;
+    if (overlaps(r, (size_t)m_e * s * 4, prepared, pl.prepared_total)) return CIVIC_ERR_INVALID_ARG;
+    return launch_assign_prepare(r, m_e, s, pl, (char*)prepared, true, nullptr, (cudaStream_t)stream);
+}
+
+civic_status_t civic_kv_compressed_attention_prepared(const void* q, const void* k, const void* v, const void* prepared,
+                                                      int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim,
+                                                      int32_t s, void* out, void* workspace, size_t workspace_bytes,
+                                                      int32_t* device_status, void* stream)
+{
+    if (!prepared && n_img > 0) return CIVIC_ERR_INVALID_ARG;
+    return kv_attention_impl(q, k, v, nullptr, prepared, n_img, m_e, n_heads, head_dim, s, out, workspace,
+                             workspace_bytes, device_status, stream);
 }
 
 civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civic_select_desc_t* descs,

@@ -339,7 +339,10 @@ class KvAttnWorkload:
 
 # 8 images, 1024 compact tokens, 16 heads of 64 (vision width 1024), 256 memory anchors
 KVATTN_896 = KvAttnWorkload("kvattn_batch8_896", 8, 1024, 16, 64, 256)
-KVATTN_BY_NAME = {w.name: w for w in (KVATTN_896,)}
+# the same layer on a 1152-wide tower (16 heads of 72), and with Table 2's 512 memory anchors
+KVATTN_896_W1152 = KvAttnWorkload("kvattn_batch8_896_w1152", 8, 1024, 16, 72, 256)
+KVATTN_896_S512 = KvAttnWorkload("kvattn_batch8_896_s512", 8, 1024, 16, 64, 512)
+KVATTN_BY_NAME = {w.name: w for w in (KVATTN_896, KVATTN_896_W1152, KVATTN_896_S512)}
 
 
 def kvattn_inputs(w: KvAttnWorkload, device="cpu"):

@@ -248,15 +248,47 @@ def test_kv_compressed_attention_validation(lib):
         out=0x500000, ws=0x1000000, ws_bytes=1 << 30, status=0x600000: \
         lib.civic_kv_compressed_attention(q, k, v, r, n_img, m_e, heads, d, s, out, ws, ws_bytes, status, None)
     before = lib.civic_launch_count()
-    assert f(d=72) == 5 and f(s=100) == 5 and f(s=320) == 5 and f(d=256) == 5
+    assert f(d=68) == 5 and f(s=100) == 5 and f(s=576) == 5 and f(d=256) == 5 and f(d=136) == 5
     assert f(m_e=0) == 1 and f(heads=0) == 1 and f(q=None) == 1 and f(status=None) == 1
     assert f(k=0x200008) == 4 and f(ws=0x1000010) == 4
     assert f(ws=None) == 7 and f(ws_bytes=100) == 7
     assert f(out=0x100040) == 1  # output overlaps q
     assert f(n_img=0) == 0
-    assert lib.civic_kv_compressed_attention_workspace_bytes(1, 100, 2, 72, 128) == 0
+    assert lib.civic_kv_compressed_attention_workspace_bytes(1, 100, 2, 68, 128) == 0
     need = lib.civic_kv_compressed_attention_workspace_bytes(2, 100, 2, 64, 128)
     assert need >= 100 * 128 * 2 + 128 * 4 + 2 * 2 * 128 * 128 * 2 and need % 256 == 0
+    # the paper's shapes are accepted: 72-wide heads (stored 80 wide), 512 anchors, both with 128-wide heads
+    wide = lib.civic_kv_compressed_attention_workspace_bytes(2, 100, 2, 72, 128)
+    assert wide >= 2 * 2 * 128 * (2 * 80) * 2 and wide % 256 == 0
+    assert lib.civic_kv_compressed_attention_workspace_bytes(1, 100, 16, 64, 512) > 0
+    assert lib.civic_kv_compressed_attention_workspace_bytes(1, 100, 8, 128, 512) > 0
+    assert lib.civic_launch_count() == before
+
+
+def test_prepared_constants_validation(lib):
+    before = lib.civic_launch_count()
+    assert lib.civic_anchor_prepared_bytes(10, 100) == 0  # d_v not a multiple of 64
+    need = lib.civic_anchor_prepared_bytes(10, 128)
+    assert need >= 10 * 128 * 2 + 10 * 4 and need % 256 == 0
+    f = lib.civic_anchor_prepare
+    assert f(None, 10, 128, 0x200000, need, None) == 1
+    assert f(0x100000, 10, 128, None, need, None) == 1
+    assert f(0x100000, 10, 128, 0x200010, need, None) == 4
+    assert f(0x100000, 10, 128, 0x200000, need - 1, None) == 7
+    assert f(0x100000, 10, 100, 0x200000, need, None) == 5
+    assert f(0x100000, 10, 128, 0x100100, need, None) == 1  # output inside the anchors
+    g = lambda x=0x100000, prep=0x200000, ws=0x1000000, ws_bytes=1 << 30, status=0x400000, z=0x300000: \
+        lib.civic_anchor_aggregate_prepared(x, prep, 1, 100, 10, 128, ctypes.c_float(0.1), z, None, ws, ws_bytes, status, None)
+    assert g(prep=None) == 1 and g(prep=0x200010) == 4 and g(ws_bytes=10) == 7 and g(z=0x200000) == 1
+    assert lib.civic_kv_attention_prepared_bytes(100, 100) == 0
+    need = lib.civic_kv_attention_prepared_bytes(100, 128)
+    assert need >= 100 * 128 * 2 + 128 * 4 and need % 256 == 0
+    h = lib.civic_kv_attention_prepare
+    assert h(None, 100, 128, 0x200000, need, None) == 1 and h(0x100000, 100, 128, 0x200000, need - 1, None) == 7
+    assert h(0x100000, 100, 100, 0x200000, need, None) == 5 and h(0x100000, 100, 128, 0x200008, need, None) == 4
+    k = lambda prep=0x400000, out=0x500000, ws_bytes=1 << 30: lib.civic_kv_compressed_attention_prepared(
+        0x100000, 0x200000, 0x300000, prep, 1, 100, 2, 64, 128, out, 0x1000000, ws_bytes, 0x600000, None)
+    assert k(prep=None) == 1 and k(prep=0x400010) == 4 and k(ws_bytes=10) == 7 and k(out=0x400000) == 1
     assert lib.civic_launch_count() == before
 
 

@@ -155,3 +155,14 @@ def test_a_wait_that_never_gets_its_signal_ends_with_a_status():
     assert lib.civic_selftest_bounded_wait(0, rec.data_ptr(), None) == 1
     assert lib.civic_selftest_bounded_wait(1 << 25, rec.data_ptr(), None) == 1
     assert lib.civic_selftest_bounded_wait(100, None, None) == 1
+
+
+def test_prepared_anchors_give_the_same_bits():
+    """Q_A prepared once (civic_anchor_prepare) and reused: bit-identical to the plain call."""
+    x, a = inputs(2, 333, 257, 192, seed=77)
+    z, mass = check(x, a, 0.07)
+    prepared = civic.civic_anchor_prepare(a.to(DEV))
+    for _ in range(2):
+        z2, mass2, status = civic.civic_anchor_aggregate(x.to(DEV), prepared, 0.07)
+        assert int(status.item()) == 0
+        assert torch.equal(z2, z) and torch.equal(mass2, mass)

@@ -94,6 +94,17 @@ def check(q, k, v, r, heads):
     (1, 5, 2, 64, 64),       # fewer queries than one warp's 32 rows: one partly filled store box, three skipped
     (2, 33, 3, 128, 128),    # one row into the second warp's box
     (1, 129, 1, 64, 256),    # one row into the second query tile
+    (2, 300, 16, 72, 256),   # 72-wide heads (1152-wide towers with 16 heads): stored 80 wide, O written 64 + 8 columns
+    (1, 200, 3, 72, 64),     # the same with one block of anchors; the last head's second box runs past the tensor
+    (2, 300, 16, 64, 512),   # Table 2's 512 anchors: S fills all of tensor memory, the first chain is two MMAs wide
+    (1, 260, 8, 128, 512),   # 512 anchors, 128-wide heads: K_c resident, V_c streamed per query tile, one Q slot
+    (1, 140, 4, 128, 320),   # five blocks of anchors, streamed
+    (1, 150, 5, 64, 448),    # seven blocks of anchors, resident
+    (1, 100, 3, 40, 128),    # a head narrower than one box: K = 48, the output a single plain box of 40 columns
+    (1, 100, 3, 96, 128),    # 64 + 32 columns
+    (2, 130, 2, 112, 192),   # 64 + 48 columns
+    (1, 70, 5, 8, 64),       # the narrowest head
+    (1, 90, 2, 120, 256),    # 128-wide storage of a 120-wide head
 ])
 def test_against_oracle(n_img, m_e, heads, d, s):
     q, k, v, r = inputs(n_img, m_e, heads, d, s, seed=m_e + s)
@@ -110,3 +121,17 @@ def test_identity_assignment_is_dense_attention_and_deterministic():
     assert torch.allclose(out.float().cpu(), want, atol=0.03, rtol=0.03)
     out2, _ = civic.civic_kv_compressed_attention(q.to(DEV), k.to(DEV), v.to(DEV), torch.eye(128, device=DEV), 2)
     assert torch.equal(out2, out)
+
+
+@pytest.mark.parametrize("n_img,m_e,heads,d,s", [(2, 300, 4, 64, 128), (1, 200, 16, 72, 256), (1, 260, 2, 128, 512)])
+def test_prepared_assignment_gives_the_same_bits(n_img, m_e, heads, d, s):
+    """R converted once (civic_kv_attention_prepare) and reused: bit-identical to the plain call, twice."""
+    q, k, v, r = inputs(n_img, m_e, heads, d, s, seed=m_e + s + 1)
+    plain, _ = check(q, k, v, r, heads)
+    prepared = civic.civic_kv_attention_prepare(r.to(DEV))
+    for _ in range(2):
+        status = torch.full((1,), 77, dtype=torch.int32, device=DEV)  # the call itself clears it
+        got, status = civic.civic_kv_compressed_attention(q.to(DEV), k.to(DEV), v.to(DEV), prepared, heads,
+                                                          device_status=status)
+        assert int(status.item()) == 0
+        assert torch.equal(got, plain)

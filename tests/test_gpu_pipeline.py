@@ -60,3 +60,32 @@ def test_aggregate_select_compact_chain():
     for l in range(layers):
         assert np.array_equal(bits(kd[l]), want_k[l]) and np.array_equal(bits(vd[l]), want_v[l])
     assert merged.shape[1] == text_before + text_after + k  # Eq. 13: L + M_p rows
+
+
+def test_aggregation_feeds_kv_compressed_attention_on_one_vision_width():
+    """Eq. 8 and Eq. 9 on ONE model shape, chained on a stream: a 1152-wide vision tower with 16 heads
+    of 72.  Z_0 from the aggregation is projected (plain GEMMs: the caller's BLAS, here torch) to Q, K,
+    V of the compact encoder layer, which attends through 256 memory anchors with prepared constants."""
+    from tests.test_gpu_aggregate import check as check_aggregate
+    from tests.test_gpu_kv_attention import check as check_attention
+
+    g = torch.Generator().manual_seed(1152)
+    n_img, t_e, m_e, d_v, heads, s = 2, 1024, 256, 1152, 16, 256
+    x0 = (torch.randn((n_img, t_e, d_v), generator=g) * 1.5 + 0.7).to(torch.bfloat16)
+    anchors = torch.randn((m_e, d_v), generator=g)
+    w_q, w_k, w_v = (torch.randn((d_v, d_v), generator=g).mul_(d_v ** -0.5).to(torch.bfloat16).to(DEV) for _ in range(3))
+    r = torch.softmax(torch.randn((m_e, s), generator=g) * 3.0, dim=1)
+
+    prepared_a = civic.civic_anchor_prepare(anchors.to(DEV))
+    prepared_r = civic.civic_kv_attention_prepare(r.to(DEV))
+    z0, _, st1 = civic.civic_anchor_aggregate(x0.to(DEV), prepared_a, 0.07, want_mass=False)
+    q, k, v = (torch.matmul(z0, w) for w in (w_q, w_k, w_v))
+    out, st2 = civic.civic_kv_compressed_attention(q, k, v, prepared_r, heads)
+    torch.cuda.synchronize()
+    assert int(st1.item()) == 0 and int(st2.item()) == 0
+
+    # every stage against the oracle, the second fed with the first stage's GPU result
+    z_plain, _ = check_aggregate(x0, anchors, 0.07)
+    assert torch.equal(z_plain, z0)
+    out_plain, _ = check_attention(q.cpu(), k.cpu(), v.cpu(), r, heads)
+    assert torch.equal(out_plain, out)
