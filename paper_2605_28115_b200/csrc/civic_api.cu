@@ -449,8 +449,8 @@ civic_status_t tensor_map_encoder(EncodeTiledFn* out)
 }
 
 // bf16 tensor of rank 2 or 3, innermost dimension first; boxes of 64 elements (128 B, swizzled).
-// box_cols = 64 gives the swizzled 128-byte rows the MMA descriptors expect; any other width (a
-// multiple of 8 columns below 64) gives a plain, unswizzled box (used to store a head's last columns).
+// box_cols = 64 gives the swizzled 128-byte rows the MMA descriptors expect, 32 rows of 64 bytes with
+// the 64-byte swizzle (output staging); any other width (a multiple of 8 columns) a plain box.
 civic_status_t make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
                         const uint64_t* strides_bytes, uint32_t box_rows, uint32_t box_cols = 64)
 {
@@ -460,7 +460,8 @@ civic_status_t make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, i
     cuuint32_t estr[3] = {1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
                            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                           box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                          : (box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_error, sizeof g_cuda_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -819,27 +820,11 @@ civic_status_t civic_anchor_aggregate_prepared(const void* x0, const void* prepa
 struct KvAttnPlan {
     int32_t dim, compress_bn;
     int32_t d_pad, dim_ld;      // a head's columns in K_c / V_c (zero padded to a multiple of 16), all heads'
-    int32_t q_slots, v_stream;  // shared-memory plan of the attention kernel
+    int32_t kv_slots, q_slots, v_stream, n_buf;  // shared- and tensor-memory plan of the attention kernel
     int32_t n_parts;
     size_t r16_off, colsum_off, partial_off, kc_off, vc_off, total, attn_smem;
     size_t prepared_total;      // R in bf16 | column sums | panel sums: what civic_kv_attention_prepare writes
 };
-
-// Query tiles per block of the attention kernel: the split that needs the fewest rounds of
-// resident blocks, a block's cost being its tiles plus about a tile and a half of set-up
-// (barriers, tensor memory, the head's K_c and V_c).
-static int32_t attention_tiles_per_block(int32_t q_tiles, int64_t pairs, int blocks_per_sm)
-{
-    const int64_t resident = (int64_t)std::max(1, blocks_per_sm) * sm_count();
-    int32_t best = q_tiles;
-    double best_cost = 0.0;
-    for (int32_t per = q_tiles; per >= 1; --per) {
-        const int64_t blocks = (int64_t)((q_tiles + per - 1) / per) * pairs;
-        const double cost = (double)((blocks + resident - 1) / resident) * (per + 1.5);
-        if (per == q_tiles || cost < best_cost) { best = per; best_cost = cost; }
-    }
-    return best;
-}
 
 static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_heads, int32_t head_dim, int32_t s,
                                         KvAttnPlan& pl)
@@ -852,19 +837,21 @@ static civic_status_t plan_kv_attention(int32_t n_img, int32_t m_e, int32_t n_he
     pl.dim = (int32_t)dim;
     pl.d_pad = (head_dim + 15) / 16 * 16;
     pl.dim_ld = n_heads * pl.d_pad;
-    // shared memory: everything resident with two Q tiles in flight if that fits; else one Q tile;
-    // else V_c streamed through two slots of 64 anchors
-    const int tries[3][2] = {{2, 0}, {1, 0}, {1, 1}};
+    // shared memory, in order of preference: K_c and V_c of two pairs (the next pair loads while
+    // this one runs) and three Q tiles in flight; fewer Q tiles; one pair; V_c streamed
+    const int tries[7][3] = {{2, 3, 0}, {2, 2, 0}, {1, 3, 0}, {1, 2, 0}, {1, 1, 0}, {1, 2, 1}, {1, 1, 1}};
     pl.attn_smem = 0;
     for (const auto& t : tries) {
-        const size_t bytes = civic::attn_smem_bytes(pl.d_pad, s, t[0], t[1]);
+        const size_t bytes = civic::attn_smem_bytes(head_dim, pl.d_pad, s, t[0], t[1], t[2]);
         if (bytes <= kMaxDynamicSmem) {
-            pl.q_slots = t[0];
-            pl.v_stream = t[1];
+            pl.kv_slots = t[0];
+            pl.q_slots = t[1];
+            pl.v_stream = t[2];
             pl.attn_smem = bytes;
             break;
         }
     }
+    pl.n_buf = civic::attn_buffers(pl.d_pad, s);
     if (pl.attn_smem == 0) return CIVIC_ERR_UNSUPPORTED;
     pl.compress_bn = dim % 256 == 0 ? 256 : (dim % 192 == 0 ? 192 : 128);
     size_t off = 0;
@@ -940,17 +927,17 @@ static civic_status_t kv_attention_impl(const void* q, const void* k, const void
         const uint64_t dims[2] = {(uint64_t)s, (uint64_t)m_e}, str[1] = {(uint64_t)s * 2};
         if ((ms = make_map(enc, &map_r, r16, 2, dims, str, 64)) != CIVIC_OK) return ms;
     }
-    const int32_t tail = head_dim % 64;
+    const int32_t tail = head_dim % 32;
     {
         const uint64_t dims[3] = {(uint64_t)pl.dim, (uint64_t)m_e, (uint64_t)n_img};
         const uint64_t str[2] = {(uint64_t)pl.dim * 2, (uint64_t)m_e * pl.dim * 2};
         if ((ms = make_map(enc, &map_k_in, k, 3, dims, str, 64)) != CIVIC_OK) return ms;
         if ((ms = make_map(enc, &map_v_in, v, 3, dims, str, 64)) != CIVIC_OK) return ms;
         if ((ms = make_map(enc, &map_q, q, 3, dims, str, civic::kAggBM)) != CIVIC_OK) return ms;
-        // output boxes of 32 rows (one softmax warp's share of a tile): 64 columns wide, and the
-        // head's last columns where its width is not a multiple of 64
-        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32)) != CIVIC_OK) return ms;
-        if ((ms = make_map(enc, &map_o_tail, out, 3, dims, str, 32, tail ? (uint32_t)tail : 64u)) != CIVIC_OK) return ms;
+        // output boxes of 32 rows x 32 columns (what one softmax warp stages at a time), and the
+        // head's last columns where its width is not a multiple of 32
+        if ((ms = make_map(enc, &map_o, out, 3, dims, str, 32, 32)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_o_tail, out, 3, dims, str, 32, tail ? (uint32_t)tail : 32u)) != CIVIC_OK) return ms;
     }
     {
         const uint64_t dims[3] = {(uint64_t)pl.dim_ld, (uint64_t)s, (uint64_t)n_img};
@@ -960,41 +947,21 @@ static civic_status_t kv_attention_impl(const void* q, const void* k, const void
     }
 
     const int32_t q_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
+    const int64_t total_tiles = (int64_t)q_tiles * n_heads * n_img;
+    if (total_tiles > INT32_MAX) return CIVIC_ERR_UNSUPPORTED;
     civic::AttnParams ap;
     ap.error = device_status; ap.m_e = m_e; ap.s = s;
     ap.d = head_dim; ap.d_pad = pl.d_pad; ap.d_ld = pl.d_pad;
-    ap.q_slots = pl.q_slots; ap.v_stream = pl.v_stream;
+    ap.n_heads = n_heads; ap.q_tiles = q_tiles; ap.total_tiles = (int32_t)total_tiles;
+    ap.n_buf = pl.n_buf; ap.kv_slots = pl.kv_slots; ap.q_slots = pl.q_slots; ap.v_stream = pl.v_stream;
     ap.scale_log2e = 1.4426950408889634f / sqrtf((float)head_dim);
-    // Once per device: the kernel may use all of an SM's memory as shared memory (so that two blocks
-    // of 113 KB can be resident), and the figures that decide how many blocks fit on an SM
-    // together.  (The runtime's occupancy query answers 1 for this kernel whatever its shared
-    // memory, while two blocks were measured running side by side on the SMs.)
-    struct AttnDevice { std::atomic<int> ready; int smem_per_sm, reserved, regs_per_sm, regs_per_thread; };
-    static AttnDevice attn_dev[64];
-    AttnDevice local_info = {};
-    const int dev = device_slot();
-    AttnDevice& info = dev >= 0 ? attn_dev[dev] : local_info;
-    if (!info.ready.load(std::memory_order_acquire)) {
-        int device = 0;
-        CIVIC_CUDA_TRY(cudaGetDevice(&device));
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)kMaxDynamicSmem));
-        CIVIC_CUDA_TRY(cudaFuncSetAttribute(civic::kv_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                            (int)cudaSharedmemCarveoutMaxShared));
-        CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&info.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, device));
-        CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&info.reserved, cudaDevAttrReservedSharedMemoryPerBlock, device));
-        CIVIC_CUDA_TRY(cudaDeviceGetAttribute(&info.regs_per_sm, cudaDevAttrMaxRegistersPerMultiprocessor, device));
-        cudaFuncAttributes fattr;
-        CIVIC_CUDA_TRY(cudaFuncGetAttributes(&fattr, civic::kv_attention_kernel));
-        info.regs_per_thread = fattr.numRegs;
-        info.ready.store(1, std::memory_order_release);
+    {
+        static std::atomic<int> smem_allowed[64];
+        const civic_status_t as = allow_dynamic_smem(civic::kv_attention_kernel, kMaxDynamicSmem, smem_allowed);
+        if (as != CIVIC_OK) return as;
     }
-    const int regs_per_block = ((info.regs_per_thread + 7) / 8 * 8) * civic::kAttnThreads;
-    int blocks_per_sm = (int)((size_t)info.smem_per_sm / (pl.attn_smem + (size_t)info.reserved));
-    blocks_per_sm = std::min(blocks_per_sm, info.regs_per_sm / std::max(regs_per_block, 1));
-    blocks_per_sm = std::min(blocks_per_sm, 2048 / civic::kAttnThreads);
-    blocks_per_sm = std::min(blocks_per_sm, (int)(512 / civic::attn_tmem_cols(pl.d_pad, s)));
-    ap.tiles_per_block = attention_tiles_per_block(q_tiles, (int64_t)n_heads * n_img, blocks_per_sm);
+    // persistent: one block per SM (a block holds up to all of an SM's tensor memory)
+    const unsigned attn_blocks = (unsigned)std::min<int64_t>(total_tiles, sm_count());
 
     // everything that can fail on the host has happened: from here on work is enqueued
     const bool pdl = programmatic();
@@ -1024,11 +991,8 @@ static civic_status_t kv_attention_impl(const void* q, const void* k, const void
         else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
         if (gs != CIVIC_OK) return gs;
     }
-    CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel,
-                                 dim3((unsigned)((q_tiles + ap.tiles_per_block - 1) / ap.tiles_per_block),
-                                      (unsigned)n_heads, (unsigned)n_img),
-                                 (unsigned)civic::kAttnThreads, pl.attn_smem, stream, map_q, map_kc, map_vc, map_o,
-                                 map_o_tail, ap));
+    CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel, dim3(attn_blocks), (unsigned)civic::kAttnThreads,
+                                 pl.attn_smem, stream, map_q, map_kc, map_vc, map_o, map_o_tail, ap));
     g_launches.fetch_add(2, std::memory_order_relaxed);
     return CIVIC_OK;
 }

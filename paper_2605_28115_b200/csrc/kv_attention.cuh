@@ -70,7 +70,9 @@ __global__ void clear_status_kernel(int* __restrict__ status)
     if (threadIdx.x == 0) *status = 0;
 }
 
-constexpr int kAttnThreads = 192;  // warp 0: TMA, warp 1: TMEM + MMA, warps 2..5: one query row per thread
+// warp 0: TMA, warp 1: TMEM + MMA, warps 2..9 and 10..17: two groups of softmax warps (one per tensor
+// memory buffer, i.e. the even and the odd tiles), warps 18..21: output
+constexpr int kAttnThreads = 704;
 
 struct AttnParams {
     int* error;
@@ -78,8 +80,12 @@ struct AttnParams {
     int32_t d;                // head dimension (a multiple of 8)
     int32_t d_pad;            // d rounded up to a multiple of 16: the K of the first chain, the N of the second
     int32_t d_ld;             // columns per head of K_c and V_c (d_pad: zero columns behind the d real ones)
-    int32_t tiles_per_block;  // query tiles of 128 rows walked by one block
-    int32_t q_slots;          // Q tiles in flight: 2, or 1 where shared memory is short
+    int32_t n_heads;
+    int32_t q_tiles;          // query tiles of 128 rows per (head, image) pair
+    int32_t total_tiles;      // over all pairs; blocks take contiguous, equal shares
+    int32_t n_buf;            // S / P / O buffers in tensor memory: 2 (tiles overlap), or 1 where a tile needs more than 256 columns
+    int32_t kv_slots;         // K_c / V_c copies in shared memory: 2 (the next pair loads while this one runs) or 1
+    int32_t q_slots;          // Q tiles in flight: 1 .. 3
     int32_t v_stream;         // 0: the head's V_c stays resident; 1: streamed per query tile in blocks of 64 anchors
     float scale_log2e;        // log2(e) / sqrt(d)
 };
@@ -104,8 +110,8 @@ __device__ __forceinline__ void tmem_store8(uint32_t taddr, const uint32_t (&r)[
                  : "memory");
 }
 __device__ __forceinline__ void tmem_store_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// 16 fp32 columns at a time (the exponential pass keeps its register count down with these),
-// issue and wait split as for the 32-column loads
+// 16 fp32 columns at a time (keeps the register count of the passes down), issue and wait split as
+// for the 32-column loads
 __device__ __forceinline__ void tmem_load_issue16(uint32_t taddr, uint32_t (&r)[16])
 {
     asm volatile(
@@ -122,20 +128,23 @@ __device__ __forceinline__ void tmem_load_wait16(uint32_t (&r)[16])
                    "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
                  :: "memory");
 }
-// `cols` (a multiple of 32) columns in chunks of 16 with two register buffers
+// `cols` (a multiple of 32) columns from `taddr` on in chunks of 16 with two register buffers, from
+// the first column upwards or from the last chunk downwards; `body(acc, c0)` gets the chunk that
+// starts at column taddr + c0.
 template <class Body>
-__device__ __forceinline__ void for_each_chunk16(uint32_t taddr, int cols, Body&& body)
+__device__ __forceinline__ void for_each_chunk16(uint32_t taddr, int cols, bool downwards, Body&& body)
 {
+    const int first = downwards ? cols - 16 : 0, step = downwards ? -16 : 16;
     uint32_t even[16], odd[16];
-    tmem_load_issue16(taddr, even);
+    tmem_load_issue16(taddr + first, even);
 #pragma unroll 1
-    for (int c0 = 0; c0 < cols; c0 += 32) {
+    for (int i = 0, c0 = first; i < cols; i += 32, c0 += 2 * step) {
         tmem_load_wait16(even);
-        tmem_load_issue16(taddr + c0 + 16, odd);
+        tmem_load_issue16(taddr + c0 + step, odd);
         body(even, c0);
         tmem_load_wait16(odd);
-        if (c0 + 32 < cols) tmem_load_issue16(taddr + c0 + 32, even);
-        body(odd, c0 + 16);
+        if (i + 32 < cols) tmem_load_issue16(taddr + c0 + 2 * step, even);
+        body(odd, c0 + step);
     }
 }
 
@@ -147,56 +156,71 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     return d;
 }
 
-// 2^x for x <= 0 without the special-function unit: x = n + f with n = round(x), |f| <= 1/2;
-// 2^f by a cubic (largest relative error 7.5e-5, far below the bf16 cut that follows) and n added
-// into the exponent field.  Inputs below -125 give 2^-125 (any such weight is nothing beside the
-// row's largest, which is 1).  Eight instructions on the FMA and integer pipes.
-__device__ __forceinline__ float exp2_poly(float x)
+// x rounded up (towards +infinity) to a value with 16 zero low bits, as its upper half
+__device__ __forceinline__ uint16_t upper_half_rounded_up(float x)
 {
-    x = fmaxf(x, -125.f);
-    const float t = x + 12582912.f;  // 1.5 * 2^23: the low mantissa bits now hold round(x)
-    const float f = x - (t - 12582912.f);
-    float p = fmaf(0.0551716685f, f, 0.2426111251f);
-    p = fmaf(p, f, 0.6932609677f);
-    p = fmaf(p, f, 0.9999280572f);
-    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(t) << 23));
+    const uint32_t b = __float_as_uint(x);
+    return (uint16_t)(((b & 0x80000000u) ? b : b + 0xFFFFu) >> 16);
 }
 
 __host__ __device__ constexpr int round_up_int(int x, int a) { return (x + a - 1) / a * a; }
 
-// Shared memory: k [d_blocks][s x 128 B] | v [s/64 or 2][d_blocks][64 x 128 B] | q [q_slots][d_blocks][128 x 128 B]
-// | o [4 warps][d_blocks][32 x 128 B] | barriers, d_blocks = ceil(d_pad / 64).  Every block of data is
-// 1024-byte aligned; the kernel has no static shared memory, so the dynamic window itself starts on
-// such a boundary (checked at run time) and no slack is set aside: 113 KB for 64-wide heads and 256
-// anchors is exactly what lets two blocks share an SM.
-__host__ __device__ constexpr size_t attn_smem_bytes(int d_pad, int s, int q_slots, int v_stream)
+// Tensor memory of one tile, C columns.  The anchors are split between two sets of softmax warps:
+//   S_a = scores of anchors [0, s/2)  in columns [0, s/2),      read upwards,   P_a packed into [0, s/4)
+//   S_b = scores of anchors [s/2, s)  in columns [C - s/2, C),  read downwards, P_b packed into [C - s/4, C)
+// so that each set writes its bf16 weights behind its own reads.  The columns in the middle are free
+// by the time the second chain runs: O takes [o_col, o_col + d_pad) there and is read back in chunks
+// of 32 columns.  o_col is a multiple of the next power of two at or above d_pad: with the accumulator
+// of the second chain at column 96 (64 wide) its 16 MMAs ran for 3700 cycles instead of 600.  Where a
+// tile fits 256 columns the block holds two such buffers and works on two tiles at once.
+__host__ __device__ constexpr int attn_o_align(int d_pad) { return d_pad <= 32 ? 32 : (d_pad <= 64 ? 64 : 128); }
+__host__ __device__ constexpr uint32_t attn_o_col(int d_pad, int s)
 {
-    const size_t db = (size_t)(d_pad + 63) / 64;
-    return db * s * 128 + (size_t)(v_stream ? 2 : s / 64) * db * 8192 + (size_t)q_slots * db * 16384 + 4 * db * 4096 +
-           1024 /* barriers */;
+    return (uint32_t)round_up_int(s / 4, attn_o_align(d_pad));
 }
-// TMEM columns of a block: S in [0, s), later P in [0, s / 2) and O in [s / 2, s / 2 + d_pad), read
-// back in chunks of 32 columns
-__host__ __device__ constexpr uint32_t attn_tmem_cols(int d_pad, int s)
+__host__ __device__ constexpr uint32_t attn_tile_cols(int d_pad, int s)
 {
-    const int o_end = s / 2 + round_up_int(d_pad, 32);
-    const int need = s > o_end ? s : o_end;
+    const int mid = (int)attn_o_col(d_pad, s) + round_up_int(d_pad, 32) + s / 4;
+    const int need = s > mid ? s : mid;
     return need <= 32 ? 32u : (need <= 64 ? 64u : (need <= 128 ? 128u : (need <= 256 ? 256u : 512u)));
 }
+__host__ __device__ constexpr int attn_buffers(int d_pad, int s) { return attn_tile_cols(d_pad, s) <= 256 ? 2 : 1; }
+__host__ __device__ constexpr uint32_t attn_tmem_cols(int d_pad, int s)
+{
+    return attn_buffers(d_pad, s) == 2 ? 2 * (attn_tile_cols(d_pad, s) < 32u ? 32u : attn_tile_cols(d_pad, s))
+                                       : attn_tile_cols(d_pad, s);
+}
+// 32-column chunks of the output; an output warp stages at most two of them at a time for its 32 rows
+__host__ __device__ constexpr int attn_out_chunks(int d) { return (d + 31) / 32; }
+__host__ __device__ constexpr int attn_stage_chunks(int d) { return attn_out_chunks(d) < 2 ? attn_out_chunks(d) : 2; }
 
-// kPolyMask: which of the 16 columns of a chunk take their exponential on the FMA pipe
-// (exp2_poly) instead of the special-function unit, which is the busiest unit of this kernel
-// (16 results per clock and SM against 128 lanes of FMA).
-constexpr uint32_t kPolyMask = 0x0000u;
+// Shared memory: k [kv_slots][d_blocks][s x 128 B] | v [kv_slots][s/64][d_blocks][64 x 128 B] (streamed:
+// [2][d_blocks][64 x 128 B]) | q [q_slots][d_blocks][128 x 128 B] | o [4 warps][chunks][32 rows x 64 B] |
+// barriers and the row maxima the two sets of softmax warps show each other; d_blocks = ceil(d_pad / 64).
+// Every block of data is 1024-byte aligned; the kernel has no static shared memory, so the dynamic
+// window itself starts on such a boundary (checked at run time) and no slack is set aside.
+__host__ __device__ constexpr size_t attn_smem_bytes(int d, int d_pad, int s, int kv_slots, int q_slots, int v_stream)
+{
+    const size_t db = (size_t)(d_pad + 63) / 64;
+    return (size_t)kv_slots * db * s * 128 + (size_t)(v_stream ? 2 : kv_slots * (s / 64)) * db * 8192 +
+           (size_t)q_slots * db * 16384 + 4 * (size_t)attn_stage_chunks(d) * 2048 + 4096 /* barriers, row maxima and sums */;
+}
 
-// Registers are handed out per group of four warps, so a block of six warps is charged for eight:
-// bounding the kernel as if it had 256 threads, two blocks per SM, keeps it at 128 registers.
-__global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_constant__ CUtensorMap map_q,
-                                                                    const __grid_constant__ CUtensorMap map_k,
-                                                                    const __grid_constant__ CUtensorMap map_v,
-                                                                    const __grid_constant__ CUtensorMap map_o,
-                                                                    const __grid_constant__ CUtensorMap map_o_tail,
-                                                                    const AttnParams p)
+// One persistent block per SM.  Its warps form a pipeline over the block's query tiles:
+//   producer   K_c / V_c of a (head, image) pair whenever the pair changes (into the other slot, while the
+//              previous pair is still in use), Q tiles into a ring
+//   MMA        S(j) = Q K_c^T for the tile one ahead, then O(i) = P(i) V_c as soon as P(i) is complete
+//   softmax    maximum, exponentials, row sums of tile i; then straight on to tile i + 1, whose scores
+//              are already waiting in the other buffer
+//   output     O(i) / row sum -> bf16 -> staging -> bulk tensor store, which frees the buffer for S(i + 2)
+// so that the special-function unit (16 exponentials per clock and SM, the scarcest unit here) is kept
+// busy by the softmax warps while everything else runs beside it.
+__global__ void __launch_bounds__(kAttnThreads, 1) kv_attention_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                       const __grid_constant__ CUtensorMap map_k,
+                                                                       const __grid_constant__ CUtensorMap map_v,
+                                                                       const __grid_constant__ CUtensorMap map_o,
+                                                                       const __grid_constant__ CUtensorMap map_o_tail,
+                                                                       const AttnParams p)
 {
     extern __shared__ __align__(1024) uint8_t attn_smem[];
     uint8_t* base = attn_smem;
@@ -204,42 +228,54 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
     // the wait for the previous kernels like every other access to global memory)
     const bool misplaced = (smem_u32(base) & 1023u) != 0;
     const int d = p.d, d_pad = p.d_pad, s = p.s, d_blocks = (d_pad + 63) >> 6, s_blocks = s >> 6;
-    const int v_slots = p.v_stream ? 2 : s_blocks;
+    const int kv_slots = p.kv_slots, q_slots = p.q_slots, n_buf = p.n_buf;
+    const int out_chunks = attn_out_chunks(d), stage_chunks = attn_stage_chunks(d);
+    const int k_slot_bytes = d_blocks * s * 128, v_slot_bytes = (p.v_stream ? 1 : s_blocks) * d_blocks * 8192;
     uint8_t* k_sm = base;
-    uint8_t* v_sm = k_sm + d_blocks * s * 128;
-    uint8_t* q_sm = v_sm + v_slots * d_blocks * 8192;
-    uint8_t* o_sm = q_sm + p.q_slots * d_blocks * 16384;
+    uint8_t* v_sm = k_sm + kv_slots * k_slot_bytes;
+    uint8_t* q_sm = v_sm + (p.v_stream ? 2 : kv_slots) * v_slot_bytes;
+    uint8_t* o_sm = q_sm + q_slots * d_blocks * 16384;
     struct Sync {
-        uint64_t k_loaded, v_loaded, q_full[2], q_empty[2], v_full[2], v_empty[2], s_full, s_free, p_ready, o_done;
+        uint64_t kv_full[2], kv_empty[2], q_full[3], q_empty[3], v_full[2], v_empty[2];
+        uint64_t s_full[2], s_free[2], p_ready[2], o_done[2];
+        uint64_t pair[2][4];          // per group: the two softmax warps of a TMEM lane quarter meet here once per tile
+        uint16_t row_max[2][2][128];  // per group and side of the anchor split: upper half of the row maximum, rounded up
+        float row_sum[2][2][128];  // per buffer and side: sum of the row's cut weights, for the output warps
         uint32_t tmem_base;
         int abort;
     };
-    Sync& sy = *reinterpret_cast<Sync*>(o_sm + 4 * d_blocks * 4096);
+    static_assert(sizeof(Sync) <= 4096, "the barrier area is 4 KB");
+    Sync& sy = *reinterpret_cast<Sync*>(o_sm + 4 * stage_chunks * 2048);
     // the warp index through a shuffle: the compiler then knows it is the same in all lanes and
     // keeps what depends only on it (the MMA warp's addresses and descriptors) in uniform registers
     const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-    const int head = blockIdx.y, img = blockIdx.z;
-    const int tiles_total = (p.m_e + kAggBM - 1) / kAggBM;
-    const int first = blockIdx.x * p.tiles_per_block;
-    const int n_tiles = min(p.tiles_per_block, tiles_total - first);
+    // this block's tiles: [g0, g0 + n_tiles) of the list ordered by (image, head, query tile)
+    const int g0 = (int)((long long)p.total_tiles * blockIdx.x / gridDim.x);
+    const int n_tiles = (int)((long long)p.total_tiles * (blockIdx.x + 1) / gridDim.x) - g0;
     volatile int* abort = &sy.abort;
+    const uint32_t tile_cols = attn_tile_cols(d_pad, s) < 32u ? 32u : attn_tile_cols(d_pad, s);
     const uint32_t tmem_cols = attn_tmem_cols(d_pad, s);
-    const uint32_t o_col = (uint32_t)(s >> 1);
-    const int q_slots = p.q_slots;
+    const uint32_t o_col = attn_o_col(d_pad, s);
+    const int half_s = s >> 1;
+    const uint32_t sb_col = tile_cols - (uint32_t)half_s;         // first column of S_b
+    const uint32_t pb_col = tile_cols - (uint32_t)(half_s >> 1);  // first column of P_b
 
     if (threadIdx.x == 0) {
-        mbar_init(&sy.k_loaded, 1);
-        mbar_init(&sy.v_loaded, 1);
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&sy.q_full[b], 1);
-            mbar_init(&sy.q_empty[b], 1);
+            mbar_init(&sy.kv_full[b], 1);
+            mbar_init(&sy.kv_empty[b], 1);
             mbar_init(&sy.v_full[b], 1);
             mbar_init(&sy.v_empty[b], 1);
+            mbar_init(&sy.s_full[b], 1);
+            mbar_init(&sy.s_free[b], 4);   // one arrival per output warp
+            mbar_init(&sy.p_ready[b], 8);  // one arrival per softmax warp
+            mbar_init(&sy.o_done[b], 1);
         }
-        mbar_init(&sy.s_full, 1);
-        mbar_init(&sy.s_free, 4);   // one arrival per softmax warp
-        mbar_init(&sy.p_ready, 4);
-        mbar_init(&sy.o_done, 1);
+        for (int b = 0; b < 3; ++b) {
+            mbar_init(&sy.q_full[b], 1);
+            mbar_init(&sy.q_empty[b], 1);
+        }
+        for (int q = 0; q < 8; ++q) mbar_init(&sy.pair[q >> 2][q & 3], 2);  // one arrival per warp
         sy.abort = 0;
         fence_barrier_init();
     }
@@ -255,24 +291,38 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
     // A wait on a "free / empty" barrier uses the opposite parity, so the first pass over a
     // fresh barrier falls through.
     if (warp == 0 && lane == 0 && !stop) {
-        // ---- producer.  Columns of this head: d real ones from head * d in Q, d_ld (zero padded)
+        // ---- producer.  Columns of a head: d real ones from head * d in Q, d_ld (zero padded)
         // from head * d_ld in K_c and V_c; a 64-column box that runs past the head brings the next
         // head's columns (or the zero fill past the tensor), which meet zeros of K_c in the first
         // chain and are never read by the second.
-        const int qx = head * d, kx = head * p.d_ld;
-        mbar_expect_tx(&sy.k_loaded, d_blocks * s * 128);
-        for (int db = 0; db < d_blocks; ++db)
-            for (int r0 = 0; r0 < s; r0 += 64)  // boxes of 64 anchors
-                tma_load_3d(k_sm + db * s * 128 + r0 * 128, &map_k, kx + db * 64, r0, img, &sy.k_loaded);
         uint32_t v_it = 0;  // V_c blocks streamed so far
+        int kv_seq = -1, last_pair = -1;
         bool ok = true;
-        for (int t = 0; ok && t < n_tiles; ++t) {
-            const int st = t % q_slots, round = t / q_slots;
-            if (!mbar_wait(&sy.q_empty[st], (round & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) break;
+        for (int i = 0; ok && i < n_tiles; ++i) {
+            const int pair = (g0 + i) / p.q_tiles, tile = (g0 + i) - pair * p.q_tiles;
+            const int img = pair / p.n_heads, head = pair - img * p.n_heads;
+            const int qx = head * d, kx = head * p.d_ld;
+            if (pair != last_pair) {
+                last_pair = pair;
+                ++kv_seq;
+                const int slot = kv_seq % kv_slots, round = kv_seq / kv_slots;
+                if (!mbar_wait(&sy.kv_empty[slot], (round & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) break;
+                mbar_expect_tx(&sy.kv_full[slot], k_slot_bytes + (p.v_stream ? 0 : v_slot_bytes));
+                for (int db = 0; db < d_blocks; ++db)
+                    for (int r0 = 0; r0 < s; r0 += 64)  // boxes of 64 anchors
+                        tma_load_3d(k_sm + slot * k_slot_bytes + db * s * 128 + r0 * 128, &map_k, kx + db * 64, r0, img,
+                                    &sy.kv_full[slot]);
+                if (!p.v_stream)
+                    for (int sb = 0; sb < s_blocks; ++sb)
+                        for (int db = 0; db < d_blocks; ++db)
+                            tma_load_3d(v_sm + slot * v_slot_bytes + (sb * d_blocks + db) * 8192, &map_v, kx + db * 64,
+                                        sb * 64, img, &sy.kv_full[slot]);
+            }
+            const int st = i % q_slots;
+            if (!mbar_wait(&sy.q_empty[st], ((i / q_slots) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) break;
             mbar_expect_tx(&sy.q_full[st], d_blocks * 16384);
             for (int db = 0; db < d_blocks; ++db)
-                tma_load_3d(q_sm + (st * d_blocks + db) * 16384, &map_q, qx + db * 64, (first + t) * kAggBM, img,
-                            &sy.q_full[st]);
+                tma_load_3d(q_sm + (st * d_blocks + db) * 16384, &map_q, qx + db * 64, tile * kAggBM, img, &sy.q_full[st]);
             if (p.v_stream) {
                 for (int sb = 0; sb < s_blocks; ++sb, ++v_it) {
                     const int slot = v_it & 1;
@@ -283,12 +333,6 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
                         tma_load_3d(v_sm + (slot * d_blocks + db) * 8192, &map_v, kx + db * 64, sb * 64, img,
                                     &sy.v_full[slot]);
                 }
-            } else if (t == 0) {  // V_c is not needed before the second chain of the first tile
-                mbar_expect_tx(&sy.v_loaded, s_blocks * d_blocks * 8192);
-                for (int sb = 0; sb < s_blocks; ++sb)
-                    for (int db = 0; db < d_blocks; ++db)
-                        tma_load_3d(v_sm + (sb * d_blocks + db) * 8192, &map_v, kx + db * 64, sb * 64, img,
-                                    &sy.v_loaded);
             }
         }
         if (*abort) {  // copies still in flight after a time-out: give them ample time to land
@@ -296,150 +340,241 @@ __global__ void __launch_bounds__(256, 2) kv_attention_kernel(const __grid_const
             while ((unsigned long long)(clock64() - t0) < (1ull << 22)) {}
         }
     } else if (warp == 1 && !stop) {
-        // ---- MMA issue.  The whole warp walks the loop and the waits in step, one elected lane
-        // issues: a lone lane would hold every operand in its own registers and pay for moving
-        // them to the uniform registers the instruction reads, which made the 16 MMAs of the
-        // second chain take longer to issue than to run.  One descriptor per shared-memory
-        // operand, built once; a tile or K step further on only moves the start-address field
-        // (16-byte units in the low bits; shared memory addresses never carry out of it).
-        const int n_first = min(s, 256);  // an MMA is at most 256 columns wide: S takes one or two per K step
-        const uint32_t idesc1a = umma_idesc(n_first, 0), idesc1b = umma_idesc(s - n_first > 0 ? s - n_first : 16, 0);
-        const uint32_t idesc2 = umma_idesc(d_pad, 1);
+        // ---- MMA issue.  The whole warp walks the loops and the waits in step, one elected lane
+        // issues.  The instruction reads its operands from uniform registers: whatever the compiler
+        // cannot prove to be the same in all lanes it moves there one value at a time, which made an
+        // MMA take 100 .. 200 cycles to issue instead of 40.  So everything that changes per tile is
+        // computed once per tile and broadcast from lane 0 (after which it is provably uniform), and
+        // the inner loops only add constants to it.  Descriptors: one per shared-memory operand,
+        // built once; a slot, tile or K step further on only moves the start-address field (16-byte
+        // units in the low 32 bits; shared memory addresses never carry out of it).
+        auto uni = [](uint32_t v) { return __shfl_sync(0xFFFFFFFFu, v, 0); };
+        const uint32_t idesc1 = umma_idesc(half_s, 0), idesc2 = umma_idesc(d_pad, 1);
+        const bool one_wide = sb_col == (uint32_t)half_s && s <= 256;
+        const uint32_t idesc1w = umma_idesc(one_wide ? s : 16, 0);
         const uint64_t desc_q = umma_desc(smem_u32(q_sm), 16, 1024), desc_k = umma_desc(smem_u32(k_sm), 16, 1024);
         const uint64_t desc_v = umma_desc(smem_u32(v_sm), 8192, 1024);
-        const int k_steps = d_pad >> 4;
+        const uint32_t hi_q = (uint32_t)(desc_q >> 32), hi_k = (uint32_t)(desc_k >> 32), hi_v = (uint32_t)(desc_v >> 32);
+        auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
+        const int k_steps = d_pad >> 4, half16 = half_s >> 4;
+        const uint32_t k_db_step = (uint32_t)((s * 128) >> 4), k_half = (uint32_t)((half_s * 128) >> 4);
+        const uint32_t v_blk_step = (uint32_t)((d_blocks * 8192) >> 4);
         auto wait = [&](uint64_t* bar, uint32_t parity, int code) {
             return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort, p.error, code)) != 0;
         };
-        bool ok = wait(&sy.k_loaded, 0, kAggTimeoutFull);
+        bool ok = true;
         uint32_t v_it = 0;
-        for (int t = 0; ok && t < n_tiles; ++t) {
-            const int st = t % q_slots, round = t / q_slots;
-            // S[128, s] = Q(t) K_c^T, K = d_pad; the previous tile's O has been read out of these columns
-            if (!(ok = wait(&sy.q_full[st], round & 1, kAggTimeoutFull))) break;
-            if (!(ok = wait(&sy.s_free, (t & 1) ^ 1, kAggTimeoutAcc))) break;
-            tc_fence_after_sync();
-            for (int kk = 0; kk < k_steps; ++kk) {
-                const int db = kk >> 2, sub = kk & 3;
-                const uint64_t a = desc_q + (uint64_t)(((st * d_blocks + db) * 16384) >> 4) + 2 * sub;
-                const uint64_t b = desc_k + (uint64_t)((db * s * 128) >> 4) + 2 * sub;
+        int next = 0;                                    // first tile whose scores have not been issued yet
+        int pair1 = g0 / p.q_tiles, left1 = p.q_tiles - (g0 - pair1 * p.q_tiles);  // pair of tile `next`, its tiles left
+        int pair2 = pair1, left2 = left1;                // the same for tile i of the output stream
+        int seq1 = -1, last1 = -1;                       // pair sequence number of the scores stream
+        int seq2 = -1, last2 = -1;                       // ... of the output stream, which lags behind
+        for (int i = 0; ok && i < n_tiles; ++i) {
+            // scores of the tiles ahead: as many as there are buffers, and never into a K_c slot
+            // that a pair still waiting for its second chain occupies
+            while (ok && next < n_tiles && next < i + n_buf) {
+                if (pair1 != last1) {
+                    if (seq1 + 1 - (pair2 == last2 ? seq2 : seq2 + 1) >= kv_slots) break;
+                    last1 = pair1;
+                    ++seq1;
+                    if (!(ok = wait(&sy.kv_full[seq1 % kv_slots], (seq1 / kv_slots) & 1, kAggTimeoutFull))) break;
+                }
+                const int j = next, st = j % q_slots, buf = j % n_buf, k_slot = seq1 % kv_slots;
+                // S_a, S_b [128, s/2] = Q(j) K_c^T, K = d_pad, once the buffer's last O has been read out
+                if (!(ok = wait(&sy.q_full[st], (j / q_slots) & 1, kAggTimeoutFull))) break;
+                if (!(ok = wait(&sy.s_free[buf], ((j / n_buf) & 1) ^ 1, kAggTimeoutAcc))) break;
+                tc_fence_after_sync();
+                const uint32_t tb = uni(tmem_base + (uint32_t)buf * tile_cols);
+                const uint32_t a0 = uni((uint32_t)desc_q + (uint32_t)((st * d_blocks * 16384) >> 4));
+                const uint32_t b0 = uni((uint32_t)desc_k + (uint32_t)((k_slot * k_slot_bytes) >> 4));
+                if (one_wide) {  // S_a and S_b lie side by side: one MMA of s columns per K step
+                    for (int kk = 0; kk < k_steps; ++kk) {
+                        const uint32_t a = a0 + (uint32_t)(kk >> 2) * 1024u + 2u * (uint32_t)(kk & 3);
+                        const uint32_t b = b0 + (uint32_t)(kk >> 2) * k_db_step + 2u * (uint32_t)(kk & 3);
+                        if (elect_one()) umma_bf16(tb, desc(hi_q, a), desc(hi_k, b), idesc1w, kk != 0);
+                    }
+                } else {
+                    for (int kk = 0; kk < k_steps; ++kk) {
+                        const uint32_t a = a0 + (uint32_t)(kk >> 2) * 1024u + 2u * (uint32_t)(kk & 3);
+                        const uint32_t b = b0 + (uint32_t)(kk >> 2) * k_db_step + 2u * (uint32_t)(kk & 3);
+                        if (elect_one()) {
+                            umma_bf16(tb, desc(hi_q, a), desc(hi_k, b), idesc1, kk != 0);
+                            umma_bf16(tb + sb_col, desc(hi_q, a), desc(hi_k, b + k_half), idesc1, kk != 0);
+                        }
+                    }
+                }
                 if (elect_one()) {
-                    umma_bf16(tmem_base, a, b, idesc1a, kk != 0);
-                    if (s > 256) umma_bf16(tmem_base + 256, a, b + (uint64_t)((256 * 128) >> 4), idesc1b, kk != 0);
+                    umma_commit(&sy.q_empty[st]);
+                    umma_commit(&sy.s_full[buf]);
                 }
-            }
-            if (elect_one()) {
-                umma_commit(&sy.q_empty[st]);
-                umma_commit(&sy.s_full);
-            }
-            __syncwarp();
-            if (!p.v_stream && t == 0 && !(ok = wait(&sy.v_loaded, 0, kAggTimeoutFull))) break;
-            // O[128, d_pad] = P V_c, K = s: A from TMEM (8 columns per K step of 16), B blocks of 64
-            // anchors are d_blocks x 8 KB apart, K steps inside a block 2 KB
-            if (!(ok = wait(&sy.p_ready, t & 1, kAggTimeoutAcc))) break;
-            tc_fence_after_sync();
-            for (int sb = 0; sb < s_blocks; ++sb) {
-                int v_block = sb;
-                if (p.v_stream) {
-                    v_block = v_it & 1;
-                    if (!(ok = wait(&sy.v_full[v_block], (v_it >> 1) & 1, kAggTimeoutFull))) break;
-                    tc_fence_after_sync();
-                }
-                const uint64_t b = desc_v + (uint64_t)((v_block * d_blocks * 8192) >> 4);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    if (elect_one())
-                        umma_bf16_a_tmem(tmem_base + o_col, tmem_base + (uint32_t)(sb * 32 + kk * 8), b + 128 * kk, idesc2,
-                                         (sb | kk) != 0);
-                if (p.v_stream) {
-                    if (elect_one()) umma_commit(&sy.v_empty[v_block]);
-                    ++v_it;
-                }
+                __syncwarp();
+                ++next;
+                if (--left1 == 0) { ++pair1; left1 = p.q_tiles; }
             }
             if (!ok) break;
-            if (elect_one()) umma_commit(&sy.o_done);
+            // O(i)[128, d_pad] = P V_c, K = s in steps of 16 anchors: A from TMEM (8 columns per step;
+            // P_a for the first half of the anchors, P_b for the second), B blocks of 64 anchors are
+            // d_blocks x 8 KB apart, steps inside a block 2 KB
+            if (pair2 != last2) { last2 = pair2; ++seq2; }
+            const int buf = i % n_buf, v_slot = seq2 % kv_slots;
+            if (!(ok = wait(&sy.p_ready[buf], (i / n_buf) & 1, kAggTimeoutAcc))) break;
+            tc_fence_after_sync();
+            const uint32_t tb = uni(tmem_base + (uint32_t)buf * tile_cols);
+            const uint32_t to = tb + o_col, pa = tb, pb = tb + pb_col - (uint32_t)(half16 * 8);
+            if (!p.v_stream) {
+                const uint32_t v0 = uni((uint32_t)desc_v + (uint32_t)((v_slot * v_slot_bytes) >> 4));
+                if ((half16 & 3) == 0) {  // both halves are whole blocks of 64 anchors: four K steps per block
+                    for (int sb = 0; sb < s_blocks; ++sb) {
+                        const uint32_t b = v0 + (uint32_t)sb * v_blk_step;
+                        const uint32_t a = (sb * 4 < half16 ? pa : pb) + (uint32_t)(sb * 32);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            if (elect_one())
+                                umma_bf16_a_tmem(to, a + 8u * kk, desc(hi_v, b + 128u * kk), idesc2, (sb | kk) != 0);
+                    }
+                } else {
+                    for (int k16 = 0; k16 < 2 * half16; ++k16) {
+                        const uint32_t b = v0 + (uint32_t)(k16 >> 2) * v_blk_step + 128u * (uint32_t)(k16 & 3);
+                        const uint32_t a = (k16 < half16 ? pa : pb) + (uint32_t)(k16 * 8);
+                        if (elect_one()) umma_bf16_a_tmem(to, a, desc(hi_v, b), idesc2, k16 != 0);
+                    }
+                }
+            } else {
+                for (int sb = 0; sb < s_blocks; ++sb, ++v_it) {
+                    const int slot = v_it & 1;
+                    if (!(ok = wait(&sy.v_full[slot], (v_it >> 1) & 1, kAggTimeoutFull))) break;
+                    tc_fence_after_sync();
+                    const uint32_t v0 = uni((uint32_t)desc_v + (uint32_t)((slot * d_blocks * 8192) >> 4));
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const int k16 = sb * 4 + kk;
+                        const uint32_t a = (k16 < half16 ? pa : pb) + (uint32_t)(k16 * 8);
+                        if (elect_one()) umma_bf16_a_tmem(to, a, desc(hi_v, v0 + 128u * (uint32_t)kk), idesc2, k16 != 0);
+                    }
+                    if (elect_one()) umma_commit(&sy.v_empty[slot]);
+                }
+                if (!ok) break;
+            }
+            const bool pair_ends = left2 == 1 || i + 1 == n_tiles;  // its K_c / V_c slot may be loaded again
+            if (elect_one()) {
+                umma_commit(&sy.o_done[buf]);
+                if (pair_ends) umma_commit(&sy.kv_empty[v_slot]);
+            }
             __syncwarp();
+            if (--left2 == 0) { ++pair2; left2 = p.q_tiles; }
         }
-    } else if (warp >= 2 && !stop) {
-        // ---- softmax and output: thread = query row (TMEM lane) 32 * (warp % 4) + lane
-        const int quarter = warp & 3;
-        const uint32_t tm = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        uint8_t* o_stage = o_sm + (warp - 2) * d_blocks * 4096;  // [d_blocks][32 rows x 128 B], swizzled
-        const int full_blocks = d >> 6, tail = d & 63;           // 64-column blocks of the output, columns of the last
-        const int o_cols = round_up_int(d_pad, 32);
-        for (int t = 0; t < n_tiles; ++t) {
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.s_full, t & 1, abort, p.error, kAggTimeoutAcc))) break;
+    } else if (warp >= 2 && warp < 18 && !stop) {
+        // ---- softmax.  Two groups of eight warps: with two buffers group g takes the tiles i = g, g + 2,
+        // ... (buffer g), so that two tiles are in different phases of their softmax at any time and
+        // the special-function unit is not left idle while one tile looks for its maxima; with one
+        // buffer group 0 takes every tile.  Within a group: thread = query row (TMEM lane)
+        // 32 * (warp % 4) + lane and one side of the anchor split, S_a upwards or S_b downwards.  The two
+        // threads of a row agree on the shift of the exponentials through shared memory (each side's
+        // maximum, rounded up to 16 significant bits: any common shift at or above the true maximum
+        // is as good as the maximum itself) and leave their row sums in shared memory for the output
+        // warps.
+        const int group = (warp - 2) >> 3, quarter = warp & 3, side = ((warp - 2) >> 2) & 1;
+        const int row = quarter * 32 + lane;
+        const uint32_t s_col = side ? sb_col : 0u, p_col = side ? pb_col : 0u;
+        for (int i = group, turn = 0; i < n_tiles && group < n_buf; i += n_buf, ++turn) {
+            const int buf = group;
+            const uint32_t tm = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * tile_cols;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.s_full[buf], (i / n_buf) & 1, abort, p.error, kAggTimeoutAcc))) break;
             tc_fence_after_sync();
             float mx4[4] = {-3.0e38f, -3.0e38f, -3.0e38f, -3.0e38f};  // four chains instead of one
-            for_each_chunk(tm, s, [&](const uint32_t (&acc)[32], int) {
+            for_each_chunk16(tm + s_col, half_s, false, [&](const uint32_t (&acc)[16], int) {
 #pragma unroll
-                for (int c = 0; c < 32; c += 2)
+                for (int c = 0; c < 16; c += 2)
                     mx4[(c >> 1) & 3] = fmax3(mx4[(c >> 1) & 3], __uint_as_float(acc[c]), __uint_as_float(acc[c + 1]));
             });
-            const float shift = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2e;
-            // P(row, c) for the 16 columns of a chunk -> 8 packed columns at c / 2: always behind
-            // the columns of S this thread has already taken into registers
-            float row_sum = 0.f;
-            for_each_chunk16(tm, s, [&](const uint32_t (&acc)[16], int c0) {
+            sy.row_max[group][side][row] = upper_half_rounded_up(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sy.pair[group][quarter]);
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.pair[group][quarter], turn & 1, abort, p.error, kAggTimeoutAcc))) break;
+            const float m_a = __uint_as_float((uint32_t)sy.row_max[group][0][row] << 16);
+            const float m_b = __uint_as_float((uint32_t)sy.row_max[group][1][row] << 16);
+            const float shift = fmaxf(m_a, m_b) * p.scale_log2e;
+            // P(row, c) for the 16 columns of a chunk -> 8 packed columns at c / 2: always behind the
+            // columns of S this thread has already taken into registers (side b: above them, going down)
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+            for_each_chunk16(tm + s_col, half_s, side != 0, [&](const uint32_t (&acc)[16], int c0) {
                 uint32_t w[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     // The weights are cut to bf16 (upper halves of the fp32 words), not rounded: a
-                    // rounding conversion shares its pipe with exp2, which already bounds this
-                    // pass.  The row sum adds the cut values, so the common part of the error
-                    // cancels in O / row sum.
-                    const float a0 = fmaf(__uint_as_float(acc[2 * e]), p.scale_log2e, -shift);
-                    const float a1 = fmaf(__uint_as_float(acc[2 * e + 1]), p.scale_log2e, -shift);
-                    const uint32_t x0 = __float_as_uint(((kPolyMask >> (2 * e)) & 1u) ? exp2_poly(a0) : exp2_fast(a0));
-                    const uint32_t x1 = __float_as_uint(((kPolyMask >> (2 * e + 1)) & 1u) ? exp2_poly(a1) : exp2_fast(a1));
-                    row_sum += __uint_as_float(x0 & 0xFFFF0000u) + __uint_as_float(x1 & 0xFFFF0000u);
+                    // rounding conversion shares its pipe with exp2.  The row sum adds the cut values,
+                    // so the common part of the error cancels in O / row sum.
+                    const uint32_t x0 = __float_as_uint(exp2_fast(fmaf(__uint_as_float(acc[2 * e]), p.scale_log2e, -shift)));
+                    const uint32_t x1 = __float_as_uint(exp2_fast(fmaf(__uint_as_float(acc[2 * e + 1]), p.scale_log2e, -shift)));
+                    sum4[e & 3] += __uint_as_float(x0 & 0xFFFF0000u) + __uint_as_float(x1 & 0xFFFF0000u);
                     w[e] = __byte_perm(x0, x1, 0x7632);  // x0's upper half below x1's
                 }
-                tmem_store8(tm + (uint32_t)(c0 >> 1), w);
+                tmem_store8(tm + p_col + (uint32_t)(c0 >> 1), w);
             });
+            sy.row_sum[buf][side][row] = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             tmem_store_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sy.p_ready);
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.o_done, t & 1, abort, p.error, kAggTimeoutAcc))) break;
+            if (lane == 0) mbar_arrive(&sy.p_ready[buf]);
+        }
+    } else if (warp >= 18 && !stop) {
+        // ---- output: warp = TMEM lane quarter (warp % 4), thread = query row.  O / (sum_a + sum_b) as
+        // bf16 through swizzled staging rows and one bulk tensor store per 32 columns.
+        const int quarter = warp & 3;
+        uint8_t* o_stage = o_sm + (warp - 18) * stage_chunks * 2048;  // [1 or 2 chunks][32 rows x 64 B]
+        const int full_chunks = d >> 5, tail = d & 31;
+        for (int i = 0; i < n_tiles; ++i) {
+            const int buf = i % n_buf;
+            const int pair = (g0 + i) / p.q_tiles, tile = (g0 + i) - pair * p.q_tiles;
+            const int img = pair / p.n_heads, head = pair - img * p.n_heads;
+            const int m_first = tile * kAggBM + quarter * 32;
+            const uint32_t tm = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * tile_cols;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.o_done[buf], (i / n_buf) & 1, abort, p.error, kAggTimeoutAcc))) break;
             tc_fence_after_sync();
-            const float inv = 1.f / row_sum;  // at least one term is exp2(0) = 1
-            if (lane == 0) tma_store_wait_read();  // the previous tile's store has read the staging rows
-            __syncwarp();
-            for_each_chunk(tm + o_col, o_cols, [&](const uint32_t (&acc)[32], int c0) {
-                if (c0 + 32 >= o_cols) {  // the last of O is in registers: the next tile's S may overwrite it
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sy.s_free);
-                }
-                const int blk = c0 >> 6;  // 64-column block of the output
+            uint32_t acc[32];
+            tmem_load_issue(tm + o_col, acc);
+            const int row = quarter * 32 + lane;
+            const float inv = 1.f / (sy.row_sum[buf][0][row] + sy.row_sum[buf][1][row]);  // the largest term is about 1
+            for (int c0 = 0; c0 < out_chunks; c0 += 2) {  // two chunks per round through the staging rows
+                if (lane == 0) tma_store_wait_read();  // the previous round's stores have read the staging rows
+                __syncwarp();
+                const int c_end = min(c0 + 2, out_chunks);
+                for (int c = c0; c < c_end; ++c) {
+                    tmem_load_wait(acc);
+                    uint32_t w[16];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int col = c0 + q4 * 8;  // first of 8 output columns = one 16-byte piece
-                    if (col >= d) continue;       // padding behind the head's last column
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[q4 * 8 + 2 * e]) * inv,
-                                                                       __uint_as_float(acc[q4 * 8 + 2 * e + 1]) * inv);
+                    for (int e = 0; e < 16; ++e) {
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[2 * e]) * inv,
+                                                                       __uint_as_float(acc[2 * e + 1]) * inv);
                         w[e] = *reinterpret_cast<const uint32_t*>(&h);
                     }
-                    const int piece = (col & 63) >> 3;
-                    uint8_t* at = blk < full_blocks
-                                      ? o_stage + blk * 4096 + lane * 128 + ((piece ^ (lane & 7)) << 4)  // swizzled box of 64 columns
-                                      : o_stage + blk * 4096 + lane * (tail * 2) + (piece << 4);         // plain box of `tail` columns
-                    *reinterpret_cast<uint4*>(at) = make_uint4(w[0], w[1], w[2], w[3]);
+                    if (c + 1 < out_chunks) {
+                        tmem_load_issue(tm + o_col + 32 * (c + 1), acc);
+                    } else {  // all of O is in registers: the buffer may take the scores of the tile after next
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sy.s_free[buf]);
+                    }
+                    uint8_t* box = o_stage + (c - c0) * 2048;
+                    if (c < full_chunks) {  // 32 rows x 64 B, 64-byte swizzle: piece j of row r at j ^ ((r >> 1) & 3)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            *reinterpret_cast<uint4*>(box + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
+                                make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    } else {  // the head's last `tail` columns: a plain box, rows of tail * 2 bytes
+#pragma unroll
+                        for (int j = 0; j < 3; ++j)
+                            if (j * 8 < tail)
+                                *reinterpret_cast<uint4*>(box + lane * (tail * 2) + (j << 4)) =
+                                    make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    }
                 }
-            });
-            fence_async_smem();  // the bulk store reads the staging rows through the async proxy
-            __syncwarp();
-            if (lane == 0) {
-                const int m_first = (first + t) * kAggBM + quarter * 32;
-                if (m_first < p.m_e) {  // rows past m_e are clipped by the store
-                    for (int db = 0; db < full_blocks; ++db)
-                        tma_store_3d(&map_o, o_stage + db * 4096, head * d + db * 64, m_first, img);
-                    if (tail) tma_store_3d(&map_o_tail, o_stage + full_blocks * 4096, head * d + full_blocks * 64, m_first, img);
-                }
+                fence_async_smem();  // the bulk stores read the staging rows through the async proxy
+                __syncwarp();
+                if (lane == 0 && m_first < p.m_e)  // rows past m_e are clipped by the store
+                    for (int c = c0; c < c_end; ++c)
+                        tma_store_3d(c < full_chunks ? &map_o : &map_o_tail, o_stage + (c - c0) * 2048, head * d + c * 32,
+                                     m_first, img);
             }
         }
         if (lane == 0) tma_store_wait_read();
