@@ -156,6 +156,8 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void*
 }
 // the issuing thread's earlier stores have finished READING shared memory (it may be overwritten)
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// the issuing thread's earlier stores are complete (written)
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---- two blocks of a cluster working as one MMA unit (cta_group::2).  Block rank 0 (the leader)
 // issues the MMAs; every block loads its half of the operands into its own shared memory, but all
@@ -469,12 +471,12 @@ struct ValuesParams {
 
 constexpr int kEpilogueWarps = 8;
 
-template <int BN_, int STAGES_, bool SCORES_>
+template <int BN_, int STAGES_, bool SCORES_, bool STAGING_ = SCORES_>
 struct alignas(1024) GemmSmem {
     __nv_bfloat16 a[STAGES_][kAggBM * kAggBK];  // 128 rows x 128 B, K-major
     __nv_bfloat16 b[STAGES_][BN_ * kAggBK];
-    uint8_t out[SCORES_ ? kEpilogueWarps : 1][SCORES_ ? 32 * 128 : 1024];  // per epilogue warp: 32 rows x 64 bf16, 128-byte swizzled, for
-                                                // the bulk store of the weights (scores only)
+    uint8_t out[STAGING_ ? kEpilogueWarps : 1][STAGING_ ? 32 * 128 : 1024];  // per epilogue warp: 32 rows x 64 bf16, 128-byte swizzled,
+                                                // for the bulk store of a result (scores, compression)
     float2 stats[SCORES_ ? kEpilogueWarps : 1][128];  // per epilogue warp: (mu, r log2e / tau) of its columns (scores only)
     uint64_t full[STAGES_], empty[STAGES_], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
@@ -562,8 +564,8 @@ struct ScoresOpT {
     // through shared memory and a bulk tensor store, 32 rows x 64 columns at a time: whole
     // 128-byte lines reach L2 (16-byte stores from the registers, one row per lane, measured
     // 2.5 kcycles per 32 columns: every piece is a memory request of its own).
-    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap* map_c, uint32_t tmem,
-                                                    int ewarp, int lane, int m0, const Tile& tl)
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap* map_c, const CUtensorMap*,
+                                                    uint32_t tmem, int ewarp, int lane, int m0, const Tile& tl)
     {
         const int img = tl.img, n_tile = tl.n_tile;
         const int quarter = ewarp & 3, half = ewarp >> 2;
@@ -670,8 +672,8 @@ struct ValuesOp {
     // 16 token rows of 128 B per K step; the next 64 features start one box (8 KB) further on
     static __device__ __forceinline__ uint64_t b_desc(uint32_t b0, int kk) { return umma_desc(b0 + kk * 2048, kAggBK * 128, 1024); }
     static __device__ __forceinline__ void prefetch(const Params&, Smem&, int, int, const Tile&) {}
-    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, const CUtensorMap*, uint32_t tmem, int ewarp,
-                                                    int lane, int m0, const Tile& tl)
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem&, const CUtensorMap*, const CUtensorMap*,
+                                                    uint32_t tmem, int ewarp, int lane, int m0, const Tile& tl)
     {
         values_epilogue(p, tmem, ewarp, lane, m0, tl);
     }
@@ -697,10 +699,10 @@ struct CompressParams {
 
 template <int BN_>
 struct CompressOp {
-    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1;
+    static constexpr int BN = BN_, STAGES = BN_ == 128 ? 5 : 4, kCtas = 1;
     static constexpr bool kAMnMajor = true, kBMnMajor = true;
     using Params = CompressParams;
-    using Smem = GemmSmem<BN, STAGES, false>;
+    using Smem = GemmSmem<BN, STAGES, false, true>;
     static __device__ __forceinline__ int k_steps(const Params& p) { return (p.m_e + kAggBK - 1) / kAggBK; }
     static __device__ __forceinline__ bool tile(const Params& p, int worker, int n_workers, int i, Tile& tl)
     {
@@ -736,8 +738,10 @@ struct CompressOp {
         }
         reinterpret_cast<float*>(sm.stats[0])[ewarp * 32 + lane] = sum > 0.f ? 1.f / sum : 0.f;
     }
-    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap*, uint32_t tmem, int ewarp,
-                                                    int lane, int m0, const Tile& tl)
+    // map_k / map_v: K_c and V_c [n_img, s, d_v] with boxes of 32 rows x 64 columns, for the staged store
+    static __device__ __forceinline__ void epilogue(const Params& p, Smem& sm, const CUtensorMap* map_k,
+                                                    const CUtensorMap* map_v, uint32_t tmem, int ewarp, int lane, int m0,
+                                                    const Tile& tl)
     {
         const int half_cols = tl.n >> 1;
         const int quarter = ewarp & 3, half = ewarp >> 2;
@@ -746,6 +750,40 @@ struct CompressOp {
         const float inv = reinterpret_cast<const float*>(sm.stats[0])[ewarp * 32 + lane];
         const int nh = tl.n0 + half * half_cols;
         const bool second = tl.img >= p.n_img;
+        if (p.head_ld == p.head_dim && (half_cols & 63) == 0) {
+            // Plain layout: the rows leave through swizzled staging rows and one bulk tensor store per
+            // 32 rows x 64 columns (whole 128-byte lines; 16-byte stores straight from the registers, one
+            // row per lane, took 7000 cycles for a 128 x 256 tile, as long as half of its MMAs).
+            uint8_t* out = sm.out[ewarp];
+            const CUtensorMap* map = second ? map_v : map_k;
+            const int img = second ? tl.img - p.n_img : tl.img;
+            for_each_chunk(tmem + ((uint32_t)(quarter * 32) << 16) + half * half_cols, half_cols,
+                           [&](const uint32_t (&acc)[32], int c0) {
+                uint32_t w[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[2 * e]) * inv,
+                                                                   __uint_as_float(acc[2 * e + 1]) * inv);
+                    w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                if ((c0 & 32) == 0) {  // first half of a 64-column group: the buffer must be free again
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                }
+                const int j0 = (c0 & 32) >> 3;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+                    *reinterpret_cast<uint4*>(out + lane * 128 + (((j0 + q4) ^ (lane & 7)) << 4)) =
+                        make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+                if (c0 & 32) {  // the group is complete: hand it to the copy engine (clipped at s rows, d_v columns)
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && nh + c0 - 32 < p.d_v && m0 + quarter * 32 < p.s)
+                        tma_store_3d(map, out, nh + c0 - 32, m0 + quarter * 32, img);
+                }
+            });
+            return;
+        }
         __nv_bfloat16* out = (second ? p.out_v : p.out) +
                              ((size_t)(second ? tl.img - p.n_img : tl.img) * p.s + (row_ok ? row : 0)) * p.out_ld;
         const int pad = p.head_ld - p.head_dim;  // 0 or 8 columns (head_dim is a multiple of 8)
@@ -779,6 +817,8 @@ template <class Op>
 __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                      const __grid_constant__ CUtensorMap map_b,
                                                                      const __grid_constant__ CUtensorMap map_c,
+                                                                     const __grid_constant__ CUtensorMap map_d,
+                                                                     const __grid_constant__ CUtensorMap map_e,
                                                                      const typename Op::Params p)
 {
     constexpr int STAGES = Op::STAGES;
@@ -818,7 +858,12 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
 
     // A wait on the "empty" side uses the opposite parity, so the first pass over a fresh
     // barrier falls through (nothing has to be drained yet).
-    if (warp == 0 && lane == 0 && !stop) {
+    // Producer and MMA warp: the whole warp walks the loops and the waits in step and one elected lane
+    // issues.  A lone lane (the rest of the warp parked) keeps every operand in its own registers and
+    // moves them to the uniform registers the copy and MMA instructions read one value at a time:
+    // measured 120 cycles per tensor copy, so that a stage of six copies took 735 cycles to request
+    // and the whole K loop of the compression ran at the producer's pace, not the tensor core's.
+    if (warp == 0 && !stop) {
         // ---- producer (in every block)
         uint32_t it = 0;  // stages issued so far, over all tiles
         bool ok = true;
@@ -827,12 +872,14 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
             const int m0 = (tl.m_tile * Op::kCtas + (int)rank) * kAggBM;
             for (int k = 0; k < k_steps; ++k, ++it) {
                 const int s = it % STAGES;
-                ok = mbar_wait(&sm.empty[s], ((it / STAGES) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty);
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&sm.empty[s], ((it / STAGES) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) != 0;
                 if (!ok) break;
-                Op::load(p, sm, s, &map_a, &map_b, &map_c, k, m0, tl, rank, kPair ? cluster_address(&sm.full[s], 0) : 0u);
+                if (elect_one())
+                    Op::load(p, sm, s, &map_a, &map_b, &map_c, k, m0, tl, rank, kPair ? cluster_address(&sm.full[s], 0) : 0u);
+                __syncwarp();
             }
         }
-        if (*abort) {  // let the copies already in flight land before the block goes away
+        if (*abort && lane == 0) {  // let the copies already in flight land before the block goes away
             if (rank == 0) {
                 for (uint32_t j = it > (uint32_t)STAGES ? it - STAGES : 0; j < it; ++j) {
                     const long long t0 = clock64();
@@ -844,7 +891,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
                 while ((unsigned long long)(clock64() - t0) < (1ull << 22)) {}
             }
         }
-    } else if (warp == 1 && lane == 0 && !stop && rank == 0) {
+    } else if (warp == 1 && !stop && rank == 0) {
         // ---- MMA issue (leader only): 4 instructions of K = 16 per stage
         uint32_t it = 0;
         bool ok = true;
@@ -852,29 +899,33 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
         for (int local = 0; ok && Op::tile(p, worker, n_workers, local, tl); ++local) {
             const uint32_t idesc = umma_idesc(tl.n, Op::kBMnMajor ? 1 : 0, kAggBM * Op::kCtas, Op::kAMnMajor ? 1 : 0);
             const int buf = local & 1;
-            ok = mbar_wait(&sm.acc_empty[buf], ((local >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutAcc);
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_empty[buf], ((local >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutAcc)) != 0;
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t tmem_acc = tmem_base + buf * kAccStride;
             for (int k = 0; k < k_steps; ++k, ++it) {
                 const int s = it % STAGES;
-                ok = mbar_wait(&sm.full[s], (it / STAGES) & 1, abort, p.error, kAggTimeoutFull);
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&sm.full[s], (it / STAGES) & 1, abort, p.error, kAggTimeoutFull)) != 0;
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t a0 = smem_u32(sm.a[s]), b0 = smem_u32(sm.b[s]);
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < kAggBK / 16; ++kk) {
-                    if (kPair) umma_bf16_pair(tmem_acc, Op::a_desc(a0, kk), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
-                    else umma_bf16(tmem_acc, Op::a_desc(a0, kk), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                    for (int kk = 0; kk < kAggBK / 16; ++kk) {
+                        if (kPair) umma_bf16_pair(tmem_acc, Op::a_desc(a0, kk), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                        else umma_bf16(tmem_acc, Op::a_desc(a0, kk), Op::b_desc(b0, kk), idesc, (k | kk) != 0);
+                    }
+                    // frees the stage (in both blocks) once these MMAs have read it
+                    if (kPair) umma_commit_pair(&sm.empty[s]);
+                    else umma_commit(&sm.empty[s]);
                 }
-                // frees the stage (in both blocks) once these MMAs have read it
-                if (kPair) umma_commit_pair(&sm.empty[s]);
-                else umma_commit(&sm.empty[s]);
+                __syncwarp();
             }
-            if (ok) {
+            if (ok && elect_one()) {
                 if (kPair) umma_commit_pair(&sm.acc_full[buf]);
                 else umma_commit(&sm.acc_full[buf]);
             }
+            __syncwarp();
         }
     } else if (warp >= 2 && !stop) {
         // ---- epilogue: warps 2..9; a warp may read the TMEM lane quarter (warp index mod 4)
@@ -888,7 +939,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sm.acc_full[buf], (local >> 1) & 1, abort, p.error, kAggTimeoutAcc)))
                 break;
             tc_fence_after_sync();
-            Op::epilogue(p, sm, &map_c, tmem_base + buf * kAccStride, ewarp, lane, m0, tl);
+            Op::epilogue(p, sm, &map_d, &map_e, tmem_base + buf * kAccStride, ewarp, lane, m0, tl);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {  // this warp has drained its part of the accumulator
@@ -896,7 +947,7 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
                 else mbar_arrive(&sm.acc_empty[buf]);
             }
         }
-        if (lane == 0) tma_store_wait_read();  // this warp's bulk stores no longer need its shared memory
+        if (lane == 0) tma_store_wait_all();  // this warp's bulk stores have been written
     }
     tc_fence_before_sync();
     __syncthreads();

@@ -502,9 +502,12 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
     return CIVIC_OK;
 }
 
+// map_a, map_b, map_c: operands (what each Op loads through them); map_d, map_e: results stored by bulk
+// tensor copies (maps an Op does not use may repeat another one)
 template <class Op>
 civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c,
-                           const typename Op::Params& params, int32_t total_tiles, cudaStream_t stream)
+                           const CUtensorMap& map_d, const CUtensorMap& map_e, const typename Op::Params& params,
+                           int32_t total_tiles, cudaStream_t stream)
 {
     const size_t smem = sizeof(typename Op::Smem) + 1024;
     {
@@ -550,7 +553,7 @@ civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, c
         }
         if (workers > n) cfg.gridDim = dim3((unsigned)(n * 2));
     }
-    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_gemm_kernel<Op>, map_a, map_b, map_c, params));
+    CIVIC_CUDA_TRY(cudaLaunchKernelEx(&cfg, civic::aggregate_gemm_kernel<Op>, map_a, map_b, map_c, map_d, map_e, params));
     return CIVIC_OK;
 }
 
@@ -765,10 +768,10 @@ static civic_status_t aggregate_impl(const void* x0, const float* anchors, const
     if (m_tiles >= 2) {  // pairs of blocks share tiles of 256 anchors
         const int32_t m_pairs = (m_tiles + 1) / 2;
         sp.grid = civic::TileGrid{m_pairs, pl.n_tiles_t, n_img, m_pairs * pl.n_tiles_t * n_img};
-        gs = launch_gemm<civic::ScoresPairOp>(map_q, map_x_scores, map_p_store, sp, sp.grid.total, stream);
+        gs = launch_gemm<civic::ScoresPairOp>(map_q, map_x_scores, map_p_store, map_p_store, map_p_store, sp, sp.grid.total, stream);
     } else {
         sp.grid = civic::TileGrid{m_tiles, pl.n_tiles_t, n_img, m_tiles * pl.n_tiles_t * n_img};
-        gs = launch_gemm<civic::ScoresOp>(map_q, map_x_scores, map_p_store, sp, sp.grid.total, stream);
+        gs = launch_gemm<civic::ScoresOp>(map_q, map_x_scores, map_p_store, map_p_store, map_p_store, sp, sp.grid.total, stream);
     }
     if (gs != CIVIC_OK) return gs;
     civic::ValuesParams vp;
@@ -776,9 +779,9 @@ static civic_status_t aggregate_impl(const void* x0, const float* anchors, const
     vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t;
     const int32_t f_tiles = (d_v + pl.values_bn - 1) / pl.values_bn;
     vp.grid = civic::TileGrid{m_tiles, f_tiles, n_img, m_tiles * f_tiles * n_img};
-    if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
-    else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
-    else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, map_p, vp, vp.grid.total, stream);
+    if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, map_p, map_p, map_p, vp, vp.grid.total, stream);
+    else if (pl.values_bn == 192) gs = launch_gemm<civic::ValuesOp<192>>(map_p, map_x_values, map_p, map_p, map_p, vp, vp.grid.total, stream);
+    else gs = launch_gemm<civic::ValuesOp<128>>(map_p, map_x_values, map_p, map_p, map_p, vp, vp.grid.total, stream);
     if (gs != CIVIC_OK) return gs;
     int n_launched = 3;
     if (token_mass) {
@@ -922,7 +925,7 @@ static civic_status_t kv_attention_impl(const void* q, const void* k, const void
     EncodeTiledFn enc = nullptr;
     civic_status_t ms = tensor_map_encoder(&enc);
     if (ms != CIVIC_OK) return ms;
-    CUtensorMap map_r, map_k_in, map_v_in, map_q, map_kc, map_vc, map_o, map_o_tail;
+    CUtensorMap map_r, map_k_in, map_v_in, map_q, map_kc, map_vc, map_kc_out, map_vc_out, map_o, map_o_tail;
     {
         const uint64_t dims[2] = {(uint64_t)s, (uint64_t)m_e}, str[1] = {(uint64_t)s * 2};
         if ((ms = make_map(enc, &map_r, r16, 2, dims, str, 64)) != CIVIC_OK) return ms;
@@ -944,6 +947,9 @@ static civic_status_t kv_attention_impl(const void* q, const void* k, const void
         const uint64_t str[2] = {(uint64_t)pl.dim_ld * 2, (uint64_t)s * pl.dim_ld * 2};
         if ((ms = make_map(enc, &map_kc, kc, 3, dims, str, 64)) != CIVIC_OK) return ms;
         if ((ms = make_map(enc, &map_vc, vc, 3, dims, str, 64)) != CIVIC_OK) return ms;
+        // the compression's staged stores: 32 rows (one epilogue warp's anchors) x 64 columns
+        if ((ms = make_map(enc, &map_kc_out, kc, 3, dims, str, 32)) != CIVIC_OK) return ms;
+        if ((ms = make_map(enc, &map_vc_out, vc, 3, dims, str, 32)) != CIVIC_OK) return ms;
     }
 
     const int32_t q_tiles = (m_e + civic::kAggBM - 1) / civic::kAggBM;
@@ -986,9 +992,9 @@ static civic_status_t kv_attention_impl(const void* q, const void* k, const void
     cp.out = kc; cp.out_v = vc; cp.n_img = n_img;
     {
         civic_status_t gs;
-        if (pl.compress_bn == 256) gs = launch_gemm<civic::CompressOp<256>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
-        else if (pl.compress_bn == 192) gs = launch_gemm<civic::CompressOp<192>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
-        else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_k_in, map_v_in, cp, cp.grid.total, stream);
+        if (pl.compress_bn == 256) gs = launch_gemm<civic::CompressOp<256>>(map_r, map_k_in, map_v_in, map_kc_out, map_vc_out, cp, cp.grid.total, stream);
+        else if (pl.compress_bn == 192) gs = launch_gemm<civic::CompressOp<192>>(map_r, map_k_in, map_v_in, map_kc_out, map_vc_out, cp, cp.grid.total, stream);
+        else gs = launch_gemm<civic::CompressOp<128>>(map_r, map_k_in, map_v_in, map_kc_out, map_vc_out, cp, cp.grid.total, stream);
         if (gs != CIVIC_OK) return gs;
     }
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::kv_attention_kernel, dim3(attn_blocks), (unsigned)civic::kAttnThreads,

@@ -577,7 +577,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) kv_attention_kernel(const __g
                                      m_first, img);
             }
         }
-        if (lane == 0) tma_store_wait_read();
+        if (lane == 0) tma_store_wait_all();
     }
     tc_fence_before_sync();
     __syncthreads();
