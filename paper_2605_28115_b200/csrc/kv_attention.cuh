@@ -290,52 +290,64 @@ __global__ void __launch_bounds__(kAttnThreads, 1) kv_attention_kernel(const __g
 
     // A wait on a "free / empty" barrier uses the opposite parity, so the first pass over a
     // fresh barrier falls through.
-    if (warp == 0 && lane == 0 && !stop) {
-        // ---- producer.  Columns of a head: d real ones from head * d in Q, d_ld (zero padded)
-        // from head * d_ld in K_c and V_c; a 64-column box that runs past the head brings the next
-        // head's columns (or the zero fill past the tensor), which meet zeros of K_c in the first
-        // chain and are never read by the second.
+    if (warp == 0 && !stop) {
+        // ---- producer (the whole warp in step, an elected lane issues: see the MMA warp).  Columns of a
+        // head: d real ones from head * d in Q, d_ld (zero padded) from head * d_ld in K_c and V_c; a
+        // 64-column box that runs past the head brings the next head's columns (or the zero fill past
+        // the tensor), which meet zeros of K_c in the first chain and are never read by the second.
+        auto wait = [&](uint64_t* bar, uint32_t parity) {
+            return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort, p.error, kAggTimeoutEmpty)) != 0;
+        };
         uint32_t v_it = 0;  // V_c blocks streamed so far
-        int kv_seq = -1, last_pair = -1;
-        bool ok = true;
+        int kv_seq = -1;
+        int pair = g0 / p.q_tiles, tile = g0 - pair * p.q_tiles;
+        bool ok = true, new_pair = true;
         for (int i = 0; ok && i < n_tiles; ++i) {
-            const int pair = (g0 + i) / p.q_tiles, tile = (g0 + i) - pair * p.q_tiles;
             const int img = pair / p.n_heads, head = pair - img * p.n_heads;
             const int qx = head * d, kx = head * p.d_ld;
-            if (pair != last_pair) {
-                last_pair = pair;
+            if (new_pair) {
                 ++kv_seq;
                 const int slot = kv_seq % kv_slots, round = kv_seq / kv_slots;
-                if (!mbar_wait(&sy.kv_empty[slot], (round & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) break;
-                mbar_expect_tx(&sy.kv_full[slot], k_slot_bytes + (p.v_stream ? 0 : v_slot_bytes));
-                for (int db = 0; db < d_blocks; ++db)
-                    for (int r0 = 0; r0 < s; r0 += 64)  // boxes of 64 anchors
-                        tma_load_3d(k_sm + slot * k_slot_bytes + db * s * 128 + r0 * 128, &map_k, kx + db * 64, r0, img,
-                                    &sy.kv_full[slot]);
-                if (!p.v_stream)
-                    for (int sb = 0; sb < s_blocks; ++sb)
-                        for (int db = 0; db < d_blocks; ++db)
-                            tma_load_3d(v_sm + slot * v_slot_bytes + (sb * d_blocks + db) * 8192, &map_v, kx + db * 64,
-                                        sb * 64, img, &sy.kv_full[slot]);
+                if (!(ok = wait(&sy.kv_empty[slot], (round & 1) ^ 1))) break;
+                if (elect_one()) {
+                    mbar_expect_tx(&sy.kv_full[slot], k_slot_bytes + (p.v_stream ? 0 : v_slot_bytes));
+                    for (int db = 0; db < d_blocks; ++db)
+                        for (int r0 = 0; r0 < s; r0 += 64)  // boxes of 64 anchors
+                            tma_load_3d(k_sm + slot * k_slot_bytes + db * s * 128 + r0 * 128, &map_k, kx + db * 64, r0, img,
+                                        &sy.kv_full[slot]);
+                    if (!p.v_stream)
+                        for (int sb = 0; sb < s_blocks; ++sb)
+                            for (int db = 0; db < d_blocks; ++db)
+                                tma_load_3d(v_sm + slot * v_slot_bytes + (sb * d_blocks + db) * 8192, &map_v, kx + db * 64,
+                                            sb * 64, img, &sy.kv_full[slot]);
+                }
+                __syncwarp();
             }
             const int st = i % q_slots;
-            if (!mbar_wait(&sy.q_empty[st], ((i / q_slots) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty)) break;
-            mbar_expect_tx(&sy.q_full[st], d_blocks * 16384);
-            for (int db = 0; db < d_blocks; ++db)
-                tma_load_3d(q_sm + (st * d_blocks + db) * 16384, &map_q, qx + db * 64, tile * kAggBM, img, &sy.q_full[st]);
+            if (!(ok = wait(&sy.q_empty[st], ((i / q_slots) & 1) ^ 1))) break;
+            if (elect_one()) {
+                mbar_expect_tx(&sy.q_full[st], d_blocks * 16384);
+                for (int db = 0; db < d_blocks; ++db)
+                    tma_load_3d(q_sm + (st * d_blocks + db) * 16384, &map_q, qx + db * 64, tile * kAggBM, img, &sy.q_full[st]);
+            }
+            __syncwarp();
             if (p.v_stream) {
                 for (int sb = 0; sb < s_blocks; ++sb, ++v_it) {
                     const int slot = v_it & 1;
-                    ok = mbar_wait(&sy.v_empty[slot], ((v_it >> 1) & 1) ^ 1, abort, p.error, kAggTimeoutEmpty);
-                    if (!ok) break;
-                    mbar_expect_tx(&sy.v_full[slot], d_blocks * 8192);
-                    for (int db = 0; db < d_blocks; ++db)
-                        tma_load_3d(v_sm + (slot * d_blocks + db) * 8192, &map_v, kx + db * 64, sb * 64, img,
-                                    &sy.v_full[slot]);
+                    if (!(ok = wait(&sy.v_empty[slot], ((v_it >> 1) & 1) ^ 1))) break;
+                    if (elect_one()) {
+                        mbar_expect_tx(&sy.v_full[slot], d_blocks * 8192);
+                        for (int db = 0; db < d_blocks; ++db)
+                            tma_load_3d(v_sm + (slot * d_blocks + db) * 8192, &map_v, kx + db * 64, sb * 64, img,
+                                        &sy.v_full[slot]);
+                    }
+                    __syncwarp();
                 }
             }
+            new_pair = ++tile == p.q_tiles;
+            if (new_pair) { tile = 0; ++pair; }
         }
-        if (*abort) {  // copies still in flight after a time-out: give them ample time to land
+        if (*abort && lane == 0) {  // copies still in flight after a time-out: give them ample time to land
             const long long t0 = clock64();
             while ((unsigned long long)(clock64() - t0) < (1ull << 22)) {}
         }
