@@ -36,11 +36,15 @@ FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used when MEASURE
 
 # DRAM bytes (read + write) of ONE civic_compact_kv launch, keyed by workload name: NOT measured by
 # the run that prints them, but taken from the ncu captures summarised in profiles/ (an 8-layer case
-# of the same kernel, dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled by 36 / 8: the
-# traffic grows in proportion to the layers).  Absent = not captured for that workload.
+# of the same kernel, dram__bytes_read.sum + dram__bytes_write.sum per launch).  Scaled to the full
+# launch as: reads x layers / 8 (they grow in proportion to the layers), writes = algorithmic bytes
+# written minus what is still dirty in L2 when the kernel ends (55 .. 57 MB, a property of L2, not of
+# the layer count).  Absent = not captured for that workload.
 NCU_DRAM_TRAFFIC_PER_LAUNCH = {
-    # reads x4.5, writes = algorithmic minus the 52.0 MB that were still dirty in L2 at kernel end
-    "c3_kv_qwen3vl8b": (1_859_200_000, "profiles/gather_rows_kernel_c3_kv.md"),
+    "c3_kv_qwen3vl8b": (1_856_400_000, "profiles/gather_rows_kernel_c3_kv.md"),
+    "c5_hires_keep_1_2": (1_794_800_000, "profiles/gather_rows_kernel_layouts_c3_c5.md"),
+    "c5_hires_keep_1_3": (1_176_900_000, "profiles/gather_rows_kernel_layouts_c3_c5.md"),
+    "c5_hires_keep_1_4": (868_200_000, "profiles/gather_rows_kernel_layouts_c3_c5.md"),
 }
 TRAFFIC_SOURCE = ("ncu capture of an 8-layer case of the same kernel, scaled to {layers} layers; "
                   "not measured by this run ({file})")
@@ -472,6 +476,27 @@ def contiguous_copy_rate(st: DeviceState, launches=10):
     return nbytes / (start.elapsed_time(end) / launches * 1e-3) / 1e9
 
 
+def index_check_cost(st: DeviceState, launches=20):
+    """Microseconds per civic_compact_kv launch with the device-side index validation switched on
+    (the checked kernels: every index tested against its range, faults recorded, nothing trapped)."""
+    import torch
+
+    from paper_2605_28115_b200 import civic
+
+    record = torch.zeros(4, dtype=torch.int32, device=st.dev)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with civic.index_check(record):
+        for _ in range(3):
+            st.compact_kv()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(launches):
+            st.compact_kv()
+        end.record()
+        torch.cuda.synchronize()
+    return {"us_per_launch": start.elapsed_time(end) / launches * 1e3, "fault_record": record.cpu().tolist()}
+
+
 def kv_roofline(wl, kv_bytes, kv_ms, kv_layout="token_major", default_variant=True):
     """The roofline object of the K/V gather from event-bracketed launches (ms each)."""
     kv_avg = sum(kv_ms) / len(kv_ms)
@@ -609,7 +634,6 @@ def time_aggregate(w, dev, steps, warm):
     def step_unprepared():
         civic.civic_anchor_aggregate(x0, anchors, w.tau, z0=z0, token_mass=mass, workspace=ws, device_status=status)
 
-    unprepared_us = time_loop(step_unprepared, max(steps // 4, 1), warm)
     for _ in range(warm):
         step()
     torch.cuda.synchronize()
@@ -625,6 +649,7 @@ def time_aggregate(w, dev, steps, warm):
     clocks = sampler.stop()
     launches = civic.launch_count() - launches0
     ms = start.elapsed_time(end) / steps
+    unprepared_us = time_loop(step_unprepared, steps, warm)  # as long a loop: the same power-cap regime
     if int(status.item()) != 0:
         raise SystemExit(f"a wait inside the aggregation kernels timed out (status {int(status.item())})")
     value = w.flops / (ms * 1e-3) / 1e12
@@ -695,7 +720,6 @@ def time_kv_attention(w, dev, steps, warm):
     def step_unprepared():
         civic.civic_kv_compressed_attention(q, k, v, r, w.n_heads, out=out, workspace=ws, device_status=status)
 
-    unprepared_us = time_loop(step_unprepared, max(steps // 4, 1), warm)
     for _ in range(warm):
         step()
     torch.cuda.synchronize()
@@ -711,6 +735,7 @@ def time_kv_attention(w, dev, steps, warm):
     clocks = sampler.stop()
     launches = civic.launch_count() - launches0
     ms = start.elapsed_time(end) / steps
+    unprepared_us = time_loop(step_unprepared, steps, warm)
     if int(status.item()) != 0:
         raise SystemExit(f"a wait inside the kernels timed out (status {int(status.item())})")
     value = w.flops / (ms * 1e-3) / 1e12
@@ -846,6 +871,7 @@ def run_civic(args):
             own = contiguous_copy_rate(st)
             roofline["same_kernel_keeping_every_row_gbs"] = own
             roofline["frac_of_same_kernel_keeping_every_row"] = roofline["achieved"] / own
+            roofline["with_index_check"] = index_check_cost(st)
 
     # end to end: pinned host inputs -> path -> pinned host results, every step
     e2e = None
