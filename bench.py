@@ -310,7 +310,13 @@ class HostState:
     (small) are copied to the device, and the index results copied back.
     mode "staged": every input is copied to the device, the path runs on device buffers, every
     result is copied back.
+    mode "pipelined": the K/V kernel reads the kept rows from pinned host memory (as in zero_copy) but
+    writes them into device buffers, a few layers per launch; a second stream's copy engine moves each
+    finished chunk to pinned host memory while the kernel reads the next one.  PCIe then carries the
+    kernel's read requests and completions in one direction pair and plain bulk writes in the other.
     """
+
+    CHUNK_LAYERS = 2
 
     def __init__(self, st: DeviceState, mode: str):
         import torch
@@ -339,6 +345,17 @@ class HostState:
                            if wl.n_layers else None)
             # bytes that cross PCIe towards the device: small inputs + the kept rows the kernels read
             self.h2d_bytes = small_in + big_out
+        elif mode == "pipelined":
+            c = self.CHUNK_LAYERS
+            self.chunks = [range(l, min(l + c, wl.n_layers)) for l in range(0, wl.n_layers, c)]
+            self.chunk_tables = [civic.kv_tables([self.k_src_h[l] for l in ls], [self.v_src_h[l] for l in ls],
+                                                 [st.k_dst[l] for l in ls], [st.v_dst[l] for l in ls])
+                                 for ls in self.chunks]
+            self.copy_stream = torch.cuda.Stream()
+            self.gathered = [torch.cuda.Event() for _ in self.chunks]
+            self.drained = [torch.cuda.Event() for _ in self.chunks]
+            self.first = True
+            self.h2d_bytes = small_in + big_out
         else:
             self.h2d_bytes = small_in + sum(size(x) for x in self.k_src_h + self.v_src_h) + \
                 (size(self.hidden_h) if self.hidden_h is not None else 0)
@@ -360,6 +377,25 @@ class HostState:
                                 pos_out=st.pos_out)
             if self.tables is not None:
                 civic.civic_compact_kv(self.tables, st.seq_idx)
+        elif self.mode == "pipelined":
+            import torch
+
+            main = torch.cuda.current_stream()
+            civic.civic_select_seq(st.scores, st.desc, wl.seq_len, wl.text_before, keep_idx=st.keep, seq_idx=st.seq_idx)
+            civic.civic_compact(self.hidden_h, st.pos, st.keep, hidden_out=self.hidden_out_h, pos_out=st.pos_out)
+            for c, ls in enumerate(self.chunks):
+                if not self.first:
+                    main.wait_event(self.drained[c])  # the previous step's copy of this chunk has left the buffers
+                civic.civic_compact_kv(self.chunk_tables[c], st.seq_idx)
+                self.gathered[c].record(main)
+                with torch.cuda.stream(self.copy_stream):
+                    self.copy_stream.wait_event(self.gathered[c])
+                    for l in ls:
+                        self.k_dst_h[l].copy_(st.k_dst[l], non_blocking=True)
+                        self.v_dst_h[l].copy_(st.v_dst[l], non_blocking=True)
+                    self.drained[c].record(self.copy_stream)
+            self.first = False
+            main.wait_stream(self.copy_stream)
         else:
             if self.hidden_h is not None:
                 st.hidden.copy_(self.hidden_h, non_blocking=True)
@@ -878,7 +914,7 @@ def run_civic(args):
     if not args.no_e2e and default_variant:
         n_e2e = max(1, args.e2e_steps)
         modes = {}
-        for mode in ("zero_copy", "staged"):
+        for mode in ("zero_copy", "staged") + (("pipelined",) if wl.n_layers else ()):
             hs = HostState(st, mode)
             hs.step()
             barrier()
@@ -896,14 +932,18 @@ def run_civic(args):
                            "ms_per_step": ms_e2e, "h2d_bytes_per_step": hs.h2d_bytes,
                            "d2h_bytes_per_step": hs.d2h_bytes, "results_match_device_path": ok}
             del hs
-        best = "zero_copy"
+        best = min((m for m in modes if m != "staged"), key=lambda m: modes[m]["ms_per_step"])
         e2e = {"value": modes[best]["value"], "unit": UNIT,
                "h2d_bytes_per_step": modes[best]["h2d_bytes_per_step"],
                "d2h_bytes_per_step": modes[best]["d2h_bytes_per_step"],
                "ms_per_step": modes[best]["ms_per_step"], "steps": n_e2e, "mode": best,
-               "how": "the C-ABI calls get pinned host pointers for hidden and K/V sources and results: "
-                      "the kernels pull only the kept rows over PCIe and write the compacted rows straight "
-                      "to host memory; scores and pos ids are copied in, indices copied out",
+               "zero_copy_how": "the C-ABI calls get pinned host pointers for hidden and K/V sources and results: "
+                                "the kernels pull only the kept rows over PCIe and write the compacted rows straight "
+                                "to host memory; scores and pos ids are copied in, indices copied out",
+               "zero_copy": modes["zero_copy"], "pipelined": modes.get("pipelined"),
+               "pipelined_how": "as zero-copy for the reads, but the K/V kernel writes into device buffers two layers "
+                                "per launch and a second stream copies each finished chunk to pinned host memory "
+                                "while the kernel reads the next",
                "staged": modes["staged"],
                "staged_how": "cudaMemcpyAsync of every input to the device, device-resident path, "
                              "cudaMemcpyAsync of every result back",
