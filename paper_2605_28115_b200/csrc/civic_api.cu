@@ -353,6 +353,17 @@ civic_status_t launch_large(const float* scores, int32_t n_seg, const civic_sele
     return CIVIC_OK;
 }
 
+// Regions that get a shared-memory slot for their maximum (floor of one token per region): all of
+// them if they are few enough and the segment leaves the room, else none (the floor then walks
+// the tiles).
+int32_t select_floor_slots(const civic_select_desc_t& d, int64_t n)
+{
+    if (d.floor_per_region != 1) return 0;
+    const int64_t n_reg = (int64_t)d.t * ((d.h + d.region_h - 1) / d.region_h) * ((d.w + d.region_w - 1) / d.region_w);
+    if (n_reg > civic::kMaxFloorSlots || civic::select_smem_bytes((int)n, (int)n_reg) > kMaxDynamicSmem) return 0;
+    return (int32_t)n_reg;
+}
+
 int select_threads(int64_t n)
 {
     const int64_t threads = (n + 31) / 32 * 32;
@@ -381,16 +392,16 @@ civic_status_t select_impl(const float* scores, int32_t n_seg, const civic_selec
     p.scores = scores;
     p.keep_idx = keep_idx;
     p.shape = civic::SegShape{(int32_t)n, desc->t, desc->h, desc->w, desc->region_h, desc->region_w,
-                              desc->floor_per_region, desc->k, (int32_t)(desc->k - n_res)};
+                              desc->floor_per_region, desc->k, (int32_t)(desc->k - n_res),
+                              select_floor_slots(*desc, n)};
     p.seq_idx = seq_idx;
     p.seq_len = seq_len;
     p.vis_start = vis_start;
 
-    const size_t smem = civic::select_smem_bytes(p.shape.n);
+    const size_t smem = civic::select_smem_bytes(p.shape.n, p.shape.floor_slots);
     {
         static std::atomic<int> smem_allowed[64];
-        const civic_status_t as = allow_dynamic_smem(civic::select_kernel,
-                                                     civic::select_smem_bytes(civic_select_max_tokens()), smem_allowed);
+        const civic_status_t as = allow_dynamic_smem(civic::select_kernel, kMaxDynamicSmem, smem_allowed);
         if (as != CIVIC_OK) return as;
     }
     const int threads = select_threads(p.shape.n);
@@ -1084,22 +1095,23 @@ civic_status_t civic_select_ragged(const float* scores, int32_t n_seg, const civ
         p.keep_idx = keep_idx;
         p.flat_idx = flat_idx;
         int32_t n_max = 1;
+        size_t smem_max = 0;
         for (int s = 0; s < ns; ++s) {
             const civic_select_desc_t& d = descs[s0 + s];
             const int32_t n = d.t * d.h * d.w;
             p.shape[s] = civic::SegShape{n, d.t, d.h, d.w, d.region_h, d.region_w, d.floor_per_region, d.k,
-                                         (int32_t)(d.k - reserved_count(d))};
+                                         (int32_t)(d.k - reserved_count(d)), select_floor_slots(d, n)};
+            smem_max = std::max(smem_max, civic::select_smem_bytes(n, p.shape[s].floor_slots));
             p.score_off[s] = score_off;
             p.out_off[s] = out_off;
             score_off += n;
             out_off += d.k;
             n_max = n > n_max ? n : n_max;
         }
-        const size_t smem = civic::select_smem_bytes(n_max);
+        const size_t smem = smem_max;
         {
             static std::atomic<int> smem_allowed[64];
-            const civic_status_t as = allow_dynamic_smem(
-                civic::select_ragged_kernel, civic::select_smem_bytes(civic_select_max_tokens()), smem_allowed);
+            const civic_status_t as = allow_dynamic_smem(civic::select_ragged_kernel, kMaxDynamicSmem, smem_allowed);
             if (as != CIVIC_OK) return as;
         }
         CIVIC_CUDA_TRY(civic::launch(programmatic(), civic::select_ragged_kernel, (unsigned)ns,

@@ -4,9 +4,13 @@
 // Steps (all integer work on the fp32 bit patterns):
 //   1. key transform   monotone map fp32 -> uint32, so that unsigned key order equals
 //                      IEEE-754 totalOrder on the scores;
+//                      the same sweep counts every token's leading digit and, for m = 1, raises
+//                      its region's maximum (key, lowest index) with one shared-memory atomic;
 //   2. floor           a token is reserved iff fewer than m tokens of its region beat it
-//                      (higher key, or equal key and lower index);
-//   3. radix select    over the non-reserved tokens, up to 4 passes of 8 bits from the top:
+//                      (higher key, or equal key and lower index); a reserved token leaves the
+//                      digit count again;
+//   3. radix select    over the non-reserved tokens, up to 4 passes of 8 bits from the top (the
+//                      first pass only scans the counts of step 1):
 //                      the key T of the k'-th best (as many leading bits as are needed to tell
 //                      it apart) and how many tokens equal to T in those bits are still
 //                      needed (k' = k - number reserved);
@@ -28,7 +32,12 @@ struct SegShape {
     int32_t m;       // floor per region
     int32_t k;       // kept per segment
     int32_t k_fill;  // k - reserved count (>= 0), shape-only
+    int32_t floor_slots;  // m == 1 only: number of regions if their maxima get shared-memory slots, else 0
 };
+
+// Regions whose maxima may get a shared-memory slot each (8 bytes): beyond that, and where the
+// segment leaves no room, the floor walks every region's tile with one thread.
+constexpr int kMaxFloorSlots = 8192;
 
 struct SelectParams {
     const float* scores;  // [n_seg, n]
@@ -50,13 +59,22 @@ struct RaggedParams {
     int32_t out_off[kMaxRaggedSegs];
 };
 
-__host__ __device__ inline size_t select_smem_bytes(int n)
+__host__ __device__ inline size_t select_smem_bytes(int n, int floor_slots = 0)
 {
     const size_t words = (size_t)(n + 31) / 32;
     // one 256-bin histogram per radix pass | per-warp totals (32) | 4 scalars | reserved bit
-    // words | keys
-    return (4 * 256 + 32 + 4 + words + words * 32) * sizeof(uint32_t);
+    // words | keys | (8-byte aligned) one 64-bit slot per region
+    const size_t base = (4 * 256 + 32 + 4 + words + words * 32 + 1) / 2 * 2;
+    return (base + 2 * (size_t)floor_slots) * sizeof(uint32_t);
 }
+
+// floor(a / d) for a, d < 2^16 by one multiplication: with M = floor(2^32 / d) + 1 the product a M
+// exceeds a 2^32 / d by less than a / 2^32 < 2^-16 <= 1 / d, which cannot reach the next integer.
+struct SmallDivisor {
+    uint32_t m;  // 0: divisor 1
+    __device__ explicit SmallDivisor(uint32_t d) : m(d <= 1 ? 0u : 0xFFFFFFFFu / d + 1u) {}
+    __device__ __forceinline__ uint32_t div(uint32_t a) const { return m ? __umulhi(a, m) : a; }
+};
 
 __device__ __forceinline__ uint32_t score_key(float s)
 {
@@ -88,17 +106,58 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
     release_next_kernel();
     wait_for_prior_kernels();
 
-    // 1. keys; clear the histograms and the reserved bits
-    for (int i = tid; i < n_pad; i += nt) keys[i] = i < n ? score_key(__ldg(scores + i)) : 0u;
+    const bool fast_floor = d.floor_slots > 0;  // m == 1 and a slot per region
+    const bool fill = d.k_fill > 0;
+    unsigned long long* slots = reinterpret_cast<unsigned long long*>(smem + ((4 * 256 + 32 + 4 + n_words + n_pad + 1) & ~1));
+    const int n_rh = (d.h + d.region_h - 1) / d.region_h, n_rw = (d.w + d.region_w - 1) / d.region_w;
+    const int n_reg = d.t * n_rh * n_rw;
+
+    // 0. the first scores are requested before anything else; clear the histograms, the reserved
+    // bits and the regions' slots meanwhile
+    constexpr int kPre = 4;
+    float pre[kPre];
+#pragma unroll
+    for (int u = 0; u < kPre; ++u) pre[u] = tid + u * nt < n ? __ldg(scores + tid + u * nt) : 0.f;
     for (int b = tid; b < 4 * 256; b += nt) hist[b] = 0u;
     for (int i = tid; i < n_words; i += nt) resv[i] = 0u;
+    if (fast_floor)
+        for (int r = tid; r < n_reg; r += nt) slots[r] = 0ull;
+    __syncthreads();
+
+    // 1. keys; every token is counted under its leading digit (the reserved ones leave again in
+    // step 2); with a slot per region the token also raises its region's maximum: key in the upper
+    // half, the complement of the index in the lower, so that equal keys go to the lowest index
+    const SmallDivisor by_hw((uint32_t)(d.h * d.w)), by_w((uint32_t)d.w);
+    const SmallDivisor by_rh((uint32_t)min(d.region_h, d.h)), by_rw((uint32_t)min(d.region_w, d.w));
+    auto take = [&](int i, float score) {
+        const uint32_t key = i < n ? score_key(score) : 0u;
+        keys[i] = key;
+        if (i < n) {
+            if (fill) atomicAdd(&hist[key >> 24], 1u);
+            if (fast_floor) {
+                const uint32_t tt = by_hw.div((uint32_t)i), rem = (uint32_t)i - tt * (uint32_t)(d.h * d.w);
+                const uint32_t hh = by_w.div(rem), ww = rem - hh * (uint32_t)d.w;
+                const uint32_t r = (tt * (uint32_t)n_rh + by_rh.div(hh)) * (uint32_t)n_rw + by_rw.div(ww);
+                atomicMax(&slots[r], ((unsigned long long)key << 32) | (0xFFFFFFFFu - (uint32_t)i));
+            }
+        }
+    };
+#pragma unroll
+    for (int u = 0; u < kPre; ++u)
+        if (tid + u * nt < n_pad) take(tid + u * nt, pre[u]);
+    for (int i = tid + kPre * nt; i < n_pad; i += nt) take(i, i < n ? __ldg(scores + i) : 0.f);
     __syncthreads();
 
     // 2. floor
-    if (d.m == 1) {
+    if (fast_floor) {
+        for (int r = tid; r < n_reg; r += nt) {
+            const unsigned long long top = slots[r];
+            const uint32_t best = 0xFFFFFFFFu - (uint32_t)top;
+            atomicOr(&resv[best >> 5], 1u << (best & 31));
+            if (fill) atomicSub(&hist[(uint32_t)(top >> 56)], 1u);
+        }
+    } else if (d.m == 1) {
         // one thread per region walks its tile in index order and keeps the first maximum
-        const int n_rh = (d.h + d.region_h - 1) / d.region_h, n_rw = (d.w + d.region_w - 1) / d.region_w;
-        const int n_reg = d.t * n_rh * n_rw;
         for (int r = tid; r < n_reg; r += nt) {
             const int tt = r / (n_rh * n_rw), rem = r - tt * (n_rh * n_rw);
             const int ry = rem / n_rw, rx = rem - ry * n_rw;
@@ -114,6 +173,7 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
                 }
             }
             atomicOr(&resv[best >> 5], 1u << (best & 31));
+            if (fill) atomicSub(&hist[best_key >> 24], 1u);
         }
     } else if (d.m > 1) {
         // general m: a token is reserved iff fewer than m tokens of its tile beat it
@@ -136,6 +196,7 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
                     }
                 }
                 r = better < d.m;
+                if (r && fill) atomicSub(&hist[mine >> 24], 1u);
             }
             const uint32_t word = __ballot_sync(0xFFFFFFFFu, r);
             if (lane == 0) resv[i >> 5] = word;
@@ -153,16 +214,18 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
             uint32_t* h = hist + 256 * pass;
-            for (int i = tid; i < n_pad; i += nt) {
-                const uint32_t key = keys[i];
-                const bool cand = i < n && !((resv[i >> 5] >> (i & 31)) & 1u) && (key & mask) == prefix;
-                const uint32_t digit = (key >> shift) & 0xFFu;
-                // plain shared-memory atomics: on B200 they measured faster than aggregating
-                // equal digits per warp first (8 ballots + popc, or match.any), even when every
-                // candidate of the block falls into one bin
-                if (cand) atomicAdd(&h[digit], 1u);
+            if (pass > 0) {  // the leading digit was counted in steps 1 and 2
+                for (int i = tid; i < n_pad; i += nt) {
+                    const uint32_t key = keys[i];
+                    const bool cand = i < n && !((resv[i >> 5] >> (i & 31)) & 1u) && (key & mask) == prefix;
+                    const uint32_t digit = (key >> shift) & 0xFFu;
+                    // plain shared-memory atomics: on B200 they measured faster than aggregating
+                    // equal digits per warp first (8 ballots + popc, or match.any), even when every
+                    // candidate of the block falls into one bin
+                    if (cand) atomicAdd(&h[digit], 1u);
+                }
+                __syncthreads();
             }
-            __syncthreads();
             if (warp == 0) {
                 // lane l owns bins 8l .. 8l+7; lanes are scanned from the top bin downwards
                 const uint4 lo = reinterpret_cast<const uint4*>(h)[2 * lane];
