@@ -5,22 +5,20 @@
 // R [m_e, s] assigns the m_e compact tokens to s memory anchors; Rbar is R with every column
 // divided by its sum.  The compression is a GEMM of the persistent template (CompressOp in
 // aggregate.cuh), one launch for K and V together.  This file holds the preparation of R and the
-// attention itself: one block per (range of query tiles, head, image).  With at most 256 memory
-// anchors a head's whole K_c and V_c fit in shared memory and stay there while the block walks
-// its tiles of 128 queries; per tile there are two MMA chains and one softmax between them,
-// with no running maximum to maintain:
-//   TMA      K_c[:, head] [s, d] (K-major) and V_c[:, head] [s, d] (MN-major) once; Q tiles
-//            [128, d] into a ring of two
-//   MMA 1    S = Q K_c^T -> TMEM columns [0, s)
-//   softmax  thread per query row: maximum, exp2, row sum; P cut to bf16 and packed straight back
-//            into TMEM, columns [0, s / 2), behind the thread's own reads of S
-//   MMA 2    O = P V_c with the A operand read from TMEM -> TMEM columns [s / 2, s / 2 + d).
-//            (With P in shared memory this chain was bound by shared-memory reads: 4 KB of P
-//            for every 2 KB of V_c and only 64 or 128 output columns to amortise them.)
-//   store    O / row sum as bf16, staged in swizzled shared memory, one bulk tensor store of
-//            32 rows per warp
-// A block is a serial chain; two blocks share an SM (shared memory and tensor memory allow it
-// for 64-wide heads) and fill each other's waits.  Every wait is bounded as in aggregate.cuh.
+// attention itself: ONE PERSISTENT BLOCK PER SM that walks a contiguous share of all (image, head,
+// query tile) triples.  Per tile of 128 queries there are two MMA chains and one softmax between
+// them, with no running maximum to maintain; the block's warps form a pipeline over the tiles:
+//   TMA      K_c[:, head] [s, d] (K-major) and V_c[:, head] [s, d] (MN-major) whenever the (head,
+//            image) pair changes, into the other shared-memory slot; Q tiles [128, d] into a ring
+//   MMA 1    S = Q K_c^T into one of two tensor-memory buffers (the tile ahead of the softmax)
+//   softmax  two warps per query row, each with half of the anchors: maximum, exp2, row sum; P cut
+//            to bf16 and packed straight back into tensor memory behind the warp's own reads of S
+//   MMA 2    O = P V_c with the A operand read from tensor memory, into the columns between the
+//            two halves of P.  (With P in shared memory this chain was bound by shared-memory
+//            reads: 4 KB of P for every 2 KB of V_c and only 64 or 128 output columns to amortise.)
+//   output   O / row sum as bf16, staged in swizzled shared memory, one bulk tensor store per
+//            32 rows x 32 columns; the buffer then takes the scores of the tile after next
+// Every wait is bounded as in aggregate.cuh.
 #pragma once
 #include "aggregate.cuh"
 
@@ -187,8 +185,7 @@ __host__ __device__ constexpr uint32_t attn_tile_cols(int d_pad, int s)
 __host__ __device__ constexpr int attn_buffers(int d_pad, int s) { return attn_tile_cols(d_pad, s) <= 256 ? 2 : 1; }
 __host__ __device__ constexpr uint32_t attn_tmem_cols(int d_pad, int s)
 {
-    return attn_buffers(d_pad, s) == 2 ? 2 * (attn_tile_cols(d_pad, s) < 32u ? 32u : attn_tile_cols(d_pad, s))
-                                       : attn_tile_cols(d_pad, s);
+    return attn_buffers(d_pad, s) * attn_tile_cols(d_pad, s);
 }
 // 32-column chunks of the output; an output warp stages at most two of them at a time for its 32 rows
 __host__ __device__ constexpr int attn_out_chunks(int d) { return (d + 31) / 32; }
@@ -253,7 +250,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) kv_attention_kernel(const __g
     const int g0 = (int)((long long)p.total_tiles * blockIdx.x / gridDim.x);
     const int n_tiles = (int)((long long)p.total_tiles * (blockIdx.x + 1) / gridDim.x) - g0;
     volatile int* abort = &sy.abort;
-    const uint32_t tile_cols = attn_tile_cols(d_pad, s) < 32u ? 32u : attn_tile_cols(d_pad, s);
+    const uint32_t tile_cols = attn_tile_cols(d_pad, s);
     const uint32_t tmem_cols = attn_tmem_cols(d_pad, s);
     const uint32_t o_col = attn_o_col(d_pad, s);
     const int half_s = s >> 1;
