@@ -105,6 +105,9 @@ def check(q, k, v, r, heads):
     (2, 130, 2, 112, 192),   # 64 + 48 columns
     (1, 70, 5, 8, 64),       # the narrowest head
     (1, 90, 2, 120, 256),    # 128-wide storage of a 120-wide head
+    (2, 1300, 8, 128, 512),  # streamed V_c with more tiles than SMs: blocks walk two tiles, some across two heads
+    (1, 700, 30, 128, 320),  # the same with five blocks of anchors and one K_c slot reloaded per head
+    (40, 128, 4, 64, 256),   # one query tile per (head, image): every tile of a block starts a new pair
 ])
 def test_against_oracle(n_img, m_e, heads, d, s):
     q, k, v, r = inputs(n_img, m_e, heads, d, s, seed=m_e + s)
