@@ -692,8 +692,8 @@ def time_aggregate(w, dev, steps, warm):
     burst, sustained, which = measured_tensor_peak()
     timed_s = ms * 1e-3 * steps
     peak = sustained if timed_s > 0.5 else burst  # a long loop runs under the power cap
-    roofline = {"bound": "tensor", "kernel": "civic_anchor_aggregate_prepared: five launches, of which the two tcgen05 "
-                "contractions carry all the flops (the other three are HBM-bound helpers and are inside the time)",
+    roofline = {"bound": "tensor", "kernel": "civic_anchor_aggregate_prepared: four launches, of which the two tcgen05 "
+                "contractions carry all the flops (the other two are memory-bound helpers and are inside the time)",
                 "achieved": value, "peak": peak, "unit": "TFLOP/s", "frac": value / peak, "peak_source": which,
                 "peak_kind": "sustained" if timed_s > 0.5 else "burst", "frac_of_burst_peak": value / burst,
                 "traffic": None, "algorithmic_flops_per_step": w.flops, "us_per_step": ms * 1e3}

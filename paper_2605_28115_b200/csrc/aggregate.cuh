@@ -15,12 +15,14 @@
 //                           -> (mu_i, r_i); one warp per row, HBM-bound
 //   aggregate_gemm_kernel<ScoresOp>   tcgen05 GEMM  S = Q_A X_0^T  (both operands K-major), epilogue
 //                           P = exp((r (S - mu qsum) - 1) / tau) as bf16 + partial row sums
-//   aggregate_gemm_kernel<ValuesOp>   tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major)
-//   token_mass_*_kernel     column sums of W_A (per-token importance), HBM-bound
+//   aggregate_gemm_kernel<ValuesOp>   tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major);
+//                           four side warps add up the columns of W_A = P / l by panels of 32 anchors
+//   token_mass_reduce_kernel   adds those panels: the per-token importance
 //
-// GEMM skeleton (both): persistent blocks of 320 threads, one per SM.  Warp 0 = TMA producer (one
-// elected lane), warp 1 = TMEM allocation + MMA issue (one elected lane), warps 2..9 = epilogue
-// (each reads its own quarter of the 128 TMEM lanes).  Operand tiles arrive by
+// GEMM skeleton (both): persistent blocks of 320 threads (448 with side warps), one per SM.  Warp 0 =
+// TMA producer (one elected lane), warp 1 = TMEM allocation + MMA issue (one elected lane), warps
+// 2..9 = epilogue (each reads its own quarter of the 128 TMEM lanes), warps 10..13 = side warps of
+// an Op that has them.  Operand tiles arrive by
 // cp.async.bulk.tensor with 128-byte swizzle into a ring of stages guarded by full/empty
 // mbarriers; two accumulators alternate in TMEM so the epilogue overlaps the next tile's MMAs.
 // The score GEMM runs on pairs of blocks (cta_group::2): with both operands in shared memory a
@@ -38,7 +40,7 @@
 
 namespace civic {
 
-constexpr int kAggThreads = 320;      // producer warp, MMA warp, eight epilogue warps
+constexpr int kAggThreads = 320;      // producer warp, MMA warp, eight epilogue warps (an Op's side warps come on top)
 constexpr int kAggBM = 128;           // anchors per tile (TMEM lanes)
 constexpr int kAggBK = 64;            // 64 bf16 = one 128-byte swizzle row
 constexpr int kScoresBN = 256;        // tokens per tile of the first GEMM
@@ -464,9 +466,11 @@ struct ValuesParams {
     const float* lpart;   // [n_img, m_e, n_parts]
     __nv_bfloat16* z;     // [n_img, m_e, d_v]
     float* inv_l;         // [n_img, m_e] written by the blocks of the first feature tile
+    float* mass_partial;  // [n_img, 4 m_tiles, t_ld] column sums of W_A by panels of 32 anchors, or null
+    const __nv_bfloat16* pw;  // [n_img, m_e, t_ld] P as global memory, for the side warps
     int* error;
     TileGrid grid;
-    int32_t m_e, t_e, d_v, n_parts;
+    int32_t m_e, t_e, d_v, n_parts, t_ld;
 };
 
 constexpr int kEpilogueWarps = 8;
@@ -478,6 +482,7 @@ struct alignas(1024) GemmSmem {
     uint8_t out[STAGING_ ? kEpilogueWarps : 1][STAGING_ ? 32 * 128 : 1024];  // per epilogue warp: 32 rows x 64 bf16, 128-byte swizzled,
                                                 // for the bulk store of a result (scores, compression)
     float2 stats[SCORES_ ? kEpilogueWarps : 1][128];  // per epilogue warp: (mu, r log2e / tau) of its columns (scores only)
+    float side_w[4][32];  // per side warp: 1 / l of its 32 anchor rows (values only)
     uint64_t full[STAGES_], empty[STAGES_], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort;
@@ -491,7 +496,7 @@ struct alignas(1024) GemmSmem {
 //                 bytes it can keep in flight, not by the tensor pipe).
 template <bool PAIR>
 struct ScoresOpT {
-    static constexpr int BN = 256, STAGES = PAIR ? 5 : 3, kCtas = PAIR ? 2 : 1;
+    static constexpr int BN = 256, STAGES = PAIR ? 5 : 3, kCtas = PAIR ? 2 : 1, kSideWarps = 0;
     static constexpr bool kAMnMajor = false, kBMnMajor = false;
     using Params = ScoresParams;
     using Smem = GemmSmem<PAIR ? 128 : 256, STAGES, true>;
@@ -649,7 +654,7 @@ __device__ __forceinline__ void values_epilogue(const ValuesParams& p, uint32_t 
 
 template <int BN_>
 struct ValuesOp {
-    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1;
+    static constexpr int BN = BN_, STAGES = BN_ == 256 ? 4 : 5, kCtas = 1, kSideWarps = 4;
     static constexpr bool kAMnMajor = false, kBMnMajor = true;
     using Params = ValuesParams;
     using Smem = GemmSmem<BN, STAGES, false>;
@@ -677,6 +682,77 @@ struct ValuesOp {
     {
         values_epilogue(p, tmem, ewarp, lane, m0, tl);
     }
+    // Token mass (column sums of W_A = P / l) on the way: while a block works on a tile of the first
+    // feature panel, four side warps add up the columns of that tile's 128 rows of P, read from global
+    // memory (the rows the block's own tensor copies fetch at about the same time, so one of the two
+    // finds them in L2) and not from the stages in shared memory, whose bandwidth is what bounds the
+    // GEMM: side warps reading the stages made the tile three times slower.  Side warp sw takes the
+    // anchors 32 sw .. 32 sw + 31; lane = 8 neighbouring tokens (16 bytes) of every fourth row.  The
+    // sums of a panel of 32 anchors go to mass_partial; a small kernel adds the panels in order.
+    static __device__ __forceinline__ bool side_active(const Params& p, const Tile& tl)
+    {
+        return p.mass_partial != nullptr;
+    }
+    static __device__ __forceinline__ void side_tile(const Params& p, Smem& sm, int sw, int lane, int m0, const Tile& tl)
+    {
+        {   // 1 / l of row m0 + 32 sw + lane: the same sum, in the same order, as the epilogue's
+            const int m = m0 + sw * 32 + lane;
+            float l = 0.f;
+            if (m < p.m_e) {
+                const float* lp = p.lpart + ((size_t)tl.img * p.m_e + m) * p.n_parts;
+                int t = 0;
+                for (; t + 8 <= p.n_parts; t += 8) {
+                    float v[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[e] = __ldg(lp + t + e);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) l += v[e];
+                }
+                for (; t < p.n_parts; ++t) l += __ldg(lp + t);
+            }
+            __syncwarp();  // the previous tile's weights have been read
+            sm.side_w[sw][lane] = l > 0.f ? 1.f / l : 0.f;
+            __syncwarp();
+        }
+        const int group = lane >> 3, c8 = (lane & 7) * 8;  // rows group, group + 4, ...; tokens c8 .. c8 + 7 of a slab
+        float w[8];
+        bool row_ok[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            w[i] = sm.side_w[sw][4 * i + group];
+            row_ok[i] = m0 + sw * 32 + 4 * i + group < p.m_e;
+        }
+        const __nv_bfloat16* rows = p.pw + ((size_t)tl.img * p.m_e + m0 + sw * 32 + group) * p.t_ld + c8;
+        float* out = p.mass_partial + ((size_t)tl.img * (4 * p.grid.m_tiles) + (m0 / kAggBM) * 4 + sw) * p.t_ld + c8;
+        // slabs of 64 tokens, dealt out over the feature tiles of this panel of anchors; t_ld is a multiple of 8
+        for (int col = tl.n_tile * 64; col < p.t_ld; col += 64 * p.grid.n_tiles) {
+            const bool col_ok = col + c8 < p.t_ld;
+            uint4 u[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                u[i] = col_ok && row_ok[i] ? __ldcs(reinterpret_cast<const uint4*>(rows + (size_t)(4 * i) * p.t_ld + col))
+                                           : make_uint4(0u, 0u, 0u, 0u);
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t x[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    acc[2 * e] = fmaf(__uint_as_float(x[e] << 16), w[i], acc[2 * e]);
+                    acc[2 * e + 1] = fmaf(__uint_as_float(x[e] & 0xFFFF0000u), w[i], acc[2 * e + 1]);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {  // the four row groups, always in the same order
+                acc[e] += __shfl_xor_sync(0xFFFFFFFFu, acc[e], 8);
+                acc[e] += __shfl_xor_sync(0xFFFFFFFFu, acc[e], 16);
+            }
+            if (group == 0 && col_ok) {
+                *reinterpret_cast<float4*>(out + col) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                *reinterpret_cast<float4*>(out + col + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+            }
+        }
+    }
 };
 
 // K_c = Rbar^T K (and V_c = Rbar^T V) of the KV-compressed attention: tile of 128 memory anchors x
@@ -699,7 +775,7 @@ struct CompressParams {
 
 template <int BN_>
 struct CompressOp {
-    static constexpr int BN = BN_, STAGES = BN_ == 128 ? 5 : 4, kCtas = 1;
+    static constexpr int BN = BN_, STAGES = BN_ == 128 ? 5 : 4, kCtas = 1, kSideWarps = 0;
     static constexpr bool kAMnMajor = true, kBMnMajor = true;
     using Params = CompressParams;
     using Smem = GemmSmem<BN, STAGES, false, true>;
@@ -814,7 +890,7 @@ struct CompressOp {
 };
 
 template <class Op>
-__global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
+__global__ void __launch_bounds__(kAggThreads + 32 * Op::kSideWarps) aggregate_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                      const __grid_constant__ CUtensorMap map_b,
                                                                      const __grid_constant__ CUtensorMap map_c,
                                                                      const __grid_constant__ CUtensorMap map_d,
@@ -927,6 +1003,15 @@ __global__ void __launch_bounds__(kAggThreads) aggregate_gemm_kernel(const __gri
             }
             __syncwarp();
         }
+    } else if (warp >= 2 + kEpilogueWarps) {
+        // ---- side warps (an Op that has them): work of their own beside the tiles, no part in the pipeline
+        if constexpr (Op::kSideWarps > 0) {
+            if (!stop) {
+                Tile tl;
+                for (int local = 0; Op::tile(p, worker, n_workers, local, tl); ++local)
+                    if (Op::side_active(p, tl)) Op::side_tile(p, sm, warp - (2 + kEpilogueWarps), lane, tl.m_tile * kAggBM, tl);
+            }
+        }
     } else if (warp >= 2 && !stop) {
         // ---- epilogue: warps 2..9; a warp may read the TMEM lane quarter (warp index mod 4)
         const int ewarp = ((warp & 3) | ((warp - 2) & 4));  // quarter in bits 0-1, column half in bit 2
@@ -984,62 +1069,12 @@ __global__ void __launch_bounds__(64) bounded_wait_selftest_kernel(unsigned long
     }
 }
 
-// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m], in two deterministic steps.
-//   token_mass_partial_kernel  a block takes a panel of kMassPanel rows of P over a slab of 256 token
-//                              columns (512 contiguous bytes per row); its eight warps take every
-//                              eighth row, and their sums are added in warp order through shared
-//                              memory;
-//   token_mass_reduce_kernel   adds the panels' sums in a fixed order.
-// Measured on 8 x 1024 x 4096 weights (us, partial + reduce): panels of 16 rows over all columns,
-// thread per 8 columns: 14.8 + 4.6; the same over slabs of 1024 columns: 12.1 + 9.5 (the reduction
-// pays for 64 panels); panels of 64 rows: 21.0 + 3.6 (too few, too long threads).
-constexpr int kMassPanel = 128;
-constexpr int kMassWarps = 8;
-__global__ void __launch_bounds__(kMassWarps * 32) token_mass_partial_kernel(const __nv_bfloat16* __restrict__ p,
-                                                                             const float* __restrict__ inv_l, int m_e,
-                                                                             int t_e, int t_ld, int n_panels,
-                                                                             float* __restrict__ partial)
-{
-    __shared__ float4 sums[kMassWarps][32][2];
-    wait_for_prior_kernels();
-    const int panel = blockIdx.x, img = blockIdx.z;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_begin = panel * kMassPanel, m_end = min(m_begin + kMassPanel, m_e);
-    const float* il = inv_l + (size_t)img * m_e;
-    // lane = 8 consecutive token columns (one 16-byte load per row); t_ld is a multiple of 8
-    const int c = blockIdx.y * 256 + lane * 8;
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (c < t_ld) {
-        const __nv_bfloat16* col = p + ((size_t)img * m_e + m_begin + warp) * t_ld + c;
-#pragma unroll 8
-        for (int m = m_begin + warp; m < m_end; m += kMassWarps, col += (size_t)kMassWarps * t_ld) {
-            const uint4 u = __ldg(reinterpret_cast<const uint4*>(col));
-            const float w = __ldg(il + m);
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 f = __bfloat1622float2(h[e]);
-                acc[2 * e] += f.x * w;
-                acc[2 * e + 1] += f.y * w;
-            }
-        }
-    }
-    sums[warp][lane][0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    sums[warp][lane][1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-    __syncthreads();
-    if (threadIdx.x < 64) {  // thread = 4 of the slab's 256 columns: the warps' sums in warp order
-        const int l = threadIdx.x >> 1, half = threadIdx.x & 1;
-        float4 t = sums[0][l][half];
-#pragma unroll
-        for (int w = 1; w < kMassWarps; ++w) {
-            const float4 v = sums[w][l][half];
-            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
-        }
-        const int col = blockIdx.y * 256 + l * 8 + half * 4;
-        if (col < t_ld) *reinterpret_cast<float4*>(partial + ((size_t)img * n_panels + panel) * t_ld + col) = t;
-    }
-}
-
+// Column sums of W_A: mass[img, i] = sum_m P[m, i] / l[m], in two deterministic steps: the side
+// warps of the value GEMM leave the sums of panels of 32 anchors (ValuesOp::side_tile), and
+// token_mass_reduce_kernel adds the panels in a fixed order.
+// A kernel of its own for the first step (a block per panel of 128 rows over a slab of 256 token
+// columns, its eight warps every eighth row) took 11.8 us on 8 x 1024 x 4096 weights, reading P from
+// global memory once more after the GEMM; beside the GEMM the same reads cost it 4.5 us.
 __global__ void __launch_bounds__(64) token_mass_reduce_kernel(const float* __restrict__ partial, int t_e, int t_ld,
                                                                 int n_panels, float* __restrict__ mass)
 {

@@ -507,7 +507,7 @@ civic_status_t plan_aggregate(int32_t n_img, int32_t t_e, int32_t m_e, int32_t d
     pl.p_off = take((size_t)n_img * m_e * pl.t_ld * 2);
     pl.lpart_off = take((size_t)n_img * m_e * 2 * pl.n_tiles_t * 4);  // two column halves per token tile
     pl.invl_off = take((size_t)n_img * m_e * 4);
-    pl.n_panels = (m_e + civic::kMassPanel - 1) / civic::kMassPanel;
+    pl.n_panels = 4 * ((m_e + civic::kAggBM - 1) / civic::kAggBM);  // panels of 32 anchors
     pl.mass_off = take((size_t)n_img * pl.n_panels * pl.t_ld * 4);  // per-panel column sums of the token mass
     pl.total = off;
     return CIVIC_OK;
@@ -531,7 +531,7 @@ civic_status_t launch_gemm(const CUtensorMap& map_a, const CUtensorMap& map_b, c
     const int workers = total_tiles < workers_max ? total_tiles : workers_max;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(workers * Op::kCtas));
-    cfg.blockDim = dim3(civic::kAggThreads);
+    cfg.blockDim = dim3((unsigned)(civic::kAggThreads + 32 * Op::kSideWarps));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -787,7 +787,9 @@ static civic_status_t aggregate_impl(const void* x0, const float* anchors, const
     if (gs != CIVIC_OK) return gs;
     civic::ValuesParams vp;
     vp.lpart = lpart; vp.z = (__nv_bfloat16*)z0; vp.inv_l = inv_l; vp.error = device_status;
-    vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t;
+    vp.m_e = m_e; vp.t_e = t_e; vp.d_v = d_v; vp.n_parts = 2 * pl.n_tiles_t; vp.t_ld = pl.t_ld;
+    vp.mass_partial = token_mass ? (float*)(ws + pl.mass_off) : nullptr;
+    vp.pw = (const __nv_bfloat16*)p;
     const int32_t f_tiles = (d_v + pl.values_bn - 1) / pl.values_bn;
     vp.grid = civic::TileGrid{m_tiles, f_tiles, n_img, m_tiles * f_tiles * n_img};
     if (pl.values_bn == 256) gs = launch_gemm<civic::ValuesOp<256>>(map_p, map_x_values, map_p, map_p, map_p, vp, vp.grid.total, stream);
@@ -797,13 +799,9 @@ static civic_status_t aggregate_impl(const void* x0, const float* anchors, const
     int n_launched = 3;
     if (token_mass) {
         float* partial = (float*)(ws + pl.mass_off);
-        CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_partial_kernel,
-                                     dim3((unsigned)pl.n_panels, (unsigned)((pl.t_ld + 255) / 256), (unsigned)n_img),
-                                     (unsigned)(civic::kMassWarps * 32), 0, stream, (const __nv_bfloat16*)p,
-                                     (const float*)inv_l, m_e, t_e, pl.t_ld, pl.n_panels, partial));
         CIVIC_CUDA_TRY(civic::launch(pdl, civic::token_mass_reduce_kernel, dim3((unsigned)((t_e + 63) / 64), (unsigned)n_img),
                                      64u, 0, stream, (const float*)partial, t_e, pl.t_ld, pl.n_panels, token_mass));
-        n_launched += 2;
+        n_launched += 1;
     }
     g_launches.fetch_add(n_launched, std::memory_order_relaxed);
     return CIVIC_OK;
