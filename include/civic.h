@@ -360,7 +360,7 @@ civic_status_t civic_compact_pos_planes(const int32_t* pos, int32_t n_planes, in
  *                its time limit (the kernels then stop cleanly and the outputs are invalid).
  *                Read it after synchronising the stream.
  * d_v must be a multiple of 64 (CIVIC_ERR_UNSUPPORTED otherwise); t_e and m_e are arbitrary.
- * Inputs must be finite.  Three launches (five with token_mass); the first one clears the status word.
+ * Inputs must be finite.  Three launches (four with token_mass); the first one clears the status word.
  */
 civic_status_t civic_anchor_aggregate(const void* x0, const float* anchors, int32_t n_img, int32_t t_e,
                                       int32_t m_e, int32_t d_v, float tau, void* z0, float* token_mass,
