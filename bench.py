@@ -597,6 +597,13 @@ def time_other_path_workload(wl, dev, steps, with_oracle):
         end.record()
         torch.cuda.synchronize()
         out["graph_replay_us_per_step"] = start.elapsed_time(end) / steps * 1e3
+        # a replay has a floor of its own (about 8 us here, whatever the graph holds): 20 steps per graph
+        with torch.cuda.stream(side):
+            graph20 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph20, stream=side):
+                for _ in range(20):
+                    st.step()
+        out["graph_of_20_steps_us_per_step"] = time_loop(graph20.replay, max(steps // 20, 20), 3) / 20
         peak, _ = measured_peak()
         out["hbm_time_us_at_measured_peak"] = nbytes["total"] / peak / 1e3
         st.step()
