@@ -107,6 +107,18 @@ def test_select_all_equal_and_degenerate_regions():
     assert_select_parity(np.zeros((3, 1), np.float32), 1, 1, 1, 1, 1, 1, 1)
 
 
+def test_select_floor_of_one_by_slots_and_by_tile_walk():
+    """m = 1 beyond one token per thread: large tiles take the regions' maxima through shared-memory slots,
+    small tiles are walked by one thread each; both with ragged edge tiles and with ties inside the tiles."""
+    rng = np.random.default_rng(7)
+    for t, h, w, rh, rw in [(1, 40, 45, 10, 10), (2, 30, 33, 9, 8), (1, 40, 45, 3, 3), (3, 25, 31, 8, 8), (1, 50, 50, 7, 9)]:
+        n = t * h * w
+        n_res = O.reserved_count(t, h, w, rh, rw, 1)
+        for s in (rng.random((2, n)), rng.integers(0, 4, (2, n)), np.exp(rng.standard_normal((2, n)) * 6)):
+            for k in (n_res, n_res + 1, (n + n_res) // 2):
+                assert_select_parity(s.astype(np.float32), t, h, w, rh, rw, 1, k)
+
+
 def test_select_threshold_decided_by_the_leading_digits():
     """Keys built so that the radix search can stop after its first, second or third digit (the threshold bin
     is wanted whole), with several different keys inside the bins that are taken whole."""
