@@ -119,6 +119,7 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
 #pragma unroll
     for (int u = 0; u < kPre; ++u) pre[u] = tid + u * nt < n ? __ldg(scores + tid + u * nt) : 0.f;
     for (int b = tid; b < 4 * 256; b += nt) hist[b] = 0u;
+    if (tid == 0) warp_tot[0] = 0u;  // OR of (key XOR the first key): the bits in which keys differ (step 1)
     for (int i = tid; i < n_words; i += nt) resv[i] = 0u;
     if (fast_floor)
         for (int r = tid; r < n_reg; r += nt) slots[r] = 0ull;
@@ -129,10 +130,13 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
     // half, the complement of the index in the lower, so that equal keys go to the lowest index
     const SmallDivisor by_hw((uint32_t)(d.h * d.w)), by_w((uint32_t)d.w);
     const SmallDivisor by_rh((uint32_t)min(d.region_h, d.h)), by_rw((uint32_t)min(d.region_w, d.w));
+    const uint32_t key0 = score_key(__ldg(scores));  // n >= 1
+    uint32_t differ = 0u;
     auto take = [&](int i, float score) {
         const uint32_t key = i < n ? score_key(score) : 0u;
         keys[i] = key;
         if (i < n) {
+            differ |= key ^ key0;
             if (fill) atomicAdd(&hist[key >> 24], 1u);
             if (fast_floor) {
                 const uint32_t tt = by_hw.div((uint32_t)i), rem = (uint32_t)i - tt * (uint32_t)(d.h * d.w);
@@ -146,6 +150,10 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
     for (int u = 0; u < kPre; ++u)
         if (tid + u * nt < n_pad) take(tid + u * nt, pre[u]);
     for (int i = tid + kPre * nt; i < n_pad; i += nt) take(i, i < n ? __ldg(scores + i) : 0.f);
+    if (fill) {
+        differ = __reduce_or_sync(0xFFFFFFFFu, differ);
+        if (lane == 0 && differ) atomicOr(&warp_tot[0], differ);
+    }
     __syncthreads();
 
     // 2. floor
@@ -204,21 +212,27 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
     }
     __syncthreads();
 
-    // 3. radix select of the k_fill-th best non-reserved key, 8 bits per pass from the top
+    // 3. radix select of the k_fill-th best non-reserved key, 8 bits per pass from the top, down to
+    // the lowest bit in which the segment's keys differ at all: the bits below it are the same in
+    // every key and decide nothing (scores quantised to a few levels have constant low mantissa
+    // bits, whose passes would count every candidate into one bin and sweep the tokens for nothing).
     uint32_t prefix = 0xFFFFFFFFu, mask = 0xFFFFFFFFu, need_eq = 0;
     if (d.k_fill > 0) {
         mask = 0;
         uint32_t rank = (uint32_t)d.k_fill;  // 1-based rank among the candidates still matching
         prefix = 0;
+        const uint32_t any_differ = warp_tot[0];
+        const int win_lo = any_differ ? __ffs(any_differ) - 1 : 32;  // all keys equal: the leading digit alone
 #pragma unroll 1
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
+        for (int pass = 0; pass == 0 || 32 - 8 * pass > win_lo; ++pass) {
+            const int shift = pass == 0 ? 24 : max(24 - 8 * pass, win_lo);
+            const uint32_t digit_mask = (1u << (32 - 8 * pass - shift)) - 1u;
             uint32_t* h = hist + 256 * pass;
             if (pass > 0) {  // the leading digit was counted in steps 1 and 2
                 for (int i = tid; i < n_pad; i += nt) {
                     const uint32_t key = keys[i];
                     const bool cand = i < n && !((resv[i >> 5] >> (i & 31)) & 1u) && (key & mask) == prefix;
-                    const uint32_t digit = (key >> shift) & 0xFFu;
+                    const uint32_t digit = (key >> shift) & digit_mask;
                     // plain shared-memory atomics: on B200 they measured faster than aggregating
                     // equal digits per warp first (8 ballots + popc, or match.any), even when every
                     // candidate of the block falls into one bin
@@ -253,7 +267,7 @@ __device__ __forceinline__ void select_block(const SegShape& d, const float* __r
             }
             __syncthreads();
             prefix |= scal[0] << shift;
-            mask |= 0xFFu << shift;
+            mask |= digit_mask << shift;
             rank = scal[1];
             // Every candidate that still matches the prefix is wanted: the lower bits cannot change
             // the outcome, so the remaining passes are skipped (with continuous scores the bin of
