@@ -540,31 +540,36 @@ __global__ void __launch_bounds__(kAttnThreads, 1) kv_attention_kernel(const __g
             const uint32_t tm = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * tile_cols;
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(&sy.o_done[buf], (i / n_buf) & 1, abort, p.error, kAggTimeoutAcc))) break;
             tc_fence_after_sync();
-            uint32_t acc[32];
-            tmem_load_issue(tm + o_col, acc);
             const int row = quarter * 32 + lane;
             const float inv = 1.f / (sy.row_sum[buf][0][row] + sy.row_sum[buf][1][row]);  // the largest term is about 1
             for (int c0 = 0; c0 < out_chunks; c0 += 2) {  // two chunks per round through the staging rows
+                const int c_end = min(c0 + 2, out_chunks);
+                // both chunks of the round are asked for at once; with the last one in registers the
+                // buffer may take the scores of the tile after next
+                uint32_t acc[2][32];
+                tmem_load_issue(tm + o_col + 32 * c0, acc[0]);
+                if (c0 + 1 < c_end) tmem_load_issue(tm + o_col + 32 * (c0 + 1), acc[1]);
+                tmem_load_wait(acc[0]);
+                if (c0 + 1 < c_end) tmem_load_wait(acc[1]);
+                if (c_end == out_chunks) {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sy.s_free[buf]);
+                }
                 if (lane == 0) tma_store_wait_read();  // the previous round's stores have read the staging rows
                 __syncwarp();
-                const int c_end = min(c0 + 2, out_chunks);
-                for (int c = c0; c < c_end; ++c) {
-                    tmem_load_wait(acc);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int c = c0 + u;
+                    if (c >= c_end) break;
                     uint32_t w[16];
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[2 * e]) * inv,
-                                                                       __uint_as_float(acc[2 * e + 1]) * inv);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[u][2 * e]) * inv,
+                                                                       __uint_as_float(acc[u][2 * e + 1]) * inv);
                         w[e] = *reinterpret_cast<const uint32_t*>(&h);
                     }
-                    if (c + 1 < out_chunks) {
-                        tmem_load_issue(tm + o_col + 32 * (c + 1), acc);
-                    } else {  // all of O is in registers: the buffer may take the scores of the tile after next
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sy.s_free[buf]);
-                    }
-                    uint8_t* box = o_stage + (c - c0) * 2048;
+                    uint8_t* box = o_stage + u * 2048;
                     if (c < full_chunks) {  // 32 rows x 64 B, 64-byte swizzle: piece j of row r at j ^ ((r >> 1) & 3)
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
