@@ -11,8 +11,8 @@
 // P = exp((s - 1) / tau) cannot overflow and, for tau >= 0.025, cannot underflow bf16.
 //
 // Kernels
-//   aggregate_prep_kernel   A (fp32) -> Q_A (bf16) and the row sums of the rounded values; X_0 (bf16)
-//                           -> (mu_i, r_i); one warp per row, HBM-bound
+//   aggregate_prep_kernel   A (fp32) -> Q_A (bf16) and the row sums of the rounded values, a warp per
+//                           anchor; X_0 (bf16) -> (mu_i, r_i), eight lanes per token; HBM-bound
 //   aggregate_gemm_kernel<ScoresOp>   tcgen05 GEMM  S = Q_A X_0^T  (both operands K-major), epilogue
 //                           P = exp((r (S - mu qsum) - 1) / tau) as bf16 + partial row sums
 //   aggregate_gemm_kernel<ValuesOp>   tcgen05 GEMM  Z_0 = (P X_0) / l  (A = P K-major, B = X_0 MN-major);
@@ -255,12 +255,12 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n, int b_mn_major, int m =
 
 // ----------------------------------------------------------------------------- small kernels
 
-// Both preparations in one launch, one warp per row.  Warps [0, m_e) take an anchor each:
-// Q_A = Norm(LN(A)) rounded to bf16, and qsum[m] = sum of the ROUNDED row (what the tensor core
-// will really multiply the token mean with).  The other warps take a token each: (mu_i, r_i)
-// with K_0[i] = r_i (x_i - mu_i), r_i = 0 for a token whose features are all equal.  Few
-// registers on purpose: the token part is HBM-bound and lives on occupancy (a version that held
-// the whole row in registers measured slower).
+// Both preparations in one launch.  Warps [0, m_e) take an anchor each: Q_A = Norm(LN(A)) rounded
+// to bf16, and qsum[m] = sum of the ROUNDED row (what the tensor core will really multiply the token
+// mean with).  The other warps take 32 / kPrepLanes tokens each: (mu_i, r_i) with
+// K_0[i] = r_i (x_i - mu_i), r_i = 0 for a token whose features are all equal.  Few registers on
+// purpose: the token part is HBM-bound and lives on occupancy (a version that held the whole row in
+// registers measured slower).
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll
@@ -276,10 +276,11 @@ __device__ __forceinline__ float normalise_scale(float ss, int d_v, float ln_eps
     return ss > 0.f ? inv_std / fmaxf(norm, norm_eps) : 0.f;
 }
 
-// Token rows per warp and loads in flight per row: one row and four 16-byte loads per lane measured
-// fastest on B200 (18.3 us for 75 MB; two or four rows per warp 20 .. 29 us, deeper unrolling 22 us).
-constexpr int kPrepRows = 1;
-constexpr int kPrepUnroll = 4;
+// Token part: lanes per row and 16-byte loads in flight per lane.  Measured on 32768 rows of 1152 bf16
+// (75 MB), us: 32 lanes x 5 loads 17.8 - 25.8, 16 x 5 17.1, 16 x 9 15.7, 8 x 6 13.0 (5.8 TB/s), 8 x 18 13.0,
+// 4 x 9 16.0, 2 x 9 21.5.
+constexpr int kPrepLanes = 8;
+constexpr int kPrepUnroll = 6;
 __global__ void __launch_bounds__(256) aggregate_prep_kernel(const float* __restrict__ anchors, int m_e,
                                                              const __nv_bfloat16* __restrict__ x, long long n_tokens,
                                                              int d_v, float ln_eps, float norm_eps,
@@ -309,47 +310,42 @@ __global__ void __launch_bounds__(256) aggregate_prep_kernel(const float* __rest
         if (lane == 0) qsum[warp] = rounded_sum;
         return;
     }
-    // ---- token rows (bf16, d_v a multiple of 8): a warp takes kPrepRows consecutive rows, their
-    // 16-byte loads interleaved; sums are taken relative to the row's first element so that the
-    // variance keeps its accuracy
-    const long long tok0 = (warp - m_e) * kPrepRows;
-    if (tok0 >= n_tokens) return;
+    // ---- token rows (bf16, d_v a multiple of 8): kPrepLanes lanes per row, so that a warp's fixed work
+    // (the two reductions, the normalisation, the addressing: 40 % of its instructions with a row per
+    // warp, and the pass was bound by instruction issue at 45 % of the DRAM rate) serves four rows, and
+    // no lane idles in a last partial iteration (1152 features are 4.5 loads of 16 bytes per lane of a
+    // whole warp).  Sums are taken relative to the row's first element so that the variance keeps its
+    // accuracy.
+    const long long tok_first = (warp - m_e) * (32 / kPrepLanes);
+    if (tok_first >= n_tokens) return;  // the whole warp: nothing below touches x without a token (x may be null)
+    const long long tok = tok_first + lane / kPrepLanes;
+    const bool tok_ok = tok < n_tokens;  // past the end: the warp's first row again, not stored
+    const int l16 = lane % kPrepLanes;
     const int vecs = d_v >> 3;
-    const uint4* row[kPrepRows];
-    float shift[kPrepRows], s[kPrepRows], s2[kPrepRows];
-#pragma unroll
-    for (int r = 0; r < kPrepRows; ++r) {
-        const long long tok = tok0 + r < n_tokens ? tok0 + r : tok0;  // past the end: the first row again, not stored
-        row[r] = reinterpret_cast<const uint4*>(x + tok * d_v);
-        shift[r] = __bfloat162float(x[tok * d_v]);
-        s[r] = 0.f;
-        s2[r] = 0.f;
-    }
+    const uint4* row = reinterpret_cast<const uint4*>(x + (tok_ok ? tok : tok_first) * d_v);
+    const float shift = __bfloat162float(x[(tok_ok ? tok : tok_first) * d_v]);
+    float s = 0.f, s2 = 0.f;
 #pragma unroll kPrepUnroll
-    for (int v = lane; v < vecs; v += 32) {
-        uint4 u[kPrepRows];
+    for (int v = l16; v < vecs; v += kPrepLanes) {
+        const uint4 u = __ldg(row + v);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-        for (int r = 0; r < kPrepRows; ++r) u[r] = __ldg(row[r] + v);
-#pragma unroll
-        for (int r = 0; r < kPrepRows; ++r) {
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[r]);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 f = __bfloat1622float2(h[e]);
-                const float a = f.x - shift[r], b = f.y - shift[r];
-                s[r] += a + b;
-                s2[r] += a * a + b * b;
-            }
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            const float a = f.x - shift, b = f.y - shift;
+            s += a + b;
+            s2 += a * a + b * b;
         }
     }
 #pragma unroll
-    for (int r = 0; r < kPrepRows; ++r) {
-        const float sum = warp_sum(s[r]), sum2 = warp_sum(s2[r]);
-        if (lane == 0 && tok0 + r < n_tokens) {
-            const float mean_shifted = sum / d_v;
-            const float ss = fmaxf(sum2 - sum * mean_shifted, 0.f);  // sum (x - mu)^2
-            stats[tok0 + r] = make_float2(mean_shifted + shift[r], normalise_scale(ss, d_v, ln_eps, norm_eps));
-        }
+    for (int d = kPrepLanes / 2; d > 0; d >>= 1) {  // within the row's lanes
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+        s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, d);
+    }
+    if (l16 == 0 && tok_ok) {
+        const float mean_shifted = s / d_v;
+        const float ss = fmaxf(s2 - s * mean_shifted, 0.f);  // sum (x - mu)^2
+        stats[tok] = make_float2(mean_shifted + shift, normalise_scale(ss, d_v, ln_eps, norm_eps));
     }
 }
 

@@ -769,7 +769,8 @@ static civic_status_t aggregate_impl(const void* x0, const float* anchors, const
     const bool pdl = programmatic();
     const long long n_tokens = (long long)n_img * t_e;
     const int32_t prep_anchors = prepared ? 0 : m_e;  // prepared anchors: the launch takes the tokens only
-    const long long prep_warps = prep_anchors + (n_tokens + civic::kPrepRows - 1) / civic::kPrepRows;
+    const int rows_per_warp = 32 / civic::kPrepLanes;
+    const long long prep_warps = prep_anchors + (n_tokens + rows_per_warp - 1) / rows_per_warp;  // an anchor per warp
     CIVIC_CUDA_TRY(civic::launch(pdl, civic::aggregate_prep_kernel, (unsigned)((prep_warps + 7) / 8), 256u, 0,
                                  stream, anchors, prep_anchors, (const __nv_bfloat16*)x0, n_tokens, d_v, 1e-5f, 1e-12f, q,
                                  qsum, stats, (int*)device_status));  // also clears the status word
